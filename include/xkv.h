@@ -1,0 +1,229 @@
+/*
+ * xkv.h -- C ABI of libxkv: the data-parallel hot path of XKV (personalised per-layer
+ * KV-cache budgets) on one NVIDIA B200 (sm_100a).
+ *
+ * The path, in call order:
+ *   1. xkv_score          per layer: observation-window attention weights -> pooled importance
+ *                         scores per KV head, their descending sort, and the layer's
+ *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
+ *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
+ *   3. xkv_select_compact per layer: top-k per (sequence, KV head) and gather of the kept K/V
+ *                         rows into a ragged paged cache                             (Alg. 2 steps 5-7)
+ *   4. xkv_decode_attn    per generation step: attention over the ragged compacted caches,
+ *                         new K/V appended first                                     (Eq. 1; Sec. IV-A, generation phase)
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C types only. "dev" = pointer to device memory of the current CUDA device,
+ *     "host" = pointer to host memory. bf16 = IEEE bfloat16 stored as uint16_t bit patterns.
+ *   - The caller owns every buffer (inputs, outputs, cache pages, workspace). The library
+ *     allocates nothing, frees nothing and never synchronises the stream; work is enqueued on
+ *     `stream` (a cudaStream_t passed as void*, NULL = default stream).
+ *   - Device pointers must be 16-byte aligned; violations are rejected with XKV_ERR_INVALID_ARG.
+ *   - Arguments are validated on the host and rejected before anything is enqueued. A negative
+ *     return value means nothing was launched. Conditions only the device can see (a cache slot
+ *     beyond its page table, a bounded wait that expired) are recorded in a status word at the
+ *     start of the workspace; read it with xkv_read_device_status after the call.
+ *   - Sequences are packed: token c of sequence b is row cu_seqlens[b] + c. t_b = cu_seqlens[b+1]
+ *     - cu_seqlens[b] is the prompt length, W = dims.window, P_b = max(t_b - W, 0) the prefix
+ *     length (the tokens that can be evicted); the last min(W, t_b) tokens are always kept.
+ *   - G = n_q_heads / n_kv_heads query heads share KV head g = h / G.
+ */
+#ifndef XKV_H_
+#define XKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t xkv_status;
+#define XKV_OK               0
+#define XKV_ERR_INVALID_ARG (-1) /* null/misaligned pointer, non-positive size, inconsistent dims    */
+#define XKV_ERR_UNSUPPORTED (-2) /* head_dim not in {64,128}, G*W not a multiple of 16 or > 256, ... */
+#define XKV_ERR_WORKSPACE   (-3) /* workspace_bytes smaller than xkv_workspace_bytes() reports        */
+#define XKV_ERR_BUDGET      (-4) /* negative budget, total beyond capacity, unreachable R target      */
+#define XKV_ERR_CUDA        (-5) /* a CUDA runtime/driver call or a launch failed                     */
+#define XKV_ERR_TIMEOUT     (-6) /* device status: a bounded wait inside a kernel expired             */
+#define XKV_ERR_CAPACITY    (-7) /* device status: a sequence outgrew its page table                  */
+
+#define XKV_POOL_MAX 0
+#define XKV_POOL_AVG 1
+
+#define XKV_OP_SCORE          0
+#define XKV_OP_SELECT_COMPACT 1
+#define XKV_OP_DECODE_ATTN    2
+
+/* Problem shape shared by the device entry points. */
+typedef struct xkv_dims {
+  int32_t batch;         /* B, number of sequences                                            */
+  int32_t n_q_heads;     /* Hq                                                                 */
+  int32_t n_kv_heads;    /* Hkv, divides Hq                                                    */
+  int32_t head_dim;      /* d, 64 or 128                                                       */
+  int32_t window;        /* W = ows, observation-window size (Eq. 3); G*W multiple of 16, <=256 */
+  int32_t pool_kernel;   /* ps, odd, 1..63 (Alg. 2 step 4); 1 = no pooling                     */
+  int32_t pool_mode;     /* XKV_POOL_MAX or XKV_POOL_AVG                                       */
+  float   scale;         /* logit scale; 0 selects 1/sqrt(d) (Eq. 2)                           */
+  int64_t kv_stride_token; /* elements between consecutive tokens of k and v (>= Hkv*d, mult. of 8) */
+  int64_t kv_stride_head;  /* elements between KV heads of one token (>= d, mult. of 8)        */
+} xkv_dims;
+
+/*
+ * The ragged paged cache of all layers (the reduced caches of Sec. IV-A whose sizes differ per layer).
+ * A page holds page_size consecutive cache slots of every KV head:
+ *   k_pages / v_pages : dev bf16 [n_pages][Hkv][page_size][d]
+ *   block_table       : dev int32 [n_layers][B][max_pages_per_seq], page ids, filled by the caller;
+ *                       slot s of (layer, b) lives in page block_table[layer][b][s / page_size]
+ *   seq_lens          : dev int32 [n_layers][B], number of filled slots; written by
+ *                       xkv_select_compact, advanced by xkv_decode_attn when it appends
+ * page_size is a multiple of 16 (at most 256).
+ */
+typedef struct xkv_cache {
+  void*    k_pages;
+  void*    v_pages;
+  int32_t* block_table;
+  int32_t* seq_lens;
+  int32_t  n_layers;
+  int32_t  page_size;
+  int32_t  max_pages_per_seq;
+  int32_t  n_pages;
+} xkv_cache;
+
+/*
+ * xkv_score -- importance scoring of one layer (Eq. 2, Eq. 3; Alg. 2 steps 1-4; Eq. 4).
+ *
+ * For every sequence b and KV head g:
+ *   a[h,r,c] = softmax over the visible keys c <= P_b + r of scale * q_win[b,h,r,:] . k[c,g,:]
+ *              (the model's causal attention weights of the last W tokens, Eq. 2)
+ *   u[c]     = sum over the G query heads h of group g and the W window rows r of a[h,r,c], c < P_b
+ *              (the ows x (t-ows) block, reduced along its first dimension)
+ *   w[c]     = 1-D pooling of u, stride 1, same length, centred kernel ps:
+ *              max over the part of the kernel inside [0, P_b)   (XKV_POOL_MAX), or
+ *              sum over that part divided by ps                   (XKV_POOL_AVG, zero padding)
+ *   sorted   = w in descending order
+ *   gains[b][j] = mean over g of sorted[g][j] / sum_c w[c]   (0 for j >= P_b): the increase of the
+ *              layer's retained-importance ratio R (Eq. 4) when every head keeps one more token;
+ *   mass[b][n]  = sum_{j<=n} gains[b][j] = R at n+1 kept tokens.
+ *
+ * q_win      dev bf16 [B][Hq][W][d]; row r is the query of position t_b - W + r. Sequences shorter
+ *            than W use rows W - t_b .. W-1 only.
+ * k          dev bf16, token row cu_seqlens[b]+c, head g at element offset
+ *            (cu_seqlens[b]+c)*kv_stride_token + g*kv_stride_head
+ * cu_seqlens dev int32 [B+1], non-decreasing, cu_seqlens[0] = 0, cu_seqlens[B] = total_tokens
+ * total_tokens, max_seqlen  host values: T and an upper bound of every t_b
+ * scores     dev out fp32 [Hkv][T]: w at column cu_seqlens[b]+c for c < P_b; window columns are 0
+ * sorted     dev out fp32 [Hkv][T]: per (g, b) the P_b values of w in descending order at columns
+ *            cu_seqlens[b] .. cu_seqlens[b]+P_b-1; window columns are 0. NULL skips the sort and
+ *            the curves (gains and mass are then not written).
+ * gains      dev out fp32 [B][curve_len]
+ * mass       dev out fp32 [B][curve_len], may be NULL
+ * curve_len  number of ranks reported, >= 1
+ * workspace  dev, at least xkv_workspace_bytes(XKV_OP_SCORE, ...) bytes, 256-byte aligned
+ */
+xkv_status xkv_score(const xkv_dims* dims, const void* q_win, const void* k,
+                     const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen,
+                     float* scores, float* sorted, float* gains, float* mass, int32_t curve_len,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * xkv_alloc_budgets -- Algorithm 1 (adaptive allocation), host only, no CUDA call.
+ *
+ * gains      host fp32 [n_layers][batch][curve_len] as written by xkv_score, layer by layer
+ * prefix_len host int32 [batch], P_b; a layer can hold at most max_b P_b (or n_max) tokens per head
+ * per_sequence 0: one list for the batch from the mean over b of the gains (budgets [n_layers]);
+ *              1: one list per sequence (budgets [batch][n_layers]), sequence b capped at P_b
+ * total      N = sum of the per-layer budgets to hand out (Eq. 17). If total < 0 the R_avg mode
+ *            of Eq. 18 runs instead: hand out slots until mean-over-layers retained ratio
+ *            reaches r_target (in (0,1]).
+ * n_min,n_max box per layer: every layer starts at n_min and stops at n_max
+ *            (n_max <= 0 means no upper bound other than the capacity, n_min 0 = the paper's form)
+ * budgets    host out int32
+ * r_avg      host out double [1] or [batch]: the mean over layers of the retained ratio reached
+ *
+ * Each iteration grants one slot to the layer whose next-largest normalised score is largest;
+ * ties go to the lowest layer index. Errors: XKV_ERR_BUDGET if total exceeds the summed
+ * capacities (or is below n_layers*n_min), or r_target is not reachable.
+ */
+xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch,
+                             int32_t curve_len, const int32_t* prefix_len, int32_t per_sequence,
+                             int64_t total, double r_target, int32_t n_min, int32_t n_max,
+                             int32_t* budgets, double* r_avg);
+
+/*
+ * xkv_select_compact -- top-k and eviction of one layer (Alg. 2 steps 5-7).
+ *
+ * For every (b, g): keep the kb = min(budget, P_b) prefix positions with the largest w, ordered by
+ * (score descending, position ascending) so that among equal scores the lower position is kept,
+ * plus all window positions P_b .. t_b-1. The kept positions, in ascending order, are copied
+ * bit-exactly from k and v into cache slots 0 .. kb + (t_b - P_b) - 1 of (layer, b) and
+ * seq_lens[layer][b] is set to that count.
+ *
+ * budget     host int32 [1] (per_sequence = 0) or [B] (per_sequence = 1), each >= 0
+ * scores     dev fp32 [Hkv][T] (w of xkv_score, or any non-negative finite scores)
+ * sorted     dev fp32 [Hkv][T] (descending per (g,b), as xkv_score writes it)
+ * k, v       dev bf16, same layout and strides (dims.kv_stride_*)
+ * sel        dev out int32 [B][Hkv][sel_stride], may be NULL: the kept positions in cache order;
+ *            sel_stride >= min(budget, max_seqlen) + W
+ * workspace  dev, at least xkv_workspace_bytes(XKV_OP_SELECT_COMPACT, ...) bytes
+ * Device status XKV_ERR_CAPACITY if a sequence needs more than max_pages_per_seq pages
+ * (nothing is copied for that sequence and its seq_lens entry is set to 0).
+ */
+xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t* budget,
+                              int32_t per_sequence, const float* scores, const float* sorted,
+                              const void* k, const void* v, const int32_t* cu_seqlens,
+                              int64_t total_tokens, int32_t max_seqlen, const xkv_cache* cache,
+                              int32_t* sel, int32_t sel_stride,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * xkv_decode_attn -- one generation step of attention over the reduced caches of layers
+ * [layer_begin, layer_end) (Eq. 1 with one query row per head; Sec. IV-A generation phase).
+ *
+ * If k_new and v_new are given, row (l, b, g) is first appended to slot seq_lens[l][b] of the cache
+ * and seq_lens[l][b] advances by one (newly generated tokens are stored too and never evicted).
+ * Then for every query head h:  out[l,b,h,:] = softmax_c(scale * q[l,b,h,:] . K_c) V_c  over all
+ * n filled slots c of (l, b) and KV head h / G, computed with fp32 accumulation in chunks of
+ * cache rows whose partial results are merged by log-sum-exp.
+ *
+ * q          dev bf16 [Lr][B][Hq][d], Lr = layer_end - layer_begin
+ * k_new,v_new dev bf16 [Lr][B][Hkv][d], both NULL or both given
+ * out        dev out bf16 [Lr][B][Hq][d]; rows of empty caches (n = 0) are zero
+ * lse        dev out fp32 [Lr][B][Hq], may be NULL: natural-log sum of exp of the scaled logits
+ * chunk_rows 0 = chosen on the device from the cache lengths; otherwise a multiple of 64
+ * workspace  dev, at least xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...) bytes
+ * Device status XKV_ERR_CAPACITY if an append does not fit its page table (that row is skipped).
+ */
+xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin,
+                           int32_t layer_end, const void* q, const void* k_new, const void* v_new,
+                           void* out, float* lse, int32_t chunk_rows,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Workspace size in bytes for one call of `op` (XKV_OP_*). Unused arguments may be 0.
+ *   XKV_OP_SCORE, XKV_OP_SELECT_COMPACT: dims, max_seqlen, total_tokens
+ *   XKV_OP_DECODE_ATTN: dims, n_layers (layers per call), max_cache_len (upper bound of any
+ *                       seq_lens entry, e.g. max_pages_per_seq*page_size), chunk_rows as passed
+ * Returns 0 for invalid arguments.
+ */
+size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen,
+                           int64_t total_tokens, int32_t n_layers, int32_t max_cache_len,
+                           int32_t chunk_rows);
+
+/*
+ * Copies the device status word of `workspace` to the host, waits for `stream`, and returns it:
+ * XKV_OK, or the first XKV_ERR_* a kernel of the last call on that workspace recorded.
+ * This is the only entry point that synchronises.
+ */
+xkv_status xkv_read_device_status(const void* workspace, void* stream);
+
+/* Number of kernel launches the library enqueued since it was loaded (all entry points). */
+int64_t xkv_launch_count(void);
+
+const char* xkv_status_string(xkv_status status);
+int32_t xkv_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XKV_H_ */

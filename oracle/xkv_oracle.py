@@ -1,0 +1,347 @@
+"""CPU oracle for the XKV hot path -- TEST INFRASTRUCTURE, not part of the product.
+
+Plain, slow, fp64 numpy restatement of what the paper's method computes, step by step and in the
+paper's notation.  Only the tests, the smoke check and the CPU-baseline leg of the benchmark may
+import it; the CUDA library never does, and nothing here imports the CUDA library.  No blocking,
+fusion or reordering beyond what the cited passage states.
+
+Inputs are the same bf16 tensors the GPU path receives, widened exactly to float64 by the caller.
+
+Readings of the paper used here (each is the place where the paper is silent or garbled):
+  * Merge sums over the window rows instead of averaging them (a constant factor: same ranking,
+    same retention ratio R).
+  * With grouped-query attention the window-summed weights of the G query heads that share one
+    KV head are added before pooling; scores, selection and caches are per KV head.
+  * Pooling has stride 1, keeps the length, the kernel is centred; max-pooling clips the kernel to
+    the prefix, average-pooling pads with zeros and always divides by ps.
+  * n_i counts prefix tokens only; the ows window tokens are always kept in addition.
+  * TopK orders by (score descending, position ascending).
+  * A layer's curve is the rank-wise mean over its heads of each head's sorted, self-normalised
+    scores (for one head this is exactly Sort(w_i)/Sum(w_i) of Eq. 21).
+  * Algorithm 1's wait value of a layer that holds pos slots is its (pos+1)-th largest normalised
+    score (Eq. 21); the listing's slice expression is garbled.  Max(List_W) ties go to the lowest
+    layer index.
+  * Generation appends the new token's K/V first and then attends over all cached rows.
+
+Parity pins live in tests/test_oracle_*.py; every function below is pinned there except where its
+docstring says "parity unpinned".
+"""
+from __future__ import annotations
+
+import itertools
+import math
+
+import numpy as np
+
+NEG_INF = -np.inf
+
+
+# ----------------------------------------------------------------------------------------------
+# Alg. 2 step 1 / Eq. 2: attention weights
+# ----------------------------------------------------------------------------------------------
+def softmax_rows(S: np.ndarray) -> np.ndarray:
+    """Row-wise softmax with the usual max subtraction; -inf entries get weight 0."""
+    S = np.asarray(S, dtype=np.float64)
+    m = np.max(S, axis=-1, keepdims=True)
+    E = np.exp(S - m)
+    return E / np.sum(E, axis=-1, keepdims=True)
+
+
+def attention_weights(Q: np.ndarray, K: np.ndarray, scale: float | None = None) -> np.ndarray:
+    """Eq. 2: W_attn = softmax(Q K^T / sqrt(d_k)) of a causal model, full t x t matrix.
+
+    Q, K: [t, d].  Row i sees keys 0..i.
+    """
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    t, d = K.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    S = (Q @ K.T) * scale
+    mask = np.tril(np.ones((t, t), dtype=bool))
+    S = np.where(mask, S, NEG_INF)
+    return softmax_rows(S)
+
+
+def window_attention_weights(Q_win: np.ndarray, K: np.ndarray, scale: float | None = None) -> np.ndarray:
+    """The last ows rows of Eq. 2's matrix, computed from the window queries alone.
+
+    Q_win: [ows, d] queries of positions t-ows .. t-1;  K: [t, d].  Returns [ows, t]; row r sees
+    keys c <= t - ows + r.  If t < ows only the last t rows are meaningful; earlier rows are 0.
+    """
+    Q_win = np.asarray(Q_win, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    ows, d = Q_win.shape
+    t = K.shape[0]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    out = np.zeros((ows, t), dtype=np.float64)
+    for r in range(ows):
+        pos = t - ows + r            # position of this query in the sequence
+        if pos < 0:
+            continue
+        s = (K[: pos + 1] @ Q_win[r]) * scale
+        out[r, : pos + 1] = softmax_rows(s[None, :])[0]
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# Alg. 2 steps 2-4 / Eq. 3: the attention-processing module f
+# ----------------------------------------------------------------------------------------------
+def select(W_rows: np.ndarray, ows: int) -> np.ndarray:
+    """Alg. 2 step 2: rows of the last ows tokens, columns of the first t-ows tokens.
+
+    W_rows holds the last ows rows of W_attn ([ows, t]).  Returns [ows, max(t-ows, 0)].
+    """
+    t = W_rows.shape[1]
+    P = max(t - ows, 0)
+    return W_rows[:, :P]
+
+
+def merge(block: np.ndarray) -> np.ndarray:
+    """Alg. 2 step 3: reduce the ows x (t-ows) block along its first dimension (sum)."""
+    return np.sum(block, axis=0)
+
+
+def pooling(u: np.ndarray, ps: int, mode: str = "max") -> np.ndarray:
+    """Alg. 2 step 4: 1-D pooling, stride 1, same length, centred kernel of size ps (odd)."""
+    u = np.asarray(u, dtype=np.float64)
+    assert ps >= 1 and ps % 2 == 1
+    P = u.shape[0]
+    half = ps // 2
+    w = np.empty(P, dtype=np.float64)
+    for c in range(P):
+        lo = max(c - half, 0)
+        hi = min(c + half, P - 1)
+        if mode == "max":
+            w[c] = np.max(u[lo: hi + 1])
+        elif mode == "avg":
+            w[c] = np.sum(u[lo: hi + 1]) / ps
+        else:
+            raise ValueError(mode)
+    return w
+
+
+def column_scores(Q_win_group: np.ndarray, K: np.ndarray, ows: int, scale: float | None = None) -> np.ndarray:
+    """Select + Merge for one KV head: u[c] = sum over the group's query heads and window rows.
+
+    Q_win_group: [G, ows, d] (the G query heads sharing this KV head);  K: [t, d].  Returns [t-ows].
+    """
+    t = K.shape[0]
+    P = max(t - ows, 0)
+    u = np.zeros(P, dtype=np.float64)
+    for Qh in Q_win_group:
+        u += merge(select(window_attention_weights(Qh, K, scale), ows))
+    return u
+
+
+def score_vector(Q_win_group: np.ndarray, K: np.ndarray, ows: int, ps: int, mode: str = "max",
+                 scale: float | None = None) -> np.ndarray:
+    """Eq. 3: w = f(W_attn, ows) for one KV head -- Select, Merge, Pooling."""
+    return pooling(column_scores(Q_win_group, K, ows, scale), ps, mode)
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 4: importance-retention ratio, and the curves Algorithm 1 consumes
+# ----------------------------------------------------------------------------------------------
+def sort_descending(w: np.ndarray) -> np.ndarray:
+    return np.sort(np.asarray(w, dtype=np.float64))[::-1]
+
+
+def retention_ratio(w: np.ndarray, n: int) -> float:
+    """Eq. 4 as a fraction: R = Sum(TopK(n, w)) / Sum(w)."""
+    w = np.asarray(w, dtype=np.float64)
+    return float(np.sum(sort_descending(w)[:n]) / np.sum(w))
+
+
+def head_gains(w: np.ndarray) -> np.ndarray:
+    """Sort(w)[-(j+1)] / Sum(w) for j = 0..len-1 (the terms of Eq. 21); empty or all-zero w -> zeros."""
+    w = np.asarray(w, dtype=np.float64)
+    if w.size == 0:
+        return np.zeros(0, dtype=np.float64)
+    total = np.sum(w)
+    if total <= 0.0:
+        return np.zeros(w.size, dtype=np.float64)
+    return sort_descending(w) / total
+
+
+def layer_gains(w_heads: list[np.ndarray], curve_len: int) -> np.ndarray:
+    """Rank-wise mean over a layer's heads of head_gains; ranks beyond a head's length count 0."""
+    g = np.zeros(curve_len, dtype=np.float64)
+    for w in w_heads:
+        hg = head_gains(w)[:curve_len]
+        g[: hg.size] += hg
+    return g / max(len(w_heads), 1)
+
+
+def retained_mass(gains: np.ndarray) -> np.ndarray:
+    """mass[n] = sum_{j<=n} gains[j]: R after keeping n+1 tokens per head."""
+    return np.cumsum(np.asarray(gains, dtype=np.float64))
+
+
+# ----------------------------------------------------------------------------------------------
+# Algorithm 1: adaptive allocation
+# ----------------------------------------------------------------------------------------------
+def adaptive_allocation(gains: list[np.ndarray], N: int | None = None, R_avg: float | None = None,
+                        n_min: int = 0, n_max: int | None = None,
+                        capacity: list[int] | None = None) -> tuple[list[int], float]:
+    """Algorithm 1.  gains[i][j] is layer i's (j+1)-th largest normalised score.
+
+    Mode N (Eq. 17): hand out N slots.  Mode R_avg (Eq. 18): stop at the first iteration where the
+    mean over layers of the granted normalised scores reaches R_avg.
+    Returns (List_A, mean over layers of the retained ratio).
+    """
+    L = len(gains)
+    cap = [len(g) for g in gains] if capacity is None else list(capacity)
+    if n_max is not None:
+        cap = [min(c, n_max) for c in cap]
+
+    def wait_value(i: int, pos: int) -> float:
+        # normalised score of the token layer i would keep next, after holding pos slots
+        if pos >= cap[i]:
+            return NEG_INF
+        return float(gains[i][pos]) if pos < len(gains[i]) else 0.0
+
+    List_A = [min(n_min, cap[i]) for i in range(L)]
+    R_total = sum(float(np.sum(np.asarray(gains[i][: List_A[i]], dtype=np.float64))) for i in range(L))
+    List_W = [wait_value(i, List_A[i]) for i in range(L)]
+
+    def grant() -> None:
+        nonlocal R_total
+        maximum = max(List_W)
+        if maximum == NEG_INF:
+            raise ValueError("budget exceeds capacity")
+        index = List_W.index(maximum)          # first layer holding the maximum
+        List_A[index] += 1
+        R_total += maximum
+        pos = List_A[index]
+        List_W[index] = wait_value(index, pos)
+
+    if N is not None:
+        if N < sum(List_A):
+            raise ValueError("N below the n_min floor")
+        for _ in range(N - sum(List_A)):
+            grant()
+    elif R_avg is not None:
+        if not (0.0 < R_avg <= 1.0 + 1e-12):
+            raise ValueError("R_avg target out of range")
+        while R_total / L < R_avg:
+            grant()
+    else:
+        raise ValueError("give N or R_avg")
+    return List_A, R_total / L
+
+
+def allocation_objective(gains: list[np.ndarray], List_A: list[int]) -> float:
+    """Objective of Eq. 17: mean over layers of R_i(n_i)."""
+    return sum(float(np.sum(np.asarray(g[:n], dtype=np.float64))) for g, n in zip(gains, List_A)) / len(gains)
+
+
+def bruteforce_allocation(gains: list[np.ndarray], N: int, n_min: int = 0,
+                          n_max: int | None = None) -> tuple[list[int], float]:
+    """Enumerate every split of N over the layers (tiny inputs only) and return the best of Eq. 17."""
+    L = len(gains)
+    cap = [len(g) if n_max is None else min(len(g), n_max) for g in gains]
+    best, best_val = None, -1.0
+    for split in itertools.product(*[range(min(n_min, cap[i]), cap[i] + 1) for i in range(L)]):
+        if sum(split) != N:
+            continue
+        val = allocation_objective(gains, list(split))
+        if val > best_val:
+            best, best_val = list(split), val
+    if best is None:
+        raise ValueError("no feasible split")
+    return best, best_val
+
+
+def batch_mean_gains(gains_lb: np.ndarray) -> np.ndarray:
+    """gains_lb [L, B, curve_len] -> [L, curve_len]: mean over the sequences of a batch."""
+    return np.mean(np.asarray(gains_lb, dtype=np.float64), axis=1)
+
+
+# ----------------------------------------------------------------------------------------------
+# Alg. 2 steps 5-7: TopK and EvictByIndex
+# ----------------------------------------------------------------------------------------------
+def topk_indices(w: np.ndarray, n: int) -> np.ndarray:
+    """Alg. 2 step 5: positions of the n largest entries, ties to the lower position, ascending."""
+    w = np.asarray(w, dtype=np.float64)
+    P = w.shape[0]
+    n = min(max(n, 0), P)
+    order = np.lexsort((np.arange(P), -w))   # primary key: score descending; secondary: position
+    return np.sort(order[:n]).astype(np.int64)
+
+
+def kept_positions(w: np.ndarray, n: int, t: int, ows: int) -> np.ndarray:
+    """The retained positions of one head: TopK over the prefix, then the window positions."""
+    P = max(t - ows, 0)
+    assert w.shape[0] == P
+    return np.concatenate([topk_indices(w, n), np.arange(P, t, dtype=np.int64)])
+
+
+def evict_by_index(X: np.ndarray, index: np.ndarray) -> np.ndarray:
+    """Alg. 2 steps 6-7: keep the rows listed in index, in that order (any dtype, bit-exact copy)."""
+    return np.asarray(X)[np.asarray(index, dtype=np.int64)].copy()
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 1: generation-phase attention over a reduced cache
+# ----------------------------------------------------------------------------------------------
+def decode_attention(q: np.ndarray, K_c: np.ndarray, V_c: np.ndarray,
+                     scale: float | None = None) -> tuple[np.ndarray, float]:
+    """Eq. 1 for one query row: z = softmax(q K_c^T / sqrt(d_k)) V_c.  Returns (z, log-sum-exp)."""
+    q = np.asarray(q, dtype=np.float64)
+    K_c = np.asarray(K_c, dtype=np.float64)
+    V_c = np.asarray(V_c, dtype=np.float64)
+    d = q.shape[0]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    if K_c.shape[0] == 0:
+        return np.zeros(V_c.shape[1] if V_c.ndim == 2 else d, dtype=np.float64), NEG_INF
+    s = (K_c @ q) * scale
+    m = np.max(s)
+    e = np.exp(s - m)
+    return (e / np.sum(e)) @ V_c, float(m + math.log(np.sum(e)))
+
+
+# ----------------------------------------------------------------------------------------------
+# The path end to end on packed batches (same layouts the C ABI uses, numpy arrays)
+# ----------------------------------------------------------------------------------------------
+def score_layer(q_win: np.ndarray, k: np.ndarray, cu_seqlens: np.ndarray, ows: int, ps: int,
+                mode: str = "max", scale: float | None = None,
+                units: list[tuple[int, int]] | None = None) -> dict[tuple[int, int], np.ndarray]:
+    """w for the (b, g) units of one layer.  q_win [B,Hq,ows,d], k [T,Hkv,d] (float64).
+
+    Sequences shorter than ows use the last t_b query rows.
+    """
+    B, Hq = q_win.shape[0], q_win.shape[1]
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    out = {}
+    for b in range(B):
+        lo, hi = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        for g in range(Hkv):
+            if units is not None and (b, g) not in units:
+                continue
+            out[(b, g)] = score_vector(q_win[b, g * G:(g + 1) * G], k[lo:hi, g], ows, ps, mode, scale)
+    return out
+
+
+def layer_curves(w_units: dict[tuple[int, int], np.ndarray], B: int, Hkv: int,
+                 curve_len: int) -> np.ndarray:
+    """gains [B, curve_len] of one layer from all its (b, g) score vectors."""
+    return np.stack([layer_gains([w_units[(b, g)] for g in range(Hkv)], curve_len) for b in range(B)])
+
+
+def near_tie(w: np.ndarray, n: int, rel: float = 1e-5) -> bool:
+    """True if some score other than exact copies of the n-th largest lies within rel of it.
+
+    Inside that band a path that computes scores in lower precision may legitimately keep a
+    different token; outside it the kept set is unique.
+    """
+    w = np.asarray(w, dtype=np.float64)
+    P = w.shape[0]
+    if n <= 0 or n >= P:
+        return False
+    thr = sort_descending(w)[n - 1]
+    band = np.abs(w - thr) <= rel * abs(thr)
+    return bool(np.any(band & (w != thr)))

@@ -1,0 +1,180 @@
+"""Pins for the oracle's solver (Alg. 1; Eq. 17, 18, 21), TopK / EvictByIndex (Alg. 2 steps 5-7) and
+generation attention (Eq. 1): brute force, invariants, closed forms, library cross-checks."""
+import itertools
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import xkv_oracle as O
+
+
+def _random_gains(rng, L, lens, power=3.0):
+    return [O.head_gains(rng.random(n) ** power) for n in lens[:L]]
+
+
+# ------------------------------------------------------------------ Algorithm 1
+@pytest.mark.parametrize("seed", range(6))
+def test_allocation_matches_bruteforce_objective(seed):
+    rng = np.random.default_rng(seed)
+    L = int(rng.integers(2, 5))
+    lens = [int(rng.integers(3, 7)) for _ in range(L)]
+    gains = _random_gains(rng, L, lens)
+    for N in range(0, min(sum(lens), 14) + 1):
+        A, r = O.adaptive_allocation(gains, N=N)
+        assert sum(A) == N                                           # constraint of Eq. 17
+        best, best_val = O.bruteforce_allocation(gains, N)
+        assert abs(r - best_val) < 1e-13
+        assert abs(O.allocation_objective(gains, A) - r) < 1e-13
+
+
+def test_allocation_with_box_matches_bruteforce():
+    rng = np.random.default_rng(11)
+    gains = _random_gains(rng, 3, [6, 6, 6])
+    for N in range(3, 13):
+        A, r = O.adaptive_allocation(gains, N=N, n_min=1, n_max=4)
+        assert sum(A) == N and all(1 <= a <= 4 for a in A)
+        _, best_val = O.bruteforce_allocation(gains, N, n_min=1, n_max=4)
+        assert abs(r - best_val) < 1e-13
+    with pytest.raises(ValueError):
+        O.adaptive_allocation(gains, N=13, n_min=1, n_max=4)
+    with pytest.raises(ValueError):
+        O.adaptive_allocation(gains, N=2, n_min=1, n_max=4)
+
+
+def test_allocation_threshold_and_exchange_property():
+    rng = np.random.default_rng(12)
+    gains = _random_gains(rng, 5, [40, 30, 50, 20, 35])
+    N = 60
+    A, r = O.adaptive_allocation(gains, N=N)
+    granted = [gains[i][A[i] - 1] for i in range(5) if A[i] > 0]
+    waiting = [gains[i][A[i]] for i in range(5) if A[i] < len(gains[i])]
+    assert min(granted) >= max(waiting)
+    # Eq. 21: moving one slot between any two layers never increases the objective
+    for i, j in itertools.permutations(range(5), 2):
+        if A[i] < len(gains[i]) and A[j] > 0:
+            B = list(A); B[i] += 1; B[j] -= 1
+            delta = (gains[i][A[i]] - gains[j][A[j] - 1]) / 5
+            assert abs(O.allocation_objective(gains, B) - r - delta) < 1e-13
+            assert delta <= 1e-15
+
+
+def test_allocation_r_target_is_shortest_prefix_of_total_mode():
+    rng = np.random.default_rng(13)
+    gains = _random_gains(rng, 4, [25, 25, 25, 25])
+    for target in (0.2, 0.5, 0.9, 1.0):
+        A, r = O.adaptive_allocation(gains, R_avg=target)
+        n = sum(A)
+        assert r >= target
+        A_same, r_same = O.adaptive_allocation(gains, N=n)
+        assert A_same == A and abs(r_same - r) < 1e-15
+        if n > 0:
+            _, r_less = O.adaptive_allocation(gains, N=n - 1)
+            assert r_less < target
+    with pytest.raises(ValueError):
+        O.adaptive_allocation(gains, R_avg=1.5)
+
+
+def test_allocation_identical_layers_split_evenly_lowest_index_first():
+    g = O.head_gains(np.array([5.0, 4.0, 3.0, 2.0, 1.0]))
+    A, _ = O.adaptive_allocation([g, g, g], N=7)
+    assert A == [3, 2, 2]
+    A, _ = O.adaptive_allocation([g, g, g], N=15)
+    assert A == [5, 5, 5]
+
+
+def test_allocation_single_layer_and_batch_mean():
+    g = O.head_gains(np.array([1.0, 2.0, 3.0]))
+    A, r = O.adaptive_allocation([g], N=2)
+    assert A == [2] and abs(r - 5.0 / 6.0) < 1e-15
+    x = np.arange(24, dtype=np.float64).reshape(2, 3, 4)
+    assert np.allclose(O.batch_mean_gains(x), x.mean(axis=1))
+
+
+# ------------------------------------------------------------------ TopK / EvictByIndex
+def test_topk_matches_bruteforce_sort():
+    rng = np.random.default_rng(20)
+    for _ in range(20):
+        P = int(rng.integers(1, 30))
+        w = rng.integers(0, 6, size=P).astype(np.float64)          # many ties
+        for n in range(0, P + 2):
+            order = sorted(range(P), key=lambda c: (-w[c], c))
+            assert O.topk_indices(w, n).tolist() == sorted(order[: min(n, P)])
+
+
+def test_topk_special_cases():
+    assert O.topk_indices(np.full(9, 0.25), 4).tolist() == [0, 1, 2, 3]       # ties -> lowest positions
+    e = np.zeros(20); e[11] = 1.0
+    plateau = O.pooling(e, 7, "max")                                          # positions 8..14
+    assert O.topk_indices(plateau, 3).tolist() == [8, 9, 10]
+    assert O.topk_indices(plateau, 7).tolist() == list(range(8, 15))
+    assert O.topk_indices(plateau, 9).tolist() == [0, 1] + list(range(8, 15))
+    w = np.array([0.1, 0.9, 0.3])
+    assert O.topk_indices(w, 5).tolist() == [0, 1, 2] and O.topk_indices(w, 0).tolist() == []
+    assert O.kept_positions(w, 1, 5, 2).tolist() == [1, 3, 4]
+    assert O.kept_positions(np.zeros(0), 3, 2, 4).tolist() == [0, 1]          # t < ows: keep all
+
+
+def test_near_tie_band():
+    w = np.array([1.0, 0.5, 0.5 * (1 + 5e-6), 0.2, 0.5])
+    assert O.near_tie(w, 2) and O.near_tie(w, 3)
+    assert not O.near_tie(w, 1)
+    assert not O.near_tie(np.array([1.0, 0.5, 0.5, 0.2]), 2)   # exact copies are not near-ties
+    assert not O.near_tie(w, 0) and not O.near_tie(w, 5)
+
+
+def test_evict_by_index_is_bit_exact_and_full_budget_is_identity():
+    rng = np.random.default_rng(21)
+    X = rng.integers(0, 2 ** 16, size=(12, 4), dtype=np.uint16)
+    idx = np.array([0, 3, 4, 11])
+    Y = O.evict_by_index(X, idx)
+    assert Y.dtype == np.uint16 and np.array_equal(Y, X[[0, 3, 4, 11]])
+    w = rng.random(10)
+    full = O.kept_positions(w, 99, 12, 2)
+    assert np.array_equal(O.evict_by_index(X, full), X)
+
+
+# ------------------------------------------------------------------ Eq. 1 decode
+def test_decode_full_budget_reproduces_full_attention_bitwise():
+    rng = np.random.default_rng(30)
+    t, d, ows = 50, 16, 4
+    K, V, q = rng.normal(size=(t, d)), rng.normal(size=(t, d)), rng.normal(size=d)
+    w = rng.random(t - ows)
+    idx = O.kept_positions(w, t, t, ows)
+    z_full, lse_full = O.decode_attention(q, K, V)
+    z_c, lse_c = O.decode_attention(q, O.evict_by_index(K, idx), O.evict_by_index(V, idx))
+    assert np.array_equal(z_full, z_c) and lse_full == lse_c
+
+
+def test_decode_single_row_permutation_and_torch():
+    rng = np.random.default_rng(31)
+    n, d = 33, 8
+    K, V, q = rng.normal(size=(n, d)), rng.normal(size=(n, d)), rng.normal(size=d)
+    z1, _ = O.decode_attention(q, K[:1], V[:1])
+    assert np.allclose(z1, V[0], atol=1e-15)
+    z, lse = O.decode_attention(q, K, V)
+    perm = rng.permutation(n)
+    zp, lsep = O.decode_attention(q, K[perm], V[perm])
+    assert np.allclose(z, zp, atol=1e-12) and abs(lse - lsep) < 1e-12
+    s = torch.from_numpy(K) @ torch.from_numpy(q) / math.sqrt(d)
+    ref = torch.softmax(s, 0) @ torch.from_numpy(V)
+    assert np.allclose(z, ref.numpy(), atol=1e-14)
+    assert abs(lse - torch.logsumexp(s, 0).item()) < 1e-13
+    z0, lse0 = O.decode_attention(q, K[:0], V[:0])
+    assert np.all(z0 == 0) and lse0 == -np.inf
+
+
+@pytest.mark.parametrize("splits", [2, 3, 7])
+def test_decode_split_and_lse_merge_is_invariant(splits):
+    rng = np.random.default_rng(32)
+    n, d = 61, 8
+    K, V, q = rng.normal(size=(n, d)) * 3, rng.normal(size=(n, d)), rng.normal(size=d)
+    z, lse = O.decode_attention(q, K, V)
+    bounds = np.linspace(0, n, splits + 1).astype(int)
+    parts = [O.decode_attention(q, K[a:b], V[a:b]) for a, b in zip(bounds[:-1], bounds[1:])]
+    m = max(p[1] for p in parts)
+    wts = np.array([math.exp(p[1] - m) for p in parts])
+    merged = sum(wi * p[0] for wi, p in zip(wts, parts)) / wts.sum()
+    assert np.allclose(merged, z, atol=1e-12)
+    assert abs(m + math.log(wts.sum()) - lse) < 1e-12
