@@ -1,0 +1,644 @@
+// xkv_decode_attn: generation-phase attention (Eq. 1, one query row per head) over the ragged,
+// compacted per-layer caches.
+//
+// Kernels, in stream order:
+//   decode_append_kernel  one warp per (layer, sequence): store the new K/V row of every KV head in
+//                         slot seq_lens[l][b] and advance seq_lens.
+//   decode_plan_kernel    one CTA: cut every (layer, sequence, KV head) cache into chunks of rows and
+//                         write the work-item table; the chunk size is chosen from the total length.
+//   decode_attn_kernel    persistent CTAs, one producer warp + four consumer warps.  The producer
+//                         streams 64-row K and V tiles of a work item into a ring of shared-memory
+//                         stages with TMA tensor loads (16-row boxes, 128-byte swizzle) that complete
+//                         on mbarriers; each consumer warp owns 16 rows of a tile and runs online
+//                         softmax with mma.sync m16n8k16 for q.K^T and P.V (the G query heads of the
+//                         group sit on the M axis).  Chunk results are merged by log-sum-exp, by the
+//                         CTA itself when the unit has one chunk, else by the last CTA to finish a
+//                         chunk of that unit (atomic ticket, no waiting).
+// The path is HBM-bound: 4*d bytes per cached row per KV head per step.
+#include <cuda.h>
+
+#include <cmath>
+#include <mutex>
+
+#include "common.cuh"
+#include "ops.h"
+
+namespace xkv {
+
+namespace {
+
+constexpr int kTileRows = 64;        // cache rows per pipeline stage
+constexpr int kBoxRows = 16;         // rows per TMA box; page_size is a multiple of it
+constexpr int kConsumerWarps = 4;
+constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kTargetItems = 16 * 148;  // auto chunking aims at about this many extra work items
+constexpr int kMinChunkRows = 256;
+constexpr int kMaxGroup = 8;
+
+struct DecodeParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  __nv_bfloat16* out;
+  float* lse;
+  __nv_bfloat16* k_pages;
+  __nv_bfloat16* v_pages;
+  const int32_t* block_table;
+  int32_t* seq_lens;
+  int32_t layer_begin, n_layers, batch, n_q_heads, n_kv_heads, group;
+  int32_t page_size, max_pages_per_seq, n_pages;
+  int32_t chunk_rows_forced, max_items;
+  float scale_log2;
+  WorkspaceHeader* hdr;
+  int32_t* tickets;   // [n_layers*batch*n_kv_heads]
+  int2* unit_info;    // [n_layers*batch]: {first item of head 0, chunks per head}
+  int4* items;        // [max_items]: {unit e, kv head, row_begin, row_end}
+  float* part_o;      // [max_items][G][D]
+  float* part_ml;     // [max_items][G][2]
+};
+
+template <int D>
+struct Cfg {
+  static constexpr int kHalves = D / 64;                       // 128-byte swizzled column halves
+  static constexpr int kHalfBytes = kTileRows * 128;           // one half of a K or V tile
+  static constexpr int kTileBytes = kHalves * kHalfBytes;
+  static constexpr int kStageBytes = 2 * kTileBytes;           // K tile + V tile
+  static constexpr int kStages = (D == 128) ? 6 : 8;
+  static constexpr int kScratchFloats = kConsumerWarps * kMaxGroup * (D + 2);
+  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScratchFloats * 4 + 2 * kStages * 8 + 64;
+};
+
+// ---------------------------------------------------------------------------------------------
+__global__ void decode_append_kernel(DecodeParams p, int D) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int n_units = p.n_layers * p.batch;
+  if (warp >= n_units) return;
+  const int l_rel = warp / p.batch, b = warp % p.batch;
+  const int le = (p.layer_begin + l_rel) * p.batch + b;
+  const int n = p.seq_lens[le];
+  const int32_t* bt = p.block_table + (size_t)le * p.max_pages_per_seq;
+  int page = -1;
+  if (n >= 0 && n < p.max_pages_per_seq * p.page_size) page = bt[n / p.page_size];
+  if (page < 0 || page >= p.n_pages) {
+    if (lane == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
+    return;
+  }
+  const int chunks = D / 8;
+  for (int idx = lane; idx < p.n_kv_heads * chunks; idx += 32) {
+    const int h = idx / chunks, c = idx % chunks;
+    const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
+    const size_t src = ((size_t)warp * p.n_kv_heads + h) * D + c * 8;
+    *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
+    *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
+  }
+  __syncwarp();
+  if (lane == 0) p.seq_lens[le] = n + 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
+  __shared__ long long s_red[32];
+  __shared__ int s_scan[32];
+  __shared__ int s_carry;
+  __shared__ int s_chunk;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_units = p.n_layers * p.batch;
+
+  long long rows = 0;
+  for (int e = tid; e < n_units; e += blockDim.x) {
+    const int n = p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch];
+    rows += n > 0 ? n : 0;
+  }
+  for (int o = 16; o > 0; o >>= 1) rows += __shfl_xor_sync(0xffffffffu, rows, o);
+  if (lane == 0) s_red[warp] = rows;
+  __syncthreads();
+  if (tid == 0) {
+    long long total = 0;
+    for (int w = 0; w < 32; ++w) total += s_red[w];
+    total *= p.n_kv_heads;
+    int chunk = p.chunk_rows_forced;
+    if (chunk <= 0) {
+      long long c = (total + kTargetItems - 1) / kTargetItems;
+      c = (c + kTileRows - 1) / kTileRows * kTileRows;
+      if (c < kMinChunkRows) c = kMinChunkRows;
+      if (c > (1 << 30)) c = 1 << 30;
+      chunk = (int)c;
+    }
+    s_chunk = chunk;
+    s_carry = 0;
+    p.hdr->chunk_rows = chunk;
+  }
+  __syncthreads();
+  const int chunk = s_chunk;
+
+  for (int base = 0; base < n_units; base += blockDim.x) {
+    const int e = base + tid;
+    int n = 0, nc = 0;
+    if (e < n_units) {
+      n = p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch];
+      if (n < 0) n = 0;
+      nc = n == 0 ? 1 : (n + chunk - 1) / chunk;
+    }
+    int incl = nc;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int v = s_scan[lane], inc = v;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += u;
+      }
+      s_scan[lane] = inc - v;   // exclusive prefix of the warp totals
+    }
+    __syncthreads();
+    const int carry = s_carry;
+    const int excl = carry + s_scan[warp] + incl - nc;
+    if (e < n_units) {
+      const int first = excl * p.n_kv_heads;
+      p.unit_info[e] = make_int2(first, nc);
+      if (first + nc * p.n_kv_heads <= p.max_items) {
+        for (int h = 0; h < p.n_kv_heads; ++h)
+          for (int c = 0; c < nc; ++c) {
+            const int rb = c * chunk;
+            const int re = min(n, rb + chunk);
+            p.items[first + h * nc + c] = make_int4(e, h, rb, re);
+          }
+      }
+    }
+    __syncthreads();
+    if (tid == blockDim.x - 1) s_carry = excl + nc;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const int n_items = s_carry * p.n_kv_heads;
+    if (n_items > p.max_items) {
+      record_status(p.hdr, XKV_ERR_WORKSPACE);
+      p.hdr->n_items = 0;
+    } else {
+      p.hdr->n_items = n_items;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: two seconds of wall time at most.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (int i = 0; i < 128; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (global_timer_ns() - t0 > 2000000000ull) return false;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(kDecodeThreads, 1)
+decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                   const DecodeParams p) {
+  using C = Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* stages = smem;
+  float* scratch = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + C::kScratchFloats);
+  uint64_t* empty_bar = full_bar + C::kStages;
+  int* s_flag = reinterpret_cast<int*>(empty_bar + C::kStages);
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], kConsumerWarps);
+    }
+    fence_mbar_init();
+    prefetch_tmap(&tmap_k);
+    prefetch_tmap(&tmap_v);
+  }
+  __syncthreads();
+
+  const int n_items = p.hdr->n_items;
+  const int chunk_rows = p.hdr->chunk_rows;
+  (void)chunk_rows;
+
+  if (warp == kConsumerWarps) {
+    // ------------------------------------------------------------------ producer warp
+    uint32_t it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      const int4 I = p.items[item];
+      const int e = I.x, h = I.y;
+      const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
+      const int32_t* bt = p.block_table + (size_t)le * p.max_pages_per_seq;
+      for (int r0 = I.z; r0 < I.w; r0 += kTileRows, ++it) {
+        const int s = it % C::kStages;
+        const uint32_t ph = (it / C::kStages) & 1u;
+        const int valid = min(kTileRows, I.w - r0);
+        const int nbox = (valid + kBoxRows - 1) / kBoxRows;
+        int grow = 0;
+        if (lane < nbox) {
+          const int slot = r0 + kBoxRows * lane;
+          int page = bt[slot / p.page_size];
+          page = min(max(page, 0), p.n_pages - 1);
+          grow = (page * p.n_kv_heads + h) * p.page_size + slot % p.page_size;
+        }
+        if (lane == 0) {
+          ok = mbar_wait_bounded(&empty_bar[s], ph ^ 1u);
+          if (ok) mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(nbox * kBoxRows * D * 2 * 2));
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        if (lane < nbox) {
+          uint8_t* ks = stages + (size_t)s * C::kStageBytes;
+          uint8_t* vs = ks + C::kTileBytes;
+#pragma unroll
+          for (int hf = 0; hf < C::kHalves; ++hf) {
+            tma_load_2d(ks + hf * C::kHalfBytes + lane * kBoxRows * 128, &tmap_k, hf * 64, grow, &full_bar[s]);
+            tma_load_2d(vs + hf * C::kHalfBytes + lane * kBoxRows * 128, &tmap_v, hf * 64, grow, &full_bar[s]);
+          }
+        }
+      }
+    }
+    if (!ok) {
+      if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+      // let copies already issued land before the CTA's shared memory can be handed on
+      for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- consumer warps
+  const int gid = lane >> 2, tig = lane & 3;
+  const int mat = lane >> 3, mrow = lane & 7;
+  const int G = p.group;
+  const int ctid = tid;  // 0..127
+  uint32_t it = 0;
+  bool aborted = false;
+  float* scr_o = scratch;                                        // [4][8][D]
+  float* scr_ml = scratch + kConsumerWarps * kMaxGroup * D;      // [4][8][2]
+
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int4 I = p.items[item];
+    const int e = I.x, h = I.y;
+    const size_t q_row0 = ((size_t)e * p.n_q_heads + (size_t)h * G);
+
+    uint32_t qa[D / 16][2];
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      qa[ks][0] = 0u;
+      qa[ks][1] = 0u;
+      if (gid < G) {
+        const __nv_bfloat16* qp = p.q + (q_row0 + gid) * D + 16 * ks + 2 * tig;
+        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
+        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
+      }
+    }
+    float o[D / 8][2];
+#pragma unroll
+    for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = 0.f;
+    float m_run = -INFINITY, l_part = 0.f;
+
+    for (int r0 = I.z; r0 < I.w; r0 += kTileRows, ++it) {
+      const int s = it % C::kStages;
+      const uint32_t ph = (it / C::kStages) & 1u;
+      const int valid = min(kTileRows, I.w - r0);
+      if (!aborted && !mbar_wait_bounded(&full_bar[s], ph)) {
+        aborted = true;
+        if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+      }
+      const int wrows = valid - kBoxRows * warp;
+      bool touched = false;
+      if (!aborted && wrows > 0) {
+        const uint32_t ks_base = smem_u32(stages + (size_t)s * C::kStageBytes);
+        const uint32_t vs_base = ks_base + C::kTileBytes;
+        if (wrows < kBoxRows) {
+          // rows past the end of the cache hold whatever the page held: clear V so 0 * x stays 0
+          uint8_t* vs = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
+          const int n_bad = kBoxRows - wrows;
+          for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
+            const int row = kBoxRows * warp + wrows + idx / (D / 8);
+            const int c = idx % (D / 8);
+            *reinterpret_cast<uint4*>(vs + (c >> 3) * C::kHalfBytes + row * 128 + (c & 7) * 16) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+          touched = true;
+          __syncwarp();
+        }
+        // S[heads x 16 keys] = Q K^T
+        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const int key = kBoxRows * warp + (mat >> 1) * 8 + mrow;
+          const int c = 2 * ks + (mat & 1);
+          const uint32_t addr = ks_base + (c >> 3) * C::kHalfBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
+          uint32_t bfrag[4];
+          ldmatrix_x4(bfrag, addr);
+          const uint32_t a[4] = {qa[ks][0], 0u, qa[ks][1], 0u};
+          mma_bf16_16816(sacc[0], a, bfrag[0], bfrag[1]);
+          mma_bf16_16816(sacc[1], a, bfrag[2], bfrag[3]);
+        }
+        float s2[2][2];
+        float mt = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const bool in = (8 * nt + 2 * tig + j) < wrows;
+            s2[nt][j] = in ? sacc[nt][j] * p.scale_log2 : -INFINITY;
+            mt = fmaxf(mt, s2[nt][j]);
+          }
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+        const float m_new = fmaxf(m_run, mt);
+        const float alpha = fast_exp2(m_run - m_new);
+        float pr[2][2];
+        float psum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            pr[nt][j] = fast_exp2(s2[nt][j] - m_new);
+            psum += pr[nt][j];
+          }
+        l_part = l_part * alpha + psum;
+        m_run = m_new;
+#pragma unroll
+        for (int nt = 0; nt < D / 8; ++nt) {
+          o[nt][0] *= alpha;
+          o[nt][1] *= alpha;
+        }
+        const uint32_t pa[4] = {pack_bf16(pr[0][0], pr[0][1]), 0u, pack_bf16(pr[1][0], pr[1][1]), 0u};
+#pragma unroll
+        for (int dp = 0; dp < D / 16; ++dp) {
+          const int key = kBoxRows * warp + (mat & 1) * 8 + mrow;
+          const int c = 2 * dp + (mat >> 1);
+          const uint32_t addr = vs_base + (c >> 3) * C::kHalfBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
+          uint32_t bfrag[4];
+          ldmatrix_x4_trans(bfrag, addr);
+          float c0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
+          float c1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
+          mma_bf16_16816(c0, pa, bfrag[0], bfrag[1]);
+          mma_bf16_16816(c1, pa, bfrag[2], bfrag[3]);
+          o[2 * dp][0] = c0[0];
+          o[2 * dp][1] = c0[1];
+          o[2 * dp + 1][0] = c1[0];
+          o[2 * dp + 1][1] = c1[1];
+        }
+      }
+      if (touched) fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty_bar[s]);
+    }
+
+    // ---- merge the four warps' partial results of this work item
+    float l_row = l_part;
+    l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
+    l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
+    if (gid < G) {
+#pragma unroll
+      for (int nt = 0; nt < D / 8; ++nt)
+        *reinterpret_cast<float2*>(&scr_o[(warp * kMaxGroup + gid) * D + 8 * nt + 2 * tig]) =
+            make_float2(o[nt][0], o[nt][1]);
+      if (tig == 0) {
+        scr_ml[(warp * kMaxGroup + gid) * 2 + 0] = m_run;
+        scr_ml[(warp * kMaxGroup + gid) * 2 + 1] = l_row;
+      }
+    }
+    named_bar_sync(1, kConsumerWarps * 32);
+
+    const int nc = p.unit_info[e].y;
+    for (int idx = ctid; idx < G * D; idx += kConsumerWarps * 32) {
+      const int g = idx / D, dc = idx % D;
+      float mmax = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kConsumerWarps; ++w) mmax = fmaxf(mmax, scr_ml[(w * kMaxGroup + g) * 2]);
+      float num = 0.f, den = 0.f;
+      if (mmax > -INFINITY) {
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+          const float a = fast_exp2(scr_ml[(w * kMaxGroup + g) * 2] - mmax);
+          num += a * scr_o[(w * kMaxGroup + g) * D + dc];
+          den += a * scr_ml[(w * kMaxGroup + g) * 2 + 1];
+        }
+      }
+      if (nc == 1) {
+        const size_t row = q_row0 + g;
+        p.out[row * D + dc] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+        if (dc == 0 && p.lse != nullptr)
+          p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
+      } else {
+        p.part_o[((size_t)item * G + g) * D + dc] = num;
+        if (dc == 0) {
+          p.part_ml[((size_t)item * G + g) * 2 + 0] = mmax;
+          p.part_ml[((size_t)item * G + g) * 2 + 1] = den;
+        }
+      }
+    }
+    if (nc > 1) {
+      __threadfence();
+      named_bar_sync(1, kConsumerWarps * 32);
+      if (ctid == 0) {
+        const int old = atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1);
+        *s_flag = (old == nc - 1) ? 1 : 0;
+      }
+      named_bar_sync(1, kConsumerWarps * 32);
+      if (*s_flag) {
+        __threadfence();
+        const int first = p.unit_info[e].x + h * nc;
+        for (int idx = ctid; idx < G * D; idx += kConsumerWarps * 32) {
+          const int g = idx / D, dc = idx % D;
+          float mmax = -INFINITY;
+          for (int c = 0; c < nc; ++c) mmax = fmaxf(mmax, __ldcg(&p.part_ml[((size_t)(first + c) * G + g) * 2]));
+          float num = 0.f, den = 0.f;
+          if (mmax > -INFINITY) {
+            for (int c = 0; c < nc; ++c) {
+              const size_t pi = (size_t)(first + c) * G + g;
+              const float a = fast_exp2(__ldcg(&p.part_ml[pi * 2]) - mmax);
+              num += a * __ldcg(&p.part_o[pi * D + dc]);
+              den += a * __ldcg(&p.part_ml[pi * 2 + 1]);
+            }
+          }
+          const size_t row = q_row0 + g;
+          p.out[row * D + dc] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
+          if (dc == 0 && p.lse != nullptr)
+            p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
+        }
+        if (ctid == 0) p.tickets[e * p.n_kv_heads + h] = 0;
+      }
+    }
+    named_bar_sync(1, kConsumerWarps * 32);   // scratch and flag are reused by the next item
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (enc == nullptr) return false;
+  const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)kBoxRows};
+  const cuuint32_t estr[2] = {1u, 1u};
+  return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DecodeLayout {
+  size_t tickets, unit_info, items, part_o, part_ml, total;
+  int64_t max_items;
+};
+
+bool decode_layout(const xkv_dims* d, int n_layers, int max_cache_len, int chunk_rows, DecodeLayout* L) {
+  if (n_layers <= 0 || d->batch <= 0 || d->n_kv_heads <= 0) return false;
+  const int64_t lb = (int64_t)n_layers * d->batch;
+  const int64_t units = lb * d->n_kv_heads;
+  int64_t max_items;
+  if (chunk_rows > 0) {
+    const int64_t per = max_cache_len > 0 ? ((int64_t)max_cache_len + chunk_rows - 1) / chunk_rows : 1;
+    max_items = units * (per > 0 ? per : 1);
+  } else {
+    max_items = units + (int64_t)(kTargetItems + 1) * 1;
+    // ceil() adds at most one item per unit, the rows themselves at most kTargetItems
+    max_items += 0;
+  }
+  if (max_items > (int64_t)1 << 28) return false;
+  const int G = d->n_q_heads / d->n_kv_heads;
+  size_t off = kHeaderBytes;
+  L->tickets = off;   off = align_up(off + (size_t)units * 4, 256);
+  L->unit_info = off; off = align_up(off + (size_t)lb * 8, 256);
+  L->items = off;     off = align_up(off + (size_t)max_items * 16, 256);
+  L->part_o = off;    off = align_up(off + (size_t)max_items * G * d->head_dim * 4, 256);
+  L->part_ml = off;   off = align_up(off + (size_t)max_items * G * 2 * 4, 256);
+  L->total = off;
+  L->max_items = max_items;
+  return true;
+}
+
+template <int D>
+xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, cudaStream_t st) {
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  // opt in to the large dynamic shared-memory carve-out once per process and device in use
+  int dev = 0;
+  cudaGetDevice(&dev);
+  static bool done[64] = {};
+  if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
+  if (!done[dev]) {
+    attr_err = cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    Cfg<D>::kSmemBytes);
+    if (attr_err != cudaSuccess) return XKV_ERR_CUDA;
+    done[dev] = true;
+  }
+  (void)once;
+  decode_attn_kernel<D><<<sm_count(), kDecodeThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
+  count_launch();
+  return check_launch();
+}
+
+}  // namespace
+
+size_t decode_workspace_bytes(const xkv_dims* d, int n_layers, int max_cache_len, int chunk_rows) {
+  DecodeLayout L;
+  if (!decode_layout(d, n_layers, max_cache_len, chunk_rows, &L)) return 0;
+  return L.total;
+}
+
+xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end, const void* q,
+                       const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,
+                       void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  const int Lr = layer_end - layer_begin;
+  const int G = d->n_q_heads / d->n_kv_heads;
+  if (G > kMaxGroup) return XKV_ERR_UNSUPPORTED;
+  if (chunk_rows < 0 || chunk_rows % kTileRows != 0) return XKV_ERR_INVALID_ARG;
+  const int max_cache_len = c->max_pages_per_seq * c->page_size;
+  DecodeLayout L;
+  if (!decode_layout(d, Lr, max_cache_len, chunk_rows, &L)) return XKV_ERR_INVALID_ARG;
+  if (workspace_bytes < L.total) return XKV_ERR_WORKSPACE;
+  const uint64_t page_rows = (uint64_t)c->n_pages * d->n_kv_heads * c->page_size;
+  if (page_rows >= (1ull << 31)) return XKV_ERR_UNSUPPORTED;
+
+  CUtensorMap tk, tv;
+  if (!make_page_tmap(&tk, c->k_pages, d->head_dim, page_rows) ||
+      !make_page_tmap(&tv, c->v_pages, d->head_dim, page_rows))
+    return XKV_ERR_CUDA;
+
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  DecodeParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = lse;
+  p.k_pages = static_cast<__nv_bfloat16*>(c->k_pages);
+  p.v_pages = static_cast<__nv_bfloat16*>(c->v_pages);
+  p.block_table = c->block_table;
+  p.seq_lens = c->seq_lens;
+  p.layer_begin = layer_begin;
+  p.n_layers = Lr;
+  p.batch = d->batch;
+  p.n_q_heads = d->n_q_heads;
+  p.n_kv_heads = d->n_kv_heads;
+  p.group = G;
+  p.page_size = c->page_size;
+  p.max_pages_per_seq = c->max_pages_per_seq;
+  p.n_pages = c->n_pages;
+  p.chunk_rows_forced = chunk_rows;
+  p.max_items = (int32_t)L.max_items;
+  const float scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  p.tickets = reinterpret_cast<int32_t*>(ws + L.tickets);
+  p.unit_info = reinterpret_cast<int2*>(ws + L.unit_info);
+  p.items = reinterpret_cast<int4*>(ws + L.items);
+  p.part_o = reinterpret_cast<float*>(ws + L.part_o);
+  p.part_ml = reinterpret_cast<float*>(ws + L.part_ml);
+
+  if (cudaMemsetAsync(ws, 0, L.unit_info, st) != cudaSuccess) return XKV_ERR_CUDA;   // header + tickets
+  const int n_units = Lr * d->batch;
+  if (k_new != nullptr) {
+    const int warps_per_block = 8;
+    decode_append_kernel<<<(n_units + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
+        p, d->head_dim);
+    count_launch();
+    xkv_status s = check_launch();
+    if (s != XKV_OK) return s;
+  }
+  decode_plan_kernel<<<1, 1024, 0, st>>>(p);
+  count_launch();
+  xkv_status s = check_launch();
+  if (s != XKV_OK) return s;
+  if (d->head_dim == 128) return launch_attn<128>(tk, tv, p, st);
+  return launch_attn<64>(tk, tv, p, st);
+}
+
+}  // namespace xkv

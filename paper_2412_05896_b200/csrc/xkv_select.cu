@@ -1,0 +1,251 @@
+// xkv_select_compact: TopK and EvictByIndex of one layer (Alg. 2 steps 5-7).
+//
+//   select_kernel  one CTA per (sequence, KV head).  The k-th largest score is read from the
+//                  descending sort the scoring pass produced; one ordered sweep over the prefix then
+//                  keeps every position above it and the lowest positions equal to it until k are
+//                  kept (ties go to the lower position), which yields the kept positions already in
+//                  ascending order.  The window positions follow.
+//   gather_kernel  16-byte vectorised copy of the kept K and V rows (256-byte rows for d = 128) into
+//                  the layer's cache pages; pure data movement, HBM-bound.
+#include "common.cuh"
+#include "ops.h"
+
+namespace xkv {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelItems = 4;                 // consecutive positions per thread and sweep step
+constexpr int kGatherThreads = 256;
+constexpr int kGatherRows = 64;              // cache rows per gather CTA
+
+struct SelectParams {
+  const float* scores;
+  const float* sorted;
+  const int32_t* cu_seqlens;
+  const int32_t* budget_dev;   // [B] when per-sequence, else null
+  int32_t budget;              // shared budget otherwise
+  int32_t* sel;                // [B][Hkv][sel_stride]
+  int32_t sel_stride;
+  int32_t* seq_lens_layer;     // seq_lens + layer*B
+  const int32_t* block_table_layer;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  __nv_bfloat16* k_pages;
+  __nv_bfloat16* v_pages;
+  int64_t total_tokens, stride_token, stride_head;
+  int32_t batch, n_kv_heads, head_dim, window, page_size, max_pages_per_seq, n_pages;
+  WorkspaceHeader* hdr;
+};
+
+__device__ __forceinline__ void unit_shape(const SelectParams& p, int b, int* cu, int* t, int* P, int* kb) {
+  *cu = p.cu_seqlens[b];
+  *t = p.cu_seqlens[b + 1] - *cu;
+  *P = max(*t - p.window, 0);
+  const int budget = p.budget_dev != nullptr ? p.budget_dev[b] : p.budget;
+  *kb = min(budget, *P);
+}
+
+// Exclusive block scan of one int per thread (kSelThreads threads); returns the exclusive prefix
+// and writes the block total to *total.
+__device__ __forceinline__ int block_scan_excl(int v, int* s_warp, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int u = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += u;
+  }
+  __syncthreads();            // s_warp may still be read from the previous scan
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const int w = s_warp[lane];
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += u;
+    }
+    s_warp[lane] = winc - w;
+    if (lane == 31) s_warp[32] = winc;
+  }
+  __syncthreads();
+  *total = s_warp[32];
+  return s_warp[warp] + incl - v;
+}
+
+__global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
+  __shared__ int s_warp[33];
+  const int b = blockIdx.x / p.n_kv_heads, g = blockIdx.x % p.n_kv_heads;
+  int cu, t, P, kb;
+  unit_shape(p, b, &cu, &t, &P, &kb);
+  const int n_keep = kb + (t - P);
+  const bool fits = n_keep <= p.max_pages_per_seq * p.page_size;
+  if (threadIdx.x == 0 && g == 0) {
+    p.seq_lens_layer[b] = fits ? n_keep : 0;
+    if (!fits) record_status(p.hdr, XKV_ERR_CAPACITY);
+  }
+  if (!fits) return;
+  int32_t* sel = p.sel + ((size_t)b * p.n_kv_heads + g) * p.sel_stride;
+  for (int i = threadIdx.x; i < t - P; i += kSelThreads) sel[kb + i] = P + i;   // window positions
+  if (kb == 0) return;
+  if (kb == P) {
+    for (int i = threadIdx.x; i < P; i += kSelThreads) sel[i] = i;
+    return;
+  }
+  const float* w = p.scores + (size_t)g * p.total_tokens + cu;
+  const float* srt = p.sorted + (size_t)g * p.total_tokens + cu;
+  const float thr = srt[kb - 1];
+  // number of scores strictly above thr = first index of the descending sort holding thr
+  int lo = 0, hi = kb - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (srt[mid] > thr) lo = mid + 1; else hi = mid;
+  }
+  const int eq_needed = kb - lo;
+
+  int carry_eq = 0, carry_sel = 0;
+  for (int base = 0; base < P; base += kSelThreads * kSelItems) {
+    const int c0 = base + threadIdx.x * kSelItems;
+    float x[kSelItems];
+    int n_eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i) {
+      x[i] = (c0 + i < P) ? w[c0 + i] : -1.f;
+      n_eq += (x[i] == thr) ? 1 : 0;
+    }
+    int tot_eq;
+    int eq_before = carry_eq + block_scan_excl(n_eq, s_warp, &tot_eq);
+    bool keep[kSelItems];
+    int n_sel = 0;
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i) {
+      const bool is_eq = x[i] == thr;
+      keep[i] = (c0 + i < P) && (x[i] > thr || (is_eq && eq_before < eq_needed));
+      eq_before += is_eq ? 1 : 0;
+      n_sel += keep[i] ? 1 : 0;
+    }
+    int tot_sel;
+    int dst = carry_sel + block_scan_excl(n_sel, s_warp, &tot_sel);
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i)
+      if (keep[i] && dst < kb) sel[dst++] = c0 + i;
+    carry_eq += tot_eq;
+    carry_sel += tot_sel;
+  }
+}
+
+__global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) {
+  const int unit = blockIdx.x;
+  const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
+  int cu, t, P, kb;
+  unit_shape(p, b, &cu, &t, &P, &kb);
+  const int n_keep = kb + (t - P);
+  if (n_keep > p.max_pages_per_seq * p.page_size) return;
+  const int row0 = blockIdx.y * kGatherRows;
+  if (row0 >= n_keep) return;
+  const int32_t* sel = p.sel + (size_t)unit * p.sel_stride;
+  const int32_t* bt = p.block_table_layer + (size_t)b * p.max_pages_per_seq;
+  const int lanes_per_row = p.head_dim / 8;                   // 16-byte lanes per row
+  const int rows_per_pass = kGatherThreads / lanes_per_row;
+  const int lr = threadIdx.x / lanes_per_row, lc = threadIdx.x % lanes_per_row;
+  for (int r = row0 + lr; r < min(row0 + kGatherRows, n_keep); r += rows_per_pass) {
+    const int pos = sel[r];
+    int page = bt[r / p.page_size];
+    if (page < 0 || page >= p.n_pages) {
+      if (lc == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
+      continue;
+    }
+    const size_t src = (size_t)(cu + pos) * p.stride_token + (size_t)g * p.stride_head + lc * 8;
+    const size_t dst = (((size_t)page * p.n_kv_heads + g) * p.page_size + r % p.page_size) * p.head_dim + lc * 8;
+    const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k + src));
+    const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v + src));
+    *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
+    *reinterpret_cast<uint4*>(p.v_pages + dst) = vv;
+  }
+}
+
+struct SelectLayout {
+  size_t budget, sel, total;
+  int sel_stride;
+};
+
+void select_layout(const xkv_dims* d, int max_seqlen, SelectLayout* L) {
+  size_t off = kHeaderBytes;
+  L->budget = off; off = align_up(off + (size_t)d->batch * 4, 256);
+  L->sel_stride = (max_seqlen + 3) / 4 * 4;
+  L->sel = off;    off = align_up(off + (size_t)d->batch * d->n_kv_heads * L->sel_stride * 4, 256);
+  L->total = off;
+}
+
+}  // namespace
+
+size_t select_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens) {
+  (void)total_tokens;
+  SelectLayout L;
+  select_layout(d, max_seqlen, &L);
+  return L.total;
+}
+
+xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, int per_sequence,
+                          const float* scores, const float* sorted, const void* k, const void* v,
+                          const int32_t* cu_seqlens, int64_t total_tokens, int max_seqlen, const xkv_cache* c,
+                          int32_t* sel, int sel_stride, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  SelectLayout L;
+  select_layout(d, max_seqlen, &L);
+  if (workspace_bytes < L.total) return XKV_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+
+  int max_budget = 0;
+  for (int i = 0; i < (per_sequence ? d->batch : 1); ++i) max_budget = budget[i] > max_budget ? budget[i] : max_budget;
+  const int64_t max_keep64 = (int64_t)max_budget + d->window;
+  const int max_keep = (int)(max_keep64 < max_seqlen ? max_keep64 : max_seqlen);
+  if (sel != nullptr && sel_stride < max_keep) return XKV_ERR_INVALID_ARG;
+
+  SelectParams p;
+  p.scores = scores;
+  p.sorted = sorted;
+  p.cu_seqlens = cu_seqlens;
+  p.budget_dev = nullptr;
+  p.budget = budget[0];
+  p.sel = sel != nullptr ? sel : reinterpret_cast<int32_t*>(ws + L.sel);
+  p.sel_stride = sel != nullptr ? sel_stride : L.sel_stride;
+  p.seq_lens_layer = c->seq_lens + (size_t)layer * d->batch;
+  p.block_table_layer = c->block_table + (size_t)layer * d->batch * c->max_pages_per_seq;
+  p.k = static_cast<const __nv_bfloat16*>(k);
+  p.v = static_cast<const __nv_bfloat16*>(v);
+  p.k_pages = static_cast<__nv_bfloat16*>(c->k_pages);
+  p.v_pages = static_cast<__nv_bfloat16*>(c->v_pages);
+  p.total_tokens = total_tokens;
+  p.stride_token = d->kv_stride_token;
+  p.stride_head = d->kv_stride_head;
+  p.batch = d->batch;
+  p.n_kv_heads = d->n_kv_heads;
+  p.head_dim = d->head_dim;
+  p.window = d->window;
+  p.page_size = c->page_size;
+  p.max_pages_per_seq = c->max_pages_per_seq;
+  p.n_pages = c->n_pages;
+  p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+
+  if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;
+  if (per_sequence) {
+    if (cudaMemcpyAsync(ws + L.budget, budget, (size_t)d->batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return XKV_ERR_CUDA;
+    p.budget_dev = reinterpret_cast<const int32_t*>(ws + L.budget);
+  }
+  const int n_units = d->batch * d->n_kv_heads;
+  select_kernel<<<n_units, kSelThreads, 0, st>>>(p);
+  count_launch();
+  xkv_status s = check_launch();
+  if (s != XKV_OK) return s;
+  if (max_keep > 0) {
+    dim3 grid(n_units, (max_keep + kGatherRows - 1) / kGatherRows);
+    gather_kernel<<<grid, kGatherThreads, 0, st>>>(p);
+    count_launch();
+    s = check_launch();
+  }
+  return s;
+}
+
+}  // namespace xkv

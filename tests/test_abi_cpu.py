@@ -1,0 +1,142 @@
+"""Host-side checks that need no GPU: the library loads, exports every symbol the header declares,
+rejects bad arguments before touching CUDA, and its budget solver (Alg. 1) agrees with the oracle."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import xkv_oracle as O
+from paper_2412_05896_b200 import build, xkv
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "xkv.h")).read()
+    declared = set(re.findall(r"\b(xkv_[a-z_]+)\s*\(", header))
+    assert declared == set(xkv.EXPORTS)
+    lib = ctypes.CDLL(xkv.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert xkv.version() >= 100
+    assert xkv.status_string(xkv.ERR_WORKSPACE) == "workspace too small"
+    assert xkv.launch_count() >= 0
+
+
+def _dims(**kw):
+    base = dict(batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, window=16, pool_kernel=7, pool_mode=0,
+                scale=0.0, kv_stride_token=256, kv_stride_head=128)
+    base.update(kw)
+    return xkv.Dims(**base)
+
+
+def test_workspace_sizes_and_rejections():
+    d = _dims()
+    assert xkv.workspace_bytes(xkv.OP_SCORE, d, max_seqlen=1000, total_tokens=1500) > 0
+    assert xkv.workspace_bytes(xkv.OP_SELECT_COMPACT, d, max_seqlen=1000, total_tokens=1500) > 0
+    auto = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, d, n_layers=4, max_cache_len=4096)
+    forced = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, d, n_layers=4, max_cache_len=4096, chunk_rows=64)
+    assert auto > 0 and forced > 0
+    lib = xkv.lib()
+    for bad in (_dims(head_dim=96), _dims(window=3), _dims(n_kv_heads=3), _dims(pool_kernel=4),
+                _dims(window=128)):
+        assert lib.xkv_workspace_bytes(xkv.OP_SCORE, ctypes.byref(bad), 100, 100, 0, 0, 0) == 0
+    assert lib.xkv_workspace_bytes(99, ctypes.byref(d), 100, 100, 1, 1, 0) == 0
+    assert lib.xkv_workspace_bytes(xkv.OP_DECODE_ATTN, ctypes.byref(d), 0, 0, 4, 100, 32) == 0
+
+
+def test_entry_points_reject_bad_arguments_before_any_cuda_call():
+    lib = xkv.lib()
+    d = _dims()
+    # null pointers
+    assert lib.xkv_score(ctypes.byref(d), None, None, None, 10, 10, None, None, None, None, 1, None, 0,
+                         None) == xkv.ERR_INVALID_ARG
+    # unsupported head_dim
+    bad = _dims(head_dim=96)
+    assert lib.xkv_score(ctypes.byref(bad), 16, 16, 16, 10, 10, 16, None, None, None, 1, 256, 0,
+                         None) == xkv.ERR_UNSUPPORTED
+    # misaligned pointer
+    assert lib.xkv_score(ctypes.byref(d), 24, 16, 16, 10, 10, 16, None, None, None, 1, 256, 1 << 30,
+                         None) == xkv.ERR_INVALID_ARG
+    # workspace too small
+    assert lib.xkv_score(ctypes.byref(d), 16, 16, 16, 1500, 1000, 16, None, None, None, 1, 256, 64,
+                         None) == xkv.ERR_WORKSPACE
+    cache = xkv.Cache(256, 512, 768, 1024, 4, 16, 8, 100)
+    assert lib.xkv_decode_attn(ctypes.byref(d), ctypes.byref(cache), 0, 5, 16, None, None, 16, None, 0, 256,
+                               1 << 30, None) == xkv.ERR_INVALID_ARG          # layer range
+    assert lib.xkv_decode_attn(ctypes.byref(d), ctypes.byref(cache), 0, 4, 16, 16, None, 16, None, 0, 256,
+                               1 << 30, None) == xkv.ERR_INVALID_ARG          # k_new without v_new
+    assert lib.xkv_decode_attn(ctypes.byref(d), ctypes.byref(cache), 0, 4, 16, None, None, 16, None, 0, 256,
+                               64, None) == xkv.ERR_WORKSPACE
+    bad_cache = xkv.Cache(256, 512, 768, 1024, 4, 24, 8, 100)                 # page size not a multiple of 16
+    assert lib.xkv_decode_attn(ctypes.byref(d), ctypes.byref(bad_cache), 0, 4, 16, None, None, 16, None, 0,
+                               256, 1 << 30, None) == xkv.ERR_INVALID_ARG
+    budget = np.array([-1], dtype=np.int32)
+    assert lib.xkv_select_compact(ctypes.byref(d), 0, budget.ctypes.data, 0, 16, 16, 16, 16, 16, 1500, 1000,
+                                  ctypes.byref(cache), None, 0, 256, 1 << 30, None) == xkv.ERR_BUDGET
+
+
+def _curves(rng, L, B, n, power=3.0):
+    g = np.zeros((L, B, n), dtype=np.float32)
+    for l in range(L):
+        for b in range(B):
+            g[l, b] = O.head_gains(rng.random(n) ** (power + l))
+    return g
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_alloc_budgets_matches_oracle_and_bruteforce(seed):
+    rng = np.random.default_rng(seed)
+    L, B, n = 3, 2, 6
+    g = _curves(rng, L, B, n)
+    mean = [c for c in O.batch_mean_gains(g.astype(np.float64))]
+    for N in range(0, L * n + 1):
+        budgets, r = xkv.alloc_budgets(g, [n] * B, total=N)
+        assert budgets.sum() == N
+        A, r_o = O.adaptive_allocation(mean, N=N)
+        assert abs(r - r_o) < 1e-12 and budgets.tolist() == A
+        if N <= 12:
+            _, best = O.bruteforce_allocation(mean, N)
+            assert abs(r - best) < 1e-12
+
+
+def test_alloc_budgets_modes():
+    rng = np.random.default_rng(7)
+    L, B, n = 8, 3, 200
+    g = _curves(rng, L, B, n, power=1.5)
+    mean = [c for c in O.batch_mean_gains(g.astype(np.float64))]
+    # box constraints
+    budgets, r = xkv.alloc_budgets(g, [n] * B, total=400, n_min=10, n_max=120)
+    A, r_o = O.adaptive_allocation(mean, N=400, n_min=10, n_max=120)
+    assert budgets.tolist() == A and abs(r - r_o) < 1e-12 and budgets.min() >= 10 and budgets.max() <= 120
+    # R target mode (Eq. 18)
+    budgets, r = xkv.alloc_budgets(g, [n] * B, r_target=0.8)
+    A, r_o = O.adaptive_allocation(mean, R_avg=0.8)
+    assert budgets.tolist() == A and r >= 0.8 and abs(r - r_o) < 1e-12
+    # per-sequence lists, ragged capacities
+    prefix = [200, 150, 90]
+    g2 = g.copy()
+    for b, P in enumerate(prefix):
+        g2[:, b, P:] = 0
+    budgets, r = xkv.alloc_budgets(g2, prefix, per_sequence=True, total=300)
+    assert budgets.shape == (B, L)
+    for b, P in enumerate(prefix):
+        A, r_o = O.adaptive_allocation([g2[l, b].astype(np.float64) for l in range(L)], N=300,
+                                       capacity=[P] * L)
+        assert budgets[b].tolist() == A and abs(r[b] - r_o) < 1e-12 and budgets[b].max() <= P
+    # errors
+    for kw in (dict(total=L * n + 1), dict(total=5, n_min=10), dict(r_target=1.5)):
+        with pytest.raises(xkv.XkvError) as e:
+            xkv.alloc_budgets(g, [n] * B, **kw)
+        assert e.value.status == xkv.ERR_BUDGET
+    # identical layers: ties go to the lowest layer index
+    same = np.tile(O.head_gains(np.array([5.0, 4, 3, 2, 1])).astype(np.float32), (3, 1, 1))
+    budgets, _ = xkv.alloc_budgets(same, [5], total=7)
+    assert budgets.tolist() == [3, 2, 2]
