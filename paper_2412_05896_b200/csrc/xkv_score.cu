@@ -24,6 +24,10 @@
 namespace xkv {
 namespace {
 
+#ifndef XKV_SPLIT_ACC
+#define XKV_SPLIT_ACC 1
+#endif
+
 constexpr int kPassThreads = 128;     // 4 warps
 constexpr int kKeyTile = 128;         // keys per tile, 32 per warp
 constexpr int kSortChunk = 4096;      // scores sorted per CTA
@@ -162,10 +166,27 @@ __global__ void __launch_bounds__(kPassThreads) score_pass_kernel(const ScorePar
         const int row = 16 * mt + (mat & 1) * 8 + mrow_l;
         const int col = 16 * ks + (mat >> 1) * 8;
         ldmatrix_x4(a, q_base + row * C::kRowBytes + col * 2);
+#if XKV_SPLIT_ACC
+        // The tensor core adds into its fp32 accumulator with truncation; summing the per-k-step
+        // partial products with ordinary round-to-nearest adds keeps the logits accurate enough for
+        // the top-k decision.
+        float part[4][4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) part[nt][0] = part[nt][1] = part[nt][2] = part[nt][3] = 0.f;
+        mma_bf16_16816(part[0], a, bf[0][ks][0], bf[0][ks][1]);
+        mma_bf16_16816(part[1], a, bf[0][ks][2], bf[0][ks][3]);
+        mma_bf16_16816(part[2], a, bf[1][ks][0], bf[1][ks][1]);
+        mma_bf16_16816(part[3], a, bf[1][ks][2], bf[1][ks][3]);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[nt][j] += part[nt][j];
+#else
         mma_bf16_16816(acc[0], a, bf[0][ks][0], bf[0][ks][1]);
         mma_bf16_16816(acc[1], a, bf[0][ks][2], bf[0][ks][3]);
         mma_bf16_16816(acc[2], a, bf[1][ks][0], bf[1][ks][1]);
         mma_bf16_16816(acc[3], a, bf[1][ks][2], bf[1][ks][3]);
+#endif
       }
 #pragma unroll
       for (int half = 0; half < 2; ++half) {

@@ -1,0 +1,97 @@
+"""GPU parity of xkv_decode_attn (Eq. 1, generation phase) against the fp64 oracle, on ragged caches
+built directly with torch so that this step is tested alone."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import xkv_oracle as O
+from paper_2412_05896_b200 import xkv
+
+from gpu_util import DirectCache, check_attention, f64, require_lib
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _run_case(L, B, Hq, Hkv, d, lens, page_size, chunk_rows, append, seed, stress=False, steps=1):
+    require_lib()
+    G = Hq // Hkv
+    cache = DirectCache(L, B, Hkv, d, lens, page_size, extra_rows=steps + 1, device=DEV, seed=seed,
+                        v_shift=1.0 if stress else 0.0)
+    dims = xkv.Dims(B, Hq, Hkv, d, 16, 1, 0, 0.0, Hkv * d, d)
+    handle = cache.handle()
+    ws_bytes = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L,
+                                   max_cache_len=cache.max_pages * page_size, chunk_rows=chunk_rows)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    out = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
+    lse = torch.empty(L, B, Hq, dtype=torch.float32, device=DEV)
+    g = torch.Generator(device="cpu").manual_seed(seed + 1000)
+    for step in range(steps):
+        q = (torch.randn(L, B, Hq, d, generator=g) * (4.0 if stress else 1.0)).to(torch.bfloat16)
+        k_new = torch.randn(L, B, Hkv, d, generator=g).to(torch.bfloat16)
+        v_new = (torch.randn(L, B, Hkv, d, generator=g) + (1.0 if stress else 0.0)).to(torch.bfloat16)
+        qd = q.to(DEV)
+        if append:
+            xkv.decode_attn(dims, handle, 0, L, qd, k_new.to(DEV), v_new.to(DEV), out, lse, chunk_rows, ws)
+            cache.append_host(k_new, v_new)
+        else:
+            xkv.decode_attn(dims, handle, 0, L, qd, None, None, out, lse, chunk_rows, ws)
+        torch.cuda.synchronize()
+        assert xkv.read_device_status(ws) == xkv.OK
+        ref = np.zeros((L, B, Hq, d))
+        ref_lse = np.zeros((L, B, Hq))
+        for l in range(L):
+            for b in range(B):
+                K, V = f64(cache.K[(l, b)]), f64(cache.V[(l, b)])
+                for h in range(Hq):
+                    ref[l, b, h], ref_lse[l, b, h] = O.decode_attention(f64(q[l, b, h]), K[:, h // G], V[:, h // G])
+        check_attention(out, ref, f"step {step}", rel_l2=stress)
+        got_lse = lse.cpu().numpy().astype(np.float64)
+        finite = np.isfinite(ref_lse)
+        assert np.array_equal(np.isfinite(got_lse), finite)
+        assert np.allclose(got_lse[finite], ref_lse[finite], atol=2e-3, rtol=1e-4)
+        if append:
+            expect = np.array([[cache.K[(l, b)].shape[0] for b in range(B)] for l in range(L)])
+            assert np.array_equal(cache.seq_lens.cpu().numpy(), expect)
+
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 4, 4), (128, 4, 4), (128, 8, 2), (128, 8, 1), (64, 4, 2)])
+def test_decode_ragged_lengths_with_append(d, Hq, Hkv):
+    lens = [[0, 1, 15], [16, 17, 63], [64, 65, 300], [1000, 129, 33]]
+    _run_case(4, 3, Hq, Hkv, d, lens, 16, 0, True, seed=d + Hq, steps=2)
+
+
+@pytest.mark.parametrize("chunk_rows", [64, 128, 0])
+@pytest.mark.parametrize("page_size", [16, 64])
+def test_decode_split_invariance_and_page_sizes(chunk_rows, page_size):
+    lens = [[700, 64, 1, 0], [2050, 129, 640, 63]]
+    _run_case(2, 4, 8, 2, 128, lens, page_size, chunk_rows, False, seed=chunk_rows + page_size)
+
+
+def test_decode_peaked_attention_and_shifted_values():
+    lens = [[2000, 513], [777, 4096]]
+    _run_case(2, 2, 8, 2, 128, lens, 16, 0, True, seed=5, stress=True, steps=2)
+    _run_case(2, 2, 4, 4, 64, lens, 32, 256, True, seed=6, stress=True)
+
+
+def test_decode_many_units_long_chunks():
+    rng = np.random.default_rng(3)
+    lens = rng.integers(1, 900, size=(6, 16)).tolist()
+    _run_case(6, 16, 8, 8, 128, lens, 16, 0, True, seed=9)
+
+
+def test_decode_capacity_overflow_is_reported_not_faulted():
+    require_lib()
+    L, B, Hq, Hkv, d, ps = 1, 2, 4, 4, 64, 16
+    cache = DirectCache(L, B, Hkv, d, [[16, 5]], ps, extra_rows=0, device=DEV, seed=1)
+    assert cache.max_pages == 1                      # sequence 0 is exactly full
+    dims = xkv.Dims(B, Hq, Hkv, d, 16, 1, 0, 0.0, Hkv * d, d)
+    ws = torch.empty(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=ps),
+                     dtype=torch.uint8, device=DEV)
+    q = torch.randn(L, B, Hq, d, device=DEV).to(torch.bfloat16)
+    kn = torch.randn(L, B, Hkv, d, device=DEV).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    xkv.decode_attn(dims, cache.handle(), 0, L, q, kn, kn, out, None, 0, ws)
+    torch.cuda.synchronize()
+    assert xkv.read_device_status(ws) == xkv.ERR_CAPACITY
+    assert cache.seq_lens.cpu().tolist() == [[16, 6]]

@@ -1,0 +1,188 @@
+"""GPU parity of xkv_score and xkv_select_compact (Eq. 2-4; Alg. 2) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import xkv_oracle as O
+from paper_2412_05896_b200 import xkv
+from paper_2412_05896_b200.pipeline import XkvSession
+
+from gpu_util import bits, f64, require_lib
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+MODE = {0: "max", 1: "avg"}
+
+
+def _inputs(seed, lengths, Hq, Hkv, d, W, peaked=True):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    T = sum(lengths)
+    k = torch.randn(T, Hkv, d, generator=g)
+    u = torch.randn(Hkv, d, generator=g)
+    u = u / u.norm(dim=-1, keepdim=True)
+    heavy = (torch.rand(T, Hkv, generator=g) < 0.03).float()
+    k = k + 3.0 * heavy[..., None] * u[None]
+    q = torch.randn(len(lengths), Hq, W, d, generator=g)
+    if peaked:
+        q = (q + d ** 0.5 * u.repeat_interleave(Hq // Hkv, 0)[None, :, None, :]) / 0.7
+    v = torch.randn(T, Hkv, d, generator=g)
+    return q.to(torch.bfloat16), k.to(torch.bfloat16), v.to(torch.bfloat16)
+
+
+def _oracle_scores(q, k, cu, W, ps, mode):
+    return O.score_layer(f64(q), f64(k), cu, W, ps, MODE[mode])
+
+
+def _check_scores(sess, layer, w_ref, lengths, Hkv, W):
+    got = sess.scores[layer].cpu().numpy().astype(np.float64)
+    srt = sess.sorted[layer].cpu().numpy()
+    cu = sess.cu_host
+    worst = 0.0
+    for b, t in enumerate(lengths):
+        P = max(t - W, 0)
+        for g in range(Hkv):
+            seg = got[g, cu[b]: cu[b] + t]
+            ref = w_ref[(b, g)]
+            assert np.all(seg[P:] == 0.0) and np.all(srt[g, cu[b] + P: cu[b] + t] == 0.0)
+            if P == 0:
+                continue
+            err = np.abs(seg[:P] - ref)
+            tol = 3e-5 * ref + 1e-7 * ref.max()
+            worst = max(worst, float((err / np.maximum(ref, 1e-300))[ref > 1e-4 * ref.max()].max()))
+            assert np.all(err <= tol), f"unit {(b, g)}: score error {float((err - tol).max()):.3e} over tolerance"
+            # the sort is exact: same multiset, descending
+            s = srt[g, cu[b]: cu[b] + P]
+            assert np.array_equal(s, np.sort(sess.scores[layer][g, cu[b]: cu[b] + P].cpu().numpy())[::-1])
+    return worst
+
+
+CASES = [
+    # lengths, Hq, Hkv, d, W, ps, mode
+    ([300, 1000, 9], 4, 4, 64, 16, 5, 0),
+    ([513, 128], 8, 2, 128, 32, 7, 0),
+    ([700], 8, 2, 128, 8, 7, 1),
+    ([2500, 1200], 8, 2, 128, 32, 7, 0),         # G*W = 128 query rows
+    ([1500], 16, 4, 128, 64, 3, 0),              # G*W = 256 query rows
+    ([9000, 4097], 2, 2, 128, 16, 7, 0),         # several sort chunks and merge passes
+    ([33, 17, 16, 1], 2, 1, 64, 16, 1, 0),       # at and below the window length
+]
+
+
+@pytest.mark.parametrize("lengths,Hq,Hkv,d,W,ps,mode", CASES)
+def test_score_sort_and_curves(lengths, Hq, Hkv, d, W, ps, mode):
+    require_lib()
+    q, k, v = _inputs(len(lengths) * 7 + W, lengths, Hq, Hkv, d, W)
+    sess = XkvSession(1, Hq, Hkv, d, W, ps, lengths, pool_mode=mode, device=DEV)
+    mass = torch.empty(len(lengths), sess.curve_len, dtype=torch.float32, device=DEV)
+    sess.score_layer(0, q.to(DEV), k.to(DEV), mass=mass)
+    torch.cuda.synchronize()
+    assert sess.device_status("score") == xkv.OK
+    w_ref = _oracle_scores(q, k, sess.cu_host, W, ps, mode)
+    _check_scores(sess, 0, w_ref, lengths, Hkv, W)
+    curves = O.layer_curves(w_ref, len(lengths), Hkv, sess.curve_len)
+    got = sess.gains[0].cpu().numpy().astype(np.float64)
+    assert np.allclose(got, curves, rtol=1e-4, atol=1e-7)
+    got_mass = mass.cpu().numpy().astype(np.float64)
+    assert np.allclose(got_mass, np.cumsum(curves, axis=1), rtol=0, atol=2e-5)
+    for b, t in enumerate(lengths):
+        if t > W:
+            assert abs(got_mass[b, min(t - W, sess.curve_len) - 1] - 1.0) < 2e-5 or t - W > sess.curve_len
+
+
+def _cache_rows(sess, layer, b, g, n):
+    bt = sess.block_table[layer, b].cpu().numpy()
+    slots = np.arange(n)
+    pages = torch.from_numpy(bt[slots // sess.page_size].astype(np.int64)).to(sess.device)
+    off = torch.from_numpy(slots % sess.page_size).to(sess.device)
+    return bits(sess.k_pages[pages, g, off]), bits(sess.v_pages[pages, g, off])
+
+
+@pytest.mark.parametrize("quantised", [True, False])
+@pytest.mark.parametrize("d,page_size", [(128, 16), (64, 64)])
+def test_select_compact_is_bit_exact_on_given_scores(quantised, d, page_size):
+    """Selection and compaction alone: scores are inputs, so the kept sets must equal the oracle's
+    exactly (ties to the lower position) and the cache must hold the oracle's rows bit for bit."""
+    require_lib()
+    lengths, Hkv, W = [1000, 5000, 40, 12, 4200], 2, 16
+    B, T = len(lengths), sum(lengths)
+    g = torch.Generator(device="cpu").manual_seed(11 + d)
+    scores = torch.rand(Hkv, T, generator=g) ** 4
+    if quantised:
+        scores = torch.round(scores * 12) / 12          # many exact ties, including at the threshold
+    sess = XkvSession(1, Hkv, Hkv, d, W, 1, lengths, page_size=page_size, device=DEV)
+    cu = sess.cu_host
+    srt = torch.zeros_like(scores)
+    for b, t in enumerate(lengths):
+        P = max(t - W, 0)
+        scores[:, cu[b] + P: cu[b] + t] = 0
+        srt[:, cu[b]: cu[b] + P] = torch.sort(scores[:, cu[b]: cu[b] + P], dim=1, descending=True).values
+    k = torch.randn(T, Hkv, d, generator=g).to(torch.bfloat16)
+    v = torch.randn(T, Hkv, d, generator=g).to(torch.bfloat16)
+    sess.scores[0].copy_(scores)
+    sess.sorted[0].copy_(srt)
+    for budget in (0, 1, 7, 300, 984, 985, 4999, 10 ** 6):
+        sess.assign_pages([budget])
+        sess.k_pages.fill_(float("nan"))
+        sel = torch.full((B, Hkv, sess.max_seqlen), -1, dtype=torch.int32, device=DEV)
+        sess.select_layer(0, budget, k.to(DEV), v.to(DEV), sel=sel)
+        torch.cuda.synchronize()
+        assert sess.device_status("select") == xkv.OK
+        lens = sess.seq_lens[0].cpu().numpy()
+        for b, t in enumerate(lengths):
+            P = max(t - W, 0)
+            for h in range(Hkv):
+                keep = O.kept_positions(scores[h, cu[b]: cu[b] + P].double().numpy(), budget, t, W)
+                assert lens[b] == len(keep)
+                assert np.array_equal(sel[b, h, : len(keep)].cpu().numpy(), keep), (budget, b, h)
+                kb, vb = _cache_rows(sess, 0, b, h, len(keep))
+                assert np.array_equal(kb, O.evict_by_index(bits(k[cu[b]: cu[b] + t, h]), keep))
+                assert np.array_equal(vb, O.evict_by_index(bits(v[cu[b]: cu[b] + t, h]), keep))
+
+
+def test_select_per_sequence_budgets_and_capacity_status():
+    require_lib()
+    lengths, Hkv, W, d = [600, 900], 2, 16, 64
+    q, k, v = _inputs(3, lengths, Hkv, Hkv, d, W)
+    sess = XkvSession(1, Hkv, Hkv, d, W, 5, lengths, device=DEV, max_budget=200)
+    sess.score_layer(0, q.to(DEV), k.to(DEV))
+    budgets = np.array([[50], [120]], dtype=np.int32)
+    sess.assign_pages(budgets)
+    sess.select_layer(0, budgets[:, 0], k.to(DEV), v.to(DEV), per_sequence=True)
+    torch.cuda.synchronize()
+    assert sess.seq_lens[0].cpu().tolist() == [50 + W, 120 + W]
+    # a budget beyond the page table is reported through the status word, nothing is written
+    sess.select_layer(0, 800, k.to(DEV), v.to(DEV))
+    torch.cuda.synchronize()
+    assert sess.device_status("select") == xkv.ERR_CAPACITY
+    assert sess.seq_lens[0].cpu().tolist() == [0, 0]
+
+
+@pytest.mark.parametrize("lengths,Hq,Hkv,d,W,ps,mode", CASES[:5])
+def test_selection_from_gpu_scores_matches_oracle_outside_near_ties(lengths, Hq, Hkv, d, W, ps, mode):
+    """End to end through scoring: kept sets equal the oracle's wherever no other score lies within
+    1e-5 (relative) of the k-th largest; inside that band only the band itself may differ."""
+    require_lib()
+    q, k, v = _inputs(5 + W, lengths, Hq, Hkv, d, W)
+    sess = XkvSession(1, Hq, Hkv, d, W, ps, lengths, pool_mode=mode, device=DEV)
+    sess.score_layer(0, q.to(DEV), k.to(DEV))
+    w_ref = _oracle_scores(q, k, sess.cu_host, W, ps, mode)
+    near, total = 0, 0
+    for budget in (16, 100, 257):
+        sess.assign_pages([budget])
+        sel = torch.full((len(lengths), Hkv, sess.max_seqlen), -1, dtype=torch.int32, device=DEV)
+        sess.select_layer(0, budget, k.to(DEV), v.to(DEV), sel=sel)
+        torch.cuda.synchronize()
+        for b, t in enumerate(lengths):
+            for g in range(Hkv):
+                w = w_ref[(b, g)]
+                keep = O.kept_positions(w, budget, t, W)
+                got = sel[b, g, : len(keep)].cpu().numpy()
+                total += 1
+                if O.near_tie(w, budget):
+                    near += 1
+                    thr = O.sort_descending(w)[min(budget, len(w)) - 1]
+                    diff = np.setxor1d(got, keep)
+                    assert np.all(np.abs(w[diff] - thr) <= 1e-5 * thr)
+                else:
+                    assert np.array_equal(got, keep), (budget, b, g)
+    print(f"near-tie heads: {near} of {total}")
