@@ -1,0 +1,444 @@
+#!/usr/bin/env python
+"""Benchmark of the XKV hot path on B200.
+
+One "step" is one pass of the whole path over one batch of the seeded synthetic workload: score
+every layer, split the global budget across layers on the host, evict/compact every layer into the
+ragged paged cache, then run the workload's decode steps (append + attention over all layers).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl xkv|reference]
+
+Prints one JSON line.  `value` is the decode-attention throughput over the retained cache
+(bytes of retained K and V read per decode step / decode time), device-resident inputs;
+`e2e` is the same with host inputs and outputs; `roofline` is the attention kernel alone against
+the measured HBM bandwidth; `cpu_baseline` is the fp64 oracle timed on the host cores.
+With N > 1 (launched by torch.distributed.run) every rank runs its own batch: no data-path
+collective, weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+DEFAULT_WORKLOAD = "llama2_7b_mha"
+METRIC = "ragged-KV decode-attn GB/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_attn_kernel launch, from the ncu capture
+# summarised under profiles/ (None while no capture matches the current kernel).
+NCU_TRAFFIC = None
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# Oracle leg (CPU baseline and --impl reference)
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(w, tensors_cpu, lengths, budget: int, seconds: float, decode_steps: int):
+    """Runs the oracle, as it stands, on (layer 0, sequence 0, every KV head): scoring, top-k,
+    compaction, then decode steps; repeats decode passes until `seconds` have elapsed.
+
+    Returns (decode bytes of retained K/V read, decode seconds, prefill seconds, cpu seconds / wall).
+    """
+    import numpy as np
+    from oracle import xkv_oracle as O
+    from paper_2412_05896_b200 import workloads as WL
+
+    def f64(t):
+        return t.float().numpy().astype(np.float64)
+
+    q_win, k, v = tensors_cpu
+    t0 = lengths[0]
+    qf, kf, vf = f64(q_win[0:1]), f64(k[:t0]), f64(v[:t0])
+    cu = np.array([0, t0])
+    wall0, cpu0 = time.perf_counter(), time.process_time()
+    t_pre = time.perf_counter()
+    w_units = O.score_layer(qf, kf, cu, w.window, w.pool_kernel, "max" if w.pool_mode == 0 else "avg")
+    caches = {}
+    for g in range(w.n_kv_heads):
+        keep = O.kept_positions(w_units[(0, g)], budget, t0, w.window)
+        caches[g] = (O.evict_by_index(kf[:, g], keep), O.evict_by_index(vf[:, g], keep))
+    prefill_s = time.perf_counter() - t_pre
+    G, d = w.group, w.head_dim
+    bytes_read, dec_s, step = 0, 0.0, 0
+    deadline = time.perf_counter() + seconds
+    while True:
+        q, kn, vn = WL.decode_tensors(w, step % decode_steps, "cpu", layers=1)
+        qd, knd, vnd = f64(q[0, 0]), f64(kn[0, 0]), f64(vn[0, 0])
+        t1 = time.perf_counter()
+        for g in range(w.n_kv_heads):
+            Kc = np.concatenate([caches[g][0], knd[g][None]], 0)
+            Vc = np.concatenate([caches[g][1], vnd[g][None]], 0)
+            caches[g] = (Kc, Vc)
+            for h in range(g * G, (g + 1) * G):
+                O.decode_attention(qd[h], Kc, Vc)
+            bytes_read += Kc.shape[0] * 2 * d * 2          # the bf16 bytes this KV head's step stands for
+        dec_s += time.perf_counter() - t1
+        step += 1
+        if time.perf_counter() > deadline and step >= 4:
+            break
+    wall, cpu = time.perf_counter() - wall0, time.process_time() - cpu0
+    return bytes_read, dec_s, prefill_s, max(1, round(cpu / max(wall, 1e-9))), step
+
+
+def run_reference(args):
+    """--impl reference: the oracle timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2412_05896_b200 import workloads as WL
+    w = WL.CONFIGS[args.workload]
+    lengths = WL.prompt_lengths(w)
+    one_seq = replace(w, batch=1, prompt=lengths[0])
+    tensors = WL.layer_tensors(one_seq, 0, "cpu", [lengths[0]])
+    budget = w.avg_budget if w.budgets is None else w.budgets[0]
+    per_step_s = max(2.0, min(20.0, 60.0 / max(args.steps + args.warmup, 1)))
+    vals, cores, samples = [], 1, 0
+    t_all = time.perf_counter()
+    for i in range(args.warmup + args.steps):
+        b, s, pre, cores, n = oracle_sample(w, tensors, [lengths[0]], budget, per_step_s, w.decode_steps)
+        if i >= args.warmup:
+            vals.append((b, s))
+            samples = n
+    total_b = sum(b for b, _ in vals)
+    total_s = sum(s for _, s in vals)
+    value = total_b / total_s / 1e9
+    sample = (f"layer 0, sequence 0, all {w.n_kv_heads} KV heads: oracle scoring + top-k + compaction, then "
+              f"{samples} decode steps per bench step (~{per_step_s:.0f} s)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * (time.perf_counter() - t_all) / max(args.steps + args.warmup, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# The CUDA path
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="xkv", choices=["xkv", "reference"])
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_05896_b200 import build as _build
+    from paper_2412_05896_b200 import workloads as WL
+    from paper_2412_05896_b200 import xkv
+    from paper_2412_05896_b200.pipeline import XkvSession
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the XKV path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    xkv.lib()
+
+    w0 = WL.CONFIGS[args.workload]
+    if args.decode_steps:
+        w0 = replace(w0, decode_steps=args.decode_steps)
+    w = replace(w0, seed=w0.seed + 7919 * rank)          # every rank draws its own batch
+    L, B, Hkv, d, W = w.n_layers, w.batch, w.n_kv_heads, w.head_dim, w.window
+    lengths = WL.prompt_lengths(w)
+    n_dec = w.decode_steps
+    tens = [WL.layer_tensors(w, l, dev, lengths) for l in range(L)]
+    q_win = [t[0] for t in tens]
+    k = [t[1] for t in tens]
+    v = [t[2] for t in tens]
+    dec = [WL.decode_tensors(w, s, dev) for s in range(n_dec)]
+    N_total = None if w.budgets is not None else L * w.avg_budget
+    sess = XkvSession(L, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
+                      max_new_tokens=n_dec, max_budget=w.n_max or None, total_budget=N_total,
+                      curve_len=w.n_max or None, device=dev)
+    prefix = sess.prefix
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    k_start = [ev() for _ in range(n_dec)]
+    k_stop = [ev() for _ in range(n_dec)]
+    for e in k_start + k_stop:
+        e.record()
+
+    def decode_bytes(budgets) -> list[int]:
+        """Retained K and V bytes one decode step reads, per decode step (the cache grows by one row)."""
+        base = sum(min(int(budgets[l]), P) + min(W, t) for l in range(L) for P, t in zip(prefix, lengths))
+        return [(base + (s + 1) * L * B) * Hkv * 2 * d * 2 for s in range(n_dec)]
+
+    def prefill_bytes(budgets) -> int:
+        """Algorithmic bytes of score + select + compact: K once, score out, kept rows in and out."""
+        tot = 0
+        for l in range(L):
+            for P, t in zip(prefix, lengths):
+                kept = min(int(budgets[l]), P) + min(W, t)
+                tot += Hkv * (t * (2 * d + 8) + kept * (8 * d + 4))
+        return tot
+
+    def step(host=None, kernel_events=False):
+        """One pass of the whole path.  host: dict of pinned host buffers for the end-to-end leg."""
+        e = [ev() for _ in range(5)]
+        e[0].record()
+        if host is not None:
+            for l in range(L):
+                q_win[l].copy_(host["q_win"][l], non_blocking=True)
+                k[l].copy_(host["k"][l], non_blocking=True)
+                v[l].copy_(host["v"][l], non_blocking=True)
+        for l in range(L):
+            sess.score_layer(l, q_win[l], k[l])
+        e[1].record()
+        if w.budgets is not None:
+            budgets = np.asarray(w.budgets, dtype=np.int32)
+        else:
+            budgets, _ = sess.solve_budgets(total=N_total, n_min=w.n_min, n_max=w.n_max)
+        sess.assign_pages(budgets)
+        e[2].record()
+        for l in range(L):
+            sess.select_layer(l, int(budgets[l]), k[l], v[l])
+        e[3].record()
+        for s in range(n_dec):
+            q, kn, vn = dec[s]
+            if host is not None:
+                q.copy_(host["dec"][s][0], non_blocking=True)
+                kn.copy_(host["dec"][s][1], non_blocking=True)
+                vn.copy_(host["dec"][s][2], non_blocking=True)
+            if kernel_events:
+                xkv.profile_events(k_start[s], k_stop[s])
+            sess.decode(q, kn, vn)
+            if host is not None:
+                host["out"].copy_(sess.out, non_blocking=True)
+        e[4].record()
+        xkv.profile_events(None, None)
+        return e, budgets
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    sync_all()
+    for which in ("score", "select", "decode"):
+        st = sess.device_status(which)
+        if st != xkv.OK:
+            raise SystemExit(f"device status of {which}: {xkv.status_string(st)}")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = xkv.launch_count()
+    first, last = ev(), ev()
+    sync_all()
+    first.record()
+    recs = []
+    for _ in range(args.steps):
+        recs.append(step(kernel_events=True))
+        torch.cuda.current_stream().synchronize()    # kernel events of this step are read below
+        recs[-1] = recs[-1] + ([a.elapsed_time(b) for a, b in zip(k_start, k_stop)],)
+    last.record()
+    sync_all()
+    launches = xkv.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+
+    budgets = recs[-1][1]
+    dbytes = decode_bytes(budgets)
+    phase = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e, _, _ in recs])   # ms
+    step_ms = np.array([e[0].elapsed_time(e[4]) for e, _, _ in recs])
+    dec_ms_total = float(phase[:, 3].sum())
+    region_ms = first.elapsed_time(last)
+    kern_ms = np.array([r[2] for r in recs])                       # [steps, n_dec]
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    dec_ms_max = max_over_ranks(dec_ms_total)
+    region_ms_max = max_over_ranks(region_ms)
+    all_bytes = sum_over_ranks(float(sum(dbytes)) * args.steps)
+    value = all_bytes / (dec_ms_max * 1e-3) / 1e9
+    tokens_per_s = world * B * n_dec * args.steps / (dec_ms_max * 1e-3)
+
+    # ---------------------------------------------------------------- end-to-end leg (host buffers)
+    e2e = None
+    if not args.no_e2e:
+        try:
+            host = {"q_win": [t.cpu().pin_memory() for t in q_win], "k": [t.cpu().pin_memory() for t in k],
+                    "v": [t.cpu().pin_memory() for t in v],
+                    "dec": [tuple(x.cpu().pin_memory() for x in dec[s]) for s in range(n_dec)],
+                    "out": torch.empty(sess.out.shape, dtype=sess.out.dtype, pin_memory=True)}
+            h2d = sum(t.numel() * 2 for t in q_win + k + v) + sum(x.numel() * 2 for s in range(n_dec) for x in dec[s])
+            d2h = sess.out.numel() * 2 * n_dec + sess.gains.numel() * 4
+            step(host=host)
+            sync_all()
+            e_recs = [step(host=host) for _ in range(2)]
+            sync_all()
+            e_dec_ms = max_over_ranks(sum(e[3].elapsed_time(e[4]) for e, _ in e_recs))
+            e_step_ms = max_over_ranks(sum(e[0].elapsed_time(e[4]) for e, _ in e_recs) / len(e_recs))
+            e_bytes = sum_over_ranks(float(sum(decode_bytes(e_recs[-1][1]))) * len(e_recs))
+            e2e = {"value": e_bytes / (e_dec_ms * 1e-3) / 1e9, "unit": "GB/s",
+                   "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                   "ms_per_step": e_step_ms,
+                   "note": "value: decode phase with q/k_new/v_new copied from pinned host memory and the output "
+                           "copied back every decode step; ms_per_step: the whole pass including the host-to-device "
+                           "copy of every layer's Q_win, K and V"}
+            del host
+        except RuntimeError as err:                                  # e.g. pinned allocation refused
+            e2e = {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                   "note": f"host leg failed: {str(err)[:120]}"}
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    kern_avg_ms = float(kern_ms.mean())
+    launch_bytes = float(np.mean(dbytes))
+    achieved = launch_bytes / (kern_avg_ms * 1e-3) / 1e9
+    roofline = {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0, "peak_source": peak_src,
+                "bytes_per_launch": launch_bytes, "avg_launch_ms": kern_avg_ms, "traffic": NCU_TRAFFIC}
+
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        one_seq = replace(w, batch=1, prompt=lengths[0])
+        cpu_t = tuple(x[: (lengths[0] if i else 1)].cpu() for i, x in enumerate(tens[0]))
+        b0 = int(budgets[0])
+        nbytes, dec_s, pre_s, cores, n = oracle_sample(one_seq, cpu_t, [lengths[0]], b0, 12.0, n_dec)
+        cpu_baseline = {"value": nbytes / dec_s / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                        "sample": f"layer 0, sequence 0, all {Hkv} KV heads: {n} decode steps of fp64 numpy "
+                                  f"attention over the oracle's own compacted cache ({dec_s:.1f} s); its scoring + "
+                                  f"top-k + compaction of that layer-sequence took {pre_s:.2f} s",
+                        "prefill_seconds_layer0_seq0": pre_s}
+
+    pre_bytes = prefill_bytes(budgets)
+    score_evict_ms = float((phase[:, 0] + phase[:, 2]).mean() / L)
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": float(step_ms.mean()), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "q_heads": w.n_q_heads, "kv_heads": Hkv, "head_dim": d,
+                   "batch_per_gpu": B, "prompt": w.prompt, "window": W, "pool_kernel": w.pool_kernel,
+                   "avg_budget": w.avg_budget, "budgets": [int(x) for x in budgets], "decode_steps": n_dec,
+                   "page_size": sess.page_size, "parallelism": f"replicas x{world} (independent batches)",
+                   "l2": "inputs larger than L2 (K/V per layer 268 MB+, compacted caches of all layers > 126 MB)",
+                   "query_direction_reading": "window queries carry sqrt(d)*u so heavy hitters are heavy"},
+        "pct_of_hbm_peak": {"measured": 100.0 * value / world / peak, "nominal_8000": 100.0 * value / world / 8000.0},
+        "decode_tokens_per_s": tokens_per_s,
+        "score_evict_ms_per_layer": score_evict_ms,
+        "score_evict_roofline": {"algorithmic_bytes_per_layer": pre_bytes / L,
+                                 "achieved_GBps": pre_bytes / L / (score_evict_ms * 1e-3) / 1e9,
+                                 "frac_of_measured": pre_bytes / L / (score_evict_ms * 1e-3) / 1e9 / peak},
+        "phases_ms": {"score": float(phase[:, 0].mean()), "solver_and_page_table": float(phase[:, 1].mean()),
+                      "select_compact": float(phase[:, 2].mean()), "decode": float(phase[:, 3].mean())},
+        "timed_region_ms": region_ms_max,
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+        "clocks": clocks,
+        "paper_context": "paper reports end-to-end only (RTX A6000): 61.6% KV memory reduction, 2.1x compute "
+                         "efficiency, up to 5.2x throughput; no kernel-level number exists",
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

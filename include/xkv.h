@@ -217,6 +217,14 @@ size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen,
  */
 xkv_status xkv_read_device_status(const void* workspace, void* stream);
 
+/*
+ * Profiling hook (no counterpart in the paper): while both events are set, every xkv_decode_attn call
+ * records `start` on its stream immediately before its attention kernel and `stop` immediately after
+ * it, so a caller can time that kernel alone with cudaEventElapsedTime. Events are cudaEvent_t handles
+ * owned by the caller; pass NULL, NULL to switch the hook off (the default). Not thread-safe.
+ */
+void xkv_profile_events(void* start, void* stop);
+
 /* Number of kernel launches the library enqueued since it was loaded (all entry points). */
 int64_t xkv_launch_count(void);
 

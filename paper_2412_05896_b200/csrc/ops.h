@@ -23,4 +23,6 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
                        const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,
                        void* workspace, size_t workspace_bytes, cudaStream_t st);
 
+void set_profile_events(cudaEvent_t start, cudaEvent_t stop);
+
 }  // namespace xkv

@@ -177,6 +177,10 @@ xkv_status xkv_read_device_status(const void* workspace, void* stream) {
   return status;
 }
 
+void xkv_profile_events(void* start, void* stop) {
+  set_profile_events(static_cast<cudaEvent_t>(start), static_cast<cudaEvent_t>(stop));
+}
+
 int64_t xkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* xkv_status_string(xkv_status status) {

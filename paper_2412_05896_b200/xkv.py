@@ -21,7 +21,8 @@ POOL_MAX, POOL_AVG = 0, 1
 OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
 
 EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_workspace_bytes",
-           "xkv_read_device_status", "xkv_launch_count", "xkv_status_string", "xkv_version")
+           "xkv_read_device_status", "xkv_profile_events", "xkv_launch_count", "xkv_status_string",
+           "xkv_version")
 
 
 class XkvError(RuntimeError):
@@ -71,6 +72,8 @@ def lib() -> ctypes.CDLL:
     L.xkv_workspace_bytes.argtypes = [i32, ctypes.POINTER(Dims), i32, i64, i32, i32, i32]
     L.xkv_read_device_status.restype = i32
     L.xkv_read_device_status.argtypes = [vp, vp]
+    L.xkv_profile_events.restype = None
+    L.xkv_profile_events.argtypes = [vp, vp]
     L.xkv_launch_count.restype = i64
     L.xkv_launch_count.argtypes = []
     L.xkv_status_string.restype = ctypes.c_char_p
@@ -170,6 +173,12 @@ def decode_attn(dims: Dims, cache: Cache, layer_begin: int, layer_end: int, q, k
     _check(lib().xkv_decode_attn(ctypes.byref(dims), ctypes.byref(cache), layer_begin, layer_end, _ptr(q),
                                  _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse), chunk_rows, _ptr(workspace),
                                  _nbytes(workspace), _stream(stream)), "xkv_decode_attn")
+
+
+def profile_events(start, stop) -> None:
+    """start/stop: torch.cuda.Event(enable_timing=True) that have been recorded once, or None, None."""
+    lib().xkv_profile_events(None if start is None else start.cuda_event,
+                             None if stop is None else stop.cuda_event)
 
 
 def read_device_status(workspace, stream=None) -> int:
