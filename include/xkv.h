@@ -200,6 +200,35 @@ xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * xkv_decode_attn_static -- xkv_decode_attn for callers that cannot hand the library a workspace.
+ * (The paper has no counterpart: this is the same operation with a different memory arrangement.)
+ *
+ * Some hosts of this library may not allocate device memory at the point where they decode: code
+ * that runs inside a fixed memory plan (every buffer sized before the serving loop starts), plug-ins
+ * that only receive their input and output tensors from the framework around them, or code on a
+ * path where a cudaMalloc would stall the device. For them the scratch memory of the decode step
+ * (status word, merge tickets, work-item table, split-K partial results) is a fixed array of
+ * XKV_STATIC_SCRATCH_BYTES inside the library image. Every GPU that loads the library holds that
+ * array until the process exits. The call itself allocates and frees nothing.
+ *
+ * Arguments and results are those of xkv_decode_attn without workspace/workspace_bytes, plus
+ *   status_out  dev out int32 [1], may be NULL: receives the device status word of this call
+ *               (XKV_OK, XKV_ERR_CAPACITY, XKV_ERR_TIMEOUT) in stream order; copy it to the host to read it.
+ * Limits and rules
+ *   - Returns XKV_ERR_WORKSPACE, launching nothing, when the scratch this problem needs
+ *     (xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...)) exceeds XKV_STATIC_SCRATCH_BYTES.
+ *   - The first call on a device looks up the array's device address (a one-time set-up step);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each call
+ *     clears what it needs zeroed. Two calls that overlap on the GPU (different streams) race on
+ *     it: keep calls of this entry point on one stream, or order them yourself.
+ */
+#define XKV_STATIC_SCRATCH_BYTES (16u << 20)
+xkv_status xkv_decode_attn_static(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin,
+                                  int32_t layer_end, const void* q, const void* k_new, const void* v_new,
+                                  void* out, float* lse, int32_t chunk_rows, int32_t* status_out, void* stream);
+
+/*
  * Workspace size in bytes for one call of `op` (XKV_OP_*). Unused arguments may be 0.
  *   XKV_OP_SCORE, XKV_OP_SELECT_COMPACT: dims, max_seqlen, total_tokens
  *   XKV_OP_DECODE_ATTN: dims, n_layers (layers per call), max_cache_len (upper bound of any

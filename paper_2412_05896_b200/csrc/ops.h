@@ -23,6 +23,9 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
                        const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,
                        void* workspace, size_t workspace_bytes, cudaStream_t st);
 
+xkv_status decode_attn_static(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end,
+                              const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                              int chunk_rows, int32_t* status_out, cudaStream_t st);
 void set_profile_events(cudaEvent_t start, cudaEvent_t stop);
 
 }  // namespace xkv

@@ -147,6 +147,25 @@ xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t
                      workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
+xkv_status xkv_decode_attn_static(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin,
+                                  int32_t layer_end, const void* q, const void* k_new, const void* v_new,
+                                  void* out, float* lse, int32_t chunk_rows, int32_t* status_out, void* stream) {
+  xkv_status s = check_dims(dims);
+  if (s != XKV_OK) return s;
+  s = check_cache(cache, dims);
+  if (s != XKV_OK) return s;
+  if (q == nullptr || out == nullptr) return XKV_ERR_INVALID_ARG;
+  if ((k_new == nullptr) != (v_new == nullptr)) return XKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out) || !aligned16(lse) ||
+      (reinterpret_cast<uintptr_t>(status_out) & 3u) != 0)
+    return XKV_ERR_INVALID_ARG;
+  if (layer_begin < 0 || layer_end <= layer_begin || layer_end > cache->n_layers) return XKV_ERR_INVALID_ARG;
+  if (chunk_rows < 0 || chunk_rows % 64 != 0) return XKV_ERR_INVALID_ARG;
+  if (dims->n_q_heads / dims->n_kv_heads > 8) return XKV_ERR_UNSUPPORTED;
+  return decode_attn_static(dims, cache, layer_begin, layer_end, q, k_new, v_new, out, lse, chunk_rows,
+                            status_out, static_cast<cudaStream_t>(stream));
+}
+
 size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen, int64_t total_tokens,
                            int32_t n_layers, int32_t max_cache_len, int32_t chunk_rows) {
   if (dims == nullptr) return 0;

@@ -648,4 +648,38 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   return launch_attn<64>(tk, tv, p, st);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant: the scratch that decode_attn normally receives from the caller lives in
+// a fixed device array that is part of the library image.
+// ---------------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = XKV_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+xkv_status decode_attn_static(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end,
+                              const void* q, const void* k_new, const void* v_new, void* out, float* lse,
+                              int chunk_rows, int32_t* status_out, cudaStream_t st) {
+  // In host code g_static_scratch is only a handle for the symbol; the device address has to be
+  // asked for, once per device, while that device is current.
+  static void* scratch_ptr[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return XKV_ERR_CUDA;
+  if (scratch_ptr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return XKV_ERR_CUDA;
+    scratch_ptr[dev] = ptr;
+  }
+  const int max_cache_len = c->max_pages_per_seq * c->page_size;
+  const size_t need = decode_workspace_bytes(d, layer_end - layer_begin, max_cache_len, chunk_rows);
+  if (need == 0) return XKV_ERR_INVALID_ARG;
+  if (need > kStaticScratchBytes) return XKV_ERR_WORKSPACE;   // problem too large for the fixed scratch
+  // decode_attn clears the part of the scratch that must start at zero (status word, tickets)
+  xkv_status s = decode_attn(d, c, layer_begin, layer_end, q, k_new, v_new, out, lse, chunk_rows,
+                             scratch_ptr[dev], kStaticScratchBytes, st);
+  if (s != XKV_OK) return s;
+  if (status_out != nullptr &&
+      cudaMemcpyAsync(status_out, scratch_ptr[dev], sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return XKV_ERR_CUDA;
+  return XKV_OK;
+}
+
 }  // namespace xkv

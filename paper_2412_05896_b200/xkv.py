@@ -20,7 +20,10 @@ ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = -5, -6, -7
 POOL_MAX, POOL_AVG = 0, 1
 OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
 
-EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_workspace_bytes",
+STATIC_SCRATCH_BYTES = 16 << 20
+
+EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
+           "xkv_workspace_bytes",
            "xkv_read_device_status", "xkv_profile_events", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
 
@@ -68,6 +71,9 @@ def lib() -> ctypes.CDLL:
     L.xkv_decode_attn.restype = i32
     L.xkv_decode_attn.argtypes = [ctypes.POINTER(Dims), ctypes.POINTER(Cache), i32, i32, vp, vp, vp, vp, vp,
                                   i32, vp, sz, vp]
+    L.xkv_decode_attn_static.restype = i32
+    L.xkv_decode_attn_static.argtypes = [ctypes.POINTER(Dims), ctypes.POINTER(Cache), i32, i32, vp, vp, vp, vp,
+                                         vp, i32, vp, vp]
     L.xkv_workspace_bytes.restype = sz
     L.xkv_workspace_bytes.argtypes = [i32, ctypes.POINTER(Dims), i32, i64, i32, i32, i32]
     L.xkv_read_device_status.restype = i32
@@ -173,6 +179,16 @@ def decode_attn(dims: Dims, cache: Cache, layer_begin: int, layer_end: int, q, k
     _check(lib().xkv_decode_attn(ctypes.byref(dims), ctypes.byref(cache), layer_begin, layer_end, _ptr(q),
                                  _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse), chunk_rows, _ptr(workspace),
                                  _nbytes(workspace), _stream(stream)), "xkv_decode_attn")
+
+
+def decode_attn_static(dims: Dims, cache: Cache, layer_begin: int, layer_end: int, q, k_new, v_new, out, lse,
+                       chunk_rows: int, status_out=None, stream=None) -> None:
+    """xkv_decode_attn without a caller workspace: the scratch is a fixed array inside the library
+    (STATIC_SCRATCH_BYTES), for callers that must not allocate.  Raises XkvError(ERR_WORKSPACE) when the
+    problem needs more scratch than that.  Keep calls on one stream: they share the array."""
+    _check(lib().xkv_decode_attn_static(ctypes.byref(dims), ctypes.byref(cache), layer_begin, layer_end, _ptr(q),
+                                        _ptr(k_new), _ptr(v_new), _ptr(out), _ptr(lse), chunk_rows,
+                                        _ptr(status_out), _stream(stream)), "xkv_decode_attn_static")
 
 
 def profile_events(start, stop) -> None:
