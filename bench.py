@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -224,6 +225,8 @@ def main():
     w0 = WL.CONFIGS[args.workload]
     if args.decode_steps:
         w0 = replace(w0, decode_steps=args.decode_steps)
+    if args.layers:
+        w0 = replace(w0, n_layers=args.layers)
     w = replace(w0, seed=w0.seed + 7919 * rank)          # every rank draws its own batch
     L, B, Hkv, d, W = w.n_layers, w.batch, w.n_kv_heads, w.head_dim, w.window
     lengths = WL.prompt_lengths(w)
