@@ -17,7 +17,9 @@ struct WorkspaceHeader {
   int32_t status;      // XKV_OK or the first XKV_ERR_* recorded by a kernel
   int32_t n_items;     // decode: number of work items planned on the device
   int32_t chunk_rows;  // decode: rows per chunk chosen by the plan
-  int32_t reserved[61];
+  int32_t work_counter;  // decode: next work item to hand to a warp
+  int32_t prep_ticket;   // decode: CTAs of the prepare kernel that have finished
+  int32_t reserved[59];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

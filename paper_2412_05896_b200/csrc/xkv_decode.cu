@@ -2,19 +2,22 @@
 // compacted per-layer caches.
 //
 // Kernels, in stream order:
-//   decode_append_kernel  one warp per (layer, sequence): store the new K/V row of every KV head in
-//                         slot seq_lens[l][b] and advance seq_lens.
-//   decode_plan_kernel    one CTA: cut every (layer, sequence, KV head) cache into chunks of rows and
-//                         write the work-item table; the chunk size is chosen from the total length.
-//   decode_attn_kernel    persistent CTAs, one producer warp + four consumer warps.  The producer
-//                         streams 64-row K and V tiles of a work item into a ring of shared-memory
-//                         stages with TMA tensor loads (16-row boxes, 128-byte swizzle) that complete
-//                         on mbarriers; each consumer warp owns 16 rows of a tile and runs online
-//                         softmax with mma.sync m16n8k16 for q.K^T and P.V (the G query heads of the
-//                         group sit on the M axis).  Chunk results are merged by log-sum-exp, by the
-//                         CTA itself when the unit has one chunk, else by the last CTA to finish a
-//                         chunk of that unit (atomic ticket, no waiting).
-// The path is HBM-bound: 4*d bytes per cached row per KV head per step.
+//   decode_prepare_kernel  one CTA per (layer, sequence): store the new K/V row of every KV head in
+//                          slot seq_lens[l][b] and advance seq_lens; the last CTA to finish then cuts
+//                          every (layer, sequence, KV head) cache into chunks of rows and writes the
+//                          work-item table (the chunk size is chosen from the total cached length).
+//   decode_attn_kernel     persistent CTAs of eight independent warps.  A warp takes work items
+//                          from a global counter and streams its item's K and V rows through its own
+//                          ring of shared-memory stages: 16-row TMA tensor boxes (128-byte swizzle)
+//                          that complete on an mbarrier, issued by the warp itself a few tiles ahead
+//                          of where it computes, across item boundaries.  Per tile it runs online
+//                          softmax with mma.sync m16n8k16 for q.K^T and P.V (the G query heads of the
+//                          group sit on the M axis).  A unit with one chunk is normalised and stored by
+//                          its warp; otherwise partial (m, l, acc) go to the workspace and the last
+//                          warp to finish a chunk of the unit merges them by log-sum-exp (atomic
+//                          ticket, no waiting).
+// The path is HBM-bound: 4*d bytes per cached row per KV head per step; warps never wait for each
+// other, so item boundaries of one warp overlap with streaming in the others.
 #include <cuda.h>
 
 #include <cmath>
@@ -27,13 +30,15 @@ namespace xkv {
 
 namespace {
 
-constexpr int kTileRows = 64;        // cache rows per pipeline stage
-constexpr int kBoxRows = 16;         // rows per TMA box; page_size is a multiple of it
-constexpr int kConsumerWarps = 4;
-constexpr int kDecodeThreads = (kConsumerWarps + 1) * 32;
-constexpr int kTargetItems = 16 * 148;  // auto chunking aims at about this many extra work items
+constexpr int kTileRows = 16;        // cache rows per pipeline stage = one TMA box; page_size is a multiple
+constexpr int kChunkAlign = 64;      // chunk_rows granularity
+constexpr int kAttnWarps = 8;
+constexpr int kAttnThreads = kAttnWarps * 32;
+constexpr int kTargetItems = 4 * 148 * kAttnWarps;  // auto chunking aims at about this many extra work items
 constexpr int kMinChunkRows = 256;
 constexpr int kMaxGroup = 8;
+constexpr int kFifo = 4;             // work items a warp may have fetched but not yet finished
+constexpr int kPrepThreads = 256;
 
 struct DecodeParams {
   const __nv_bfloat16* q;
@@ -60,54 +65,30 @@ struct DecodeParams {
 template <int D>
 struct Cfg {
   static constexpr int kHalves = D / 64;                       // 128-byte swizzled column halves
-  static constexpr int kHalfBytes = kTileRows * 128;           // one half of a K or V tile
-  static constexpr int kTileBytes = kHalves * kHalfBytes;
+  static constexpr int kBoxBytes = kTileRows * 128;            // one half of a K or V tile (one TMA box)
+  static constexpr int kTileBytes = kHalves * kBoxBytes;
   static constexpr int kStageBytes = 2 * kTileBytes;           // K tile + V tile
-  static constexpr int kStages = (D == 128) ? 6 : 8;
-  static constexpr int kScratchFloats = kConsumerWarps * kMaxGroup * (D + 2);
-  static constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kScratchFloats * 4 + 2 * kStages * 8 + 64;
+  static constexpr int kStages = (D == 128) ? 3 : 6;
+  static constexpr int kRingBytes = kStages * kStageBytes;     // per warp
+  static constexpr int kSmemBytes = 1024 + kAttnWarps * kRingBytes + kAttnWarps * kStages * 8 +
+                                    kAttnWarps * kFifo * 16 + 64;
 };
 
 // ---------------------------------------------------------------------------------------------
-__global__ void decode_append_kernel(DecodeParams p, int D) {
-  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  const int n_units = p.n_layers * p.batch;
-  if (warp >= n_units) return;
-  const int l_rel = warp / p.batch, b = warp % p.batch;
-  const int le = (p.layer_begin + l_rel) * p.batch + b;
-  const int n = p.seq_lens[le];
-  const int32_t* bt = p.block_table + (size_t)le * p.max_pages_per_seq;
-  int page = -1;
-  if (n >= 0 && n < p.max_pages_per_seq * p.page_size) page = bt[n / p.page_size];
-  if (page < 0 || page >= p.n_pages) {
-    if (lane == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
-    return;
-  }
-  const int chunks = D / 8;
-  for (int idx = lane; idx < p.n_kv_heads * chunks; idx += 32) {
-    const int h = idx / chunks, c = idx % chunks;
-    const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
-    const size_t src = ((size_t)warp * p.n_kv_heads + h) * D + c * 8;
-    *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
-    *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
-  }
-  __syncwarp();
-  if (lane == 0) p.seq_lens[le] = n + 1;
-}
-
+// Append (optional) and plan.  grid = n_layers*batch CTAs when appending, else 1.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
+__device__ void plan_items(const DecodeParams& p) {
   __shared__ long long s_red[32];
   __shared__ int s_scan[32];
   __shared__ int s_carry;
   __shared__ int s_chunk;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int n_warps = blockDim.x >> 5;
   const int n_units = p.n_layers * p.batch;
 
   long long rows = 0;
   for (int e = tid; e < n_units; e += blockDim.x) {
-    const int n = p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch];
+    const int n = __ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]);
     rows += n > 0 ? n : 0;
   }
   for (int o = 16; o > 0; o >>= 1) rows += __shfl_xor_sync(0xffffffffu, rows, o);
@@ -115,12 +96,12 @@ __global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
   __syncthreads();
   if (tid == 0) {
     long long total = 0;
-    for (int w = 0; w < 32; ++w) total += s_red[w];
+    for (int w = 0; w < n_warps; ++w) total += s_red[w];
     total *= p.n_kv_heads;
     int chunk = p.chunk_rows_forced;
     if (chunk <= 0) {
       long long c = (total + kTargetItems - 1) / kTargetItems;
-      c = (c + kTileRows - 1) / kTileRows * kTileRows;
+      c = (c + kChunkAlign - 1) / kChunkAlign * kChunkAlign;
       if (c < kMinChunkRows) c = kMinChunkRows;
       if (c > (1 << 30)) c = 1 << 30;
       chunk = (int)c;
@@ -136,7 +117,7 @@ __global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
     const int e = base + tid;
     int n = 0, nc = 0;
     if (e < n_units) {
-      n = p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch];
+      n = __ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]);
       if (n < 0) n = 0;
       nc = n == 0 ? 1 : (n + chunk - 1) / chunk;
     }
@@ -148,7 +129,7 @@ __global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
     if (lane == 31) s_scan[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int v = s_scan[lane], inc = v;
+      int v = lane < n_warps ? s_scan[lane] : 0, inc = v;
       for (int o = 1; o < 32; o <<= 1) {
         const int u = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= o) inc += u;
@@ -185,6 +166,52 @@ __global__ void __launch_bounds__(1024) decode_plan_kernel(DecodeParams p) {
   }
 }
 
+__global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodeParams p, int D, int do_append) {
+  __shared__ int s_page;
+  __shared__ int s_last;
+  const int tid = threadIdx.x;
+  if (do_append) {
+    const int e = blockIdx.x;
+    const int l_rel = e / p.batch, b = e % p.batch;
+    const int le = (p.layer_begin + l_rel) * p.batch + b;
+    const int n = p.seq_lens[le];
+    if (tid == 0) {
+      int page = -1;
+      if (n >= 0 && n < p.max_pages_per_seq * p.page_size)
+        page = p.block_table[(size_t)le * p.max_pages_per_seq + n / p.page_size];
+      if (page < 0 || page >= p.n_pages) {
+        page = -1;
+        record_status(p.hdr, XKV_ERR_CAPACITY);
+      }
+      s_page = page;
+    }
+    __syncthreads();
+    const int page = s_page;
+    if (page >= 0) {
+      const int chunks = D / 8;
+      for (int idx = tid; idx < p.n_kv_heads * chunks; idx += blockDim.x) {
+        const int h = idx / chunks, c = idx % chunks;
+        const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
+        const size_t src = ((size_t)e * p.n_kv_heads + h) * D + c * 8;
+        *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
+        *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
+      }
+      if (tid == 0) p.seq_lens[le] = n + 1;
+    }
+  }
+  // the last CTA to get here sees every sequence length already advanced and writes the plan
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int ticket = atomicAdd(&p.hdr->prep_ticket, 1);
+    s_last = (ticket == (int)gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  plan_items(p);
+}
+
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint64_t global_timer_ns() {
   uint64_t t;
@@ -204,24 +231,21 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
 }
 
 template <int D>
-__global__ void __launch_bounds__(kDecodeThreads, 1)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const DecodeParams p) {
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* stages = smem;
-  float* scratch = reinterpret_cast<float*>(smem + C::kStages * C::kStageBytes);
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + C::kScratchFloats);
-  uint64_t* empty_bar = full_bar + C::kStages;
-  int* s_flag = reinterpret_cast<int*>(empty_bar + C::kStages);
-
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint8_t* ring = smem + (size_t)warp * C::kRingBytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes) + warp * C::kStages;
+  int4* fifo = reinterpret_cast<int4*>(smem + (size_t)kAttnWarps * C::kRingBytes + kAttnWarps * C::kStages * 8) +
+               warp * kFifo;
+
   if (tid == 0) {
-    for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], kConsumerWarps);
-    }
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes);
+    for (int s = 0; s < kAttnWarps * C::kStages; ++s) mbar_init(&bars[s], 1);
     fence_mbar_init();
     prefetch_tmap(&tmap_k);
     prefetch_tmap(&tmap_v);
@@ -229,68 +253,86 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   __syncthreads();
 
   const int n_items = p.hdr->n_items;
-  const int chunk_rows = p.hdr->chunk_rows;
-  (void)chunk_rows;
-
-  if (warp == kConsumerWarps) {
-    // ------------------------------------------------------------------ producer warp
-    uint32_t it = 0;
-    bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-      const int4 I = p.items[item];
-      const int e = I.x, h = I.y;
-      const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
-      const int32_t* bt = p.block_table + (size_t)le * p.max_pages_per_seq;
-      for (int r0 = I.z; r0 < I.w; r0 += kTileRows, ++it) {
-        const int s = it % C::kStages;
-        const uint32_t ph = (it / C::kStages) & 1u;
-        const int valid = min(kTileRows, I.w - r0);
-        const int nbox = (valid + kBoxRows - 1) / kBoxRows;
-        int grow = 0;
-        if (lane < nbox) {
-          const int slot = r0 + kBoxRows * lane;
-          int page = bt[slot / p.page_size];
-          page = min(max(page, 0), p.n_pages - 1);
-          grow = (page * p.n_kv_heads + h) * p.page_size + slot % p.page_size;
-        }
-        if (lane == 0) {
-          ok = mbar_wait_bounded(&empty_bar[s], ph ^ 1u);
-          if (ok) mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(nbox * kBoxRows * D * 2 * 2));
-        }
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        if (lane < nbox) {
-          uint8_t* ks = stages + (size_t)s * C::kStageBytes;
-          uint8_t* vs = ks + C::kTileBytes;
-#pragma unroll
-          for (int hf = 0; hf < C::kHalves; ++hf) {
-            tma_load_2d(ks + hf * C::kHalfBytes + lane * kBoxRows * 128, &tmap_k, hf * 64, grow, &full_bar[s]);
-            tma_load_2d(vs + hf * C::kHalfBytes + lane * kBoxRows * 128, &tmap_v, hf * 64, grow, &full_bar[s]);
-          }
-        }
-      }
-    }
-    if (!ok) {
-      if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
-      // let copies already issued land before the CTA's shared memory can be handed on
-      for (int i = 0; i < 1000; ++i) __nanosleep(1000);
-    }
-    return;
-  }
-
-  // -------------------------------------------------------------------- consumer warps
   const int gid = lane >> 2, tig = lane & 3;
   const int mat = lane >> 3, mrow = lane & 7;
   const int G = p.group;
-  const int ctid = tid;  // 0..127
-  uint32_t it = 0;
-  bool aborted = false;
-  float* scr_o = scratch;                                        // [4][8][D]
-  float* scr_ml = scratch + kConsumerWarps * kMaxGroup * D;      // [4][8][2]
+  constexpr uint32_t kTxBytes = C::kStageBytes;
 
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  // ---- producer side of this warp: runs up to kStages tiles ahead of the consumer side
+  bool p_valid = false, no_more = false, aborted = false;
+  int4 p_desc = make_int4(0, 0, 0, 0);
+  int p_row = 0, p_page_tile0 = 0, p_pages = 0, p_item = 0;
+  const int32_t* p_bt = p.block_table;
+  int fifo_head = 0, fifo_count = 0;
+  uint32_t issued = 0, consumed = 0;
+  int next_idx = 0;
+  if (lane == 0) next_idx = atomicAdd(&p.hdr->work_counter, 1);
+
+  auto produce_one = [&]() -> bool {
+    while (true) {
+      if (!p_valid) {
+        if (no_more || fifo_count == kFifo) return false;
+        const int idx = __shfl_sync(0xffffffffu, next_idx, 0);
+        if (idx >= n_items) {
+          no_more = true;
+          return false;
+        }
+        if (lane == 0) next_idx = atomicAdd(&p.hdr->work_counter, 1);   // fetched early, used at the next item
+        p_desc = p.items[idx];
+        p_item = idx;
+        const int slot = (fifo_head + fifo_count) % kFifo;
+        if (lane == 0) fifo[slot] = make_int4(idx, 0, 0, 0);
+        ++fifo_count;
+        p_row = p_desc.z;
+        if (p_row >= p_desc.w) continue;          // empty cache: the consumer side writes zeros
+        const int e = p_desc.x;
+        const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
+        p_bt = p.block_table + (size_t)le * p.max_pages_per_seq;
+        p_page_tile0 = -1000000;
+        p_valid = true;
+      }
+      const int tile = p_row / kTileRows;
+      if (tile - p_page_tile0 >= 32 || tile < p_page_tile0) {       // refill the page ids of the next 32 tiles
+        p_page_tile0 = tile;
+        const int slot_row = (tile + lane) * kTileRows;
+        p_pages = slot_row < p_desc.w ? p_bt[slot_row / p.page_size] : 0;
+      }
+      int page = __shfl_sync(0xffffffffu, p_pages, tile - p_page_tile0);
+      page = min(max(page, 0), p.n_pages - 1);
+      if (lane == 0) {
+        const int grow = (page * p.n_kv_heads + p_desc.y) * p.page_size + p_row % p.page_size;
+        const int s = issued % C::kStages;
+        uint8_t* ks = ring + (size_t)s * C::kStageBytes;
+        uint8_t* vs = ks + C::kTileBytes;
+        mbar_arrive_expect_tx(&full_bar[s], kTxBytes);
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf) {
+          tma_load_2d(ks + hf * C::kBoxBytes, &tmap_k, hf * 64, grow, &full_bar[s]);
+          tma_load_2d(vs + hf * C::kBoxBytes, &tmap_v, hf * 64, grow, &full_bar[s]);
+        }
+      }
+      ++issued;
+      p_row += kTileRows;
+      if (p_row >= p_desc.w) p_valid = false;
+      return true;
+    }
+  };
+  auto fill = [&]() {
+    while (!aborted && issued - consumed < (uint32_t)C::kStages && produce_one()) {
+    }
+  };
+
+  // ---- consumer side
+  while (true) {
+    fill();
+    if (fifo_count == 0) break;
+    __syncwarp();
+    const int item = fifo[fifo_head].x;
+    fifo_head = (fifo_head + 1) % kFifo;
+    --fifo_count;
     const int4 I = p.items[item];
     const int e = I.x, h = I.y;
+    const int nc = p.unit_info[e].y;
     const size_t q_row0 = ((size_t)e * p.n_q_heads + (size_t)h * G);
 
     uint32_t qa[D / 16][2];
@@ -309,39 +351,42 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = 0.f;
     float m_run = -INFINITY, l_part = 0.f;
 
-    for (int r0 = I.z; r0 < I.w; r0 += kTileRows, ++it) {
-      const int s = it % C::kStages;
-      const uint32_t ph = (it / C::kStages) & 1u;
-      const int valid = min(kTileRows, I.w - r0);
-      if (!aborted && !mbar_wait_bounded(&full_bar[s], ph)) {
-        aborted = true;
-        if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+    for (int r0 = I.z; r0 < I.w; r0 += kTileRows) {
+      if (issued == consumed) fill();
+      const int s = consumed % C::kStages;
+      const uint32_t ph = (consumed / C::kStages) & 1u;
+      if (!aborted) {
+        const bool ok = (issued != consumed) && mbar_wait_bounded(&full_bar[s], ph);
+        if (!__all_sync(0xffffffffu, ok)) {
+          aborted = true;
+          no_more = true;
+          if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+        }
       }
-      const int wrows = valid - kBoxRows * warp;
-      bool touched = false;
-      if (!aborted && wrows > 0) {
-        const uint32_t ks_base = smem_u32(stages + (size_t)s * C::kStageBytes);
+      const int wrows = min(kTileRows, I.w - r0);
+      if (!aborted) {
+        const uint32_t ks_base = smem_u32(ring + (size_t)s * C::kStageBytes);
         const uint32_t vs_base = ks_base + C::kTileBytes;
-        if (wrows < kBoxRows) {
+        if (wrows < kTileRows) {
           // rows past the end of the cache hold whatever the page held: clear V so 0 * x stays 0
-          uint8_t* vs = stages + (size_t)s * C::kStageBytes + C::kTileBytes;
-          const int n_bad = kBoxRows - wrows;
+          uint8_t* vs = ring + (size_t)s * C::kStageBytes + C::kTileBytes;
+          const int n_bad = kTileRows - wrows;
           for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
-            const int row = kBoxRows * warp + wrows + idx / (D / 8);
+            const int row = wrows + idx / (D / 8);
             const int c = idx % (D / 8);
-            *reinterpret_cast<uint4*>(vs + (c >> 3) * C::kHalfBytes + row * 128 + (c & 7) * 16) =
+            *reinterpret_cast<uint4*>(vs + (c >> 3) * C::kBoxBytes + row * 128 + (c & 7) * 16) =
                 make_uint4(0u, 0u, 0u, 0u);
           }
-          touched = true;
+          fence_proxy_async_smem();
           __syncwarp();
         }
         // S[heads x 16 keys] = Q K^T
         float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const int key = kBoxRows * warp + (mat >> 1) * 8 + mrow;
+          const int key = (mat >> 1) * 8 + mrow;
           const int c = 2 * ks + (mat & 1);
-          const uint32_t addr = ks_base + (c >> 3) * C::kHalfBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
+          const uint32_t addr = ks_base + (c >> 3) * C::kBoxBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
           uint32_t bfrag[4];
           ldmatrix_x4(bfrag, addr);
           const uint32_t a[4] = {qa[ks][0], 0u, qa[ks][1], 0u};
@@ -381,9 +426,9 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const uint32_t pa[4] = {pack_bf16(pr[0][0], pr[0][1]), 0u, pack_bf16(pr[1][0], pr[1][1]), 0u};
 #pragma unroll
         for (int dp = 0; dp < D / 16; ++dp) {
-          const int key = kBoxRows * warp + (mat & 1) * 8 + mrow;
+          const int key = (mat & 1) * 8 + mrow;
           const int c = 2 * dp + (mat >> 1);
-          const uint32_t addr = vs_base + (c >> 3) * C::kHalfBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
+          const uint32_t addr = vs_base + (c >> 3) * C::kBoxBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
           uint32_t bfrag[4];
           ldmatrix_x4_trans(bfrag, addr);
           float c0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
@@ -396,67 +441,45 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           o[2 * dp + 1][1] = c1[1];
         }
       }
-      if (touched) fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[s]);
+      ++consumed;
+      fill();                                   // the stage just released takes the next tile
     }
 
-    // ---- merge the four warps' partial results of this work item
+    // ---- finish the work item
     float l_row = l_part;
     l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
     l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
-    if (gid < G) {
+    if (nc == 1) {
+      if (gid < G) {
+        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+        __nv_bfloat16* orow = p.out + (q_row0 + gid) * D;
 #pragma unroll
-      for (int nt = 0; nt < D / 8; ++nt)
-        *reinterpret_cast<float2*>(&scr_o[(warp * kMaxGroup + gid) * D + 8 * nt + 2 * tig]) =
-            make_float2(o[nt][0], o[nt][1]);
-      if (tig == 0) {
-        scr_ml[(warp * kMaxGroup + gid) * 2 + 0] = m_run;
-        scr_ml[(warp * kMaxGroup + gid) * 2 + 1] = l_row;
+        for (int nt = 0; nt < D / 8; ++nt)
+          *reinterpret_cast<uint32_t*>(orow + 8 * nt + 2 * tig) = pack_bf16(o[nt][0] * inv, o[nt][1] * inv);
+        if (tig == 0 && p.lse != nullptr)
+          p.lse[q_row0 + gid] = l_row > 0.f ? (m_run + log2f(l_row)) * 0.6931471805599453f : -INFINITY;
       }
-    }
-    named_bar_sync(1, kConsumerWarps * 32);
-
-    const int nc = p.unit_info[e].y;
-    for (int idx = ctid; idx < G * D; idx += kConsumerWarps * 32) {
-      const int g = idx / D, dc = idx % D;
-      float mmax = -INFINITY;
+    } else {
+      if (gid < G) {
+        float* po = p.part_o + ((size_t)item * G + gid) * D;
 #pragma unroll
-      for (int w = 0; w < kConsumerWarps; ++w) mmax = fmaxf(mmax, scr_ml[(w * kMaxGroup + g) * 2]);
-      float num = 0.f, den = 0.f;
-      if (mmax > -INFINITY) {
-#pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
-          const float a = fast_exp2(scr_ml[(w * kMaxGroup + g) * 2] - mmax);
-          num += a * scr_o[(w * kMaxGroup + g) * D + dc];
-          den += a * scr_ml[(w * kMaxGroup + g) * 2 + 1];
+        for (int nt = 0; nt < D / 8; ++nt)
+          *reinterpret_cast<float2*>(po + 8 * nt + 2 * tig) = make_float2(o[nt][0], o[nt][1]);
+        if (tig == 0) {
+          p.part_ml[((size_t)item * G + gid) * 2 + 0] = m_run;
+          p.part_ml[((size_t)item * G + gid) * 2 + 1] = l_row;
         }
       }
-      if (nc == 1) {
-        const size_t row = q_row0 + g;
-        p.out[row * D + dc] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
-        if (dc == 0 && p.lse != nullptr)
-          p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
-      } else {
-        p.part_o[((size_t)item * G + g) * D + dc] = num;
-        if (dc == 0) {
-          p.part_ml[((size_t)item * G + g) * 2 + 0] = mmax;
-          p.part_ml[((size_t)item * G + g) * 2 + 1] = den;
-        }
-      }
-    }
-    if (nc > 1) {
       __threadfence();
-      named_bar_sync(1, kConsumerWarps * 32);
-      if (ctid == 0) {
-        const int old = atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1);
-        *s_flag = (old == nc - 1) ? 1 : 0;
-      }
-      named_bar_sync(1, kConsumerWarps * 32);
-      if (*s_flag) {
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) last = (atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1) == nc - 1) ? 1 : 0;
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
         __threadfence();
         const int first = p.unit_info[e].x + h * nc;
-        for (int idx = ctid; idx < G * D; idx += kConsumerWarps * 32) {
+        for (int idx = lane; idx < G * D; idx += 32) {
           const int g = idx / D, dc = idx % D;
           float mmax = -INFINITY;
           for (int c = 0; c < nc; ++c) mmax = fmaxf(mmax, __ldcg(&p.part_ml[((size_t)(first + c) * G + g) * 2]));
@@ -474,10 +497,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           if (dc == 0 && p.lse != nullptr)
             p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
         }
-        if (ctid == 0) p.tickets[e * p.n_kv_heads + h] = 0;
+        if (lane == 0) p.tickets[e * p.n_kv_heads + h] = 0;
       }
     }
-    named_bar_sync(1, kConsumerWarps * 32);   // scratch and flag are reused by the next item
+  }
+  if (aborted) {
+    // let copies already issued land before this CTA's shared memory can be handed on
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);
   }
 }
 
@@ -506,7 +532,7 @@ bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows) {
   if (enc == nullptr) return false;
   const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
-  const cuuint32_t box[2] = {64u, (cuuint32_t)kBoxRows};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)kTileRows};
   const cuuint32_t estr[2] = {1u, 1u};
   return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -561,7 +587,7 @@ xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const Decod
     done[dev] = true;
   }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_start, st);
-  decode_attn_kernel<D><<<sm_count(), kDecodeThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
+  decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_stop, st);
   count_launch();
   return check_launch();
@@ -586,7 +612,7 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   const int Lr = layer_end - layer_begin;
   const int G = d->n_q_heads / d->n_kv_heads;
   if (G > kMaxGroup) return XKV_ERR_UNSUPPORTED;
-  if (chunk_rows < 0 || chunk_rows % kTileRows != 0) return XKV_ERR_INVALID_ARG;
+  if (chunk_rows < 0 || chunk_rows % kChunkAlign != 0) return XKV_ERR_INVALID_ARG;
   const int max_cache_len = c->max_pages_per_seq * c->page_size;
   DecodeLayout L;
   if (!decode_layout(d, Lr, max_cache_len, chunk_rows, &L)) return XKV_ERR_INVALID_ARG;
@@ -632,15 +658,8 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
 
   if (cudaMemsetAsync(ws, 0, L.unit_info, st) != cudaSuccess) return XKV_ERR_CUDA;   // header + tickets
   const int n_units = Lr * d->batch;
-  if (k_new != nullptr) {
-    const int warps_per_block = 8;
-    decode_append_kernel<<<(n_units + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, st>>>(
-        p, d->head_dim);
-    count_launch();
-    xkv_status s = check_launch();
-    if (s != XKV_OK) return s;
-  }
-  decode_plan_kernel<<<1, 1024, 0, st>>>(p);
+  const int do_append = k_new != nullptr ? 1 : 0;
+  decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append);
   count_launch();
   xkv_status s = check_launch();
   if (s != XKV_OK) return s;
