@@ -1,11 +1,16 @@
 // xkv_score: importance scoring of one layer (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4).
 //
 // Kernels, in stream order:
-//   score_pass_kernel<D,1>  softmax row statistics (max, sum of exponentials) of the G*W window
-//                           query rows over their visible keys, per split of the key axis
-//   stats_merge_kernel      merge the per-split statistics into one log2-domain normaliser per row
-//   score_pass_kernel<D,2>  recompute the logits and accumulate the column sums u[c] over the
-//                           G*W rows (Select + Merge; the GQA group is summed before pooling)
+//   score_resident_kernel<D> / score_stream_kernel<D>  persistent CTAs working through key splits:
+//                           pass 1  softmax row statistics (max, sum of exponentials) of the G*W
+//                                   window query rows over their visible keys; the last split of a
+//                                   unit merges them into one log2-domain normaliser per row
+//                           pass 2  recompute the logits and accumulate the column sums u[c] over
+//                                   the G*W rows (Select + Merge; the GQA group is summed before
+//                                   pooling)
+//                           The resident variant keeps a split's keys in shared memory between the
+//                           passes (K is read from HBM once); the streaming variant, for sequences
+//                           too long for that, runs all pass-1 items and then all pass-2 items.
 //   pool_sort_kernel        1-D pooling (max or zero-padded average) of u into the scores w, and a
 //                           descending bitonic sort of each 4096-score chunk in shared memory
 //   merge_kernel            merge-path passes that combine the sorted chunks of a segment
@@ -23,10 +28,6 @@
 
 namespace xkv {
 namespace {
-
-#ifndef XKV_SPLIT_ACC
-#define XKV_SPLIT_ACC 1
-#endif
 
 constexpr int kPassThreads = 128;     // 4 warps
 constexpr int kKeyTile = 128;         // keys per tile, 32 per warp
@@ -49,244 +50,393 @@ struct ScoreParams {
   float2* stats_part;  // [units][n_splits][M]
   float* mrow;         // [units][M]
   float* part_sum;     // [units][n_chunks]
+  WorkspaceHeader* hdr;
+  int32_t* unit_ticket;  // [units] pass-1 items of the unit that have finished
+  int32_t* unit_ready;   // [units] 1 once mrow of the unit is final
+  int32_t slice_tiles, n_work;
   int64_t total_tokens, stride_token, stride_head;
   int32_t batch, n_q_heads, n_kv_heads, group, window, M, pool_kernel, pool_mode;
   int32_t split_keys, n_splits, n_chunks, curve_len;
   float scale_log2;
 };
 
+constexpr int kPassStages = 3;        // cp.async ring of key tiles (streaming variant)
+
 template <int D>
 struct PassCfg {
-  static constexpr int kRowElems = D + 8;   // padded shared-memory row: conflict-free ldmatrix
-  static constexpr int kRowBytes = kRowElems * 2;
+  static constexpr int kRowBytes = D * 2;                 // unpadded rows, 16-byte chunks XOR-swizzled
   static constexpr int kTileBytes = kKeyTile * kRowBytes;
-  static size_t smem_bytes(int M) { return (size_t)M * kRowBytes + 2 * kTileBytes + (size_t)4 * M * 8; }
+  static size_t smem_bytes(int M, int tiles) {
+    return (size_t)M * kRowBytes + (size_t)tiles * kTileBytes + (size_t)4 * M * 8 + 64;
+  }
 };
 
-// One CTA: unit (b, g) = blockIdx.x, key range split = blockIdx.y.
+// Byte offset of 16-byte chunk c of row r: chunks are XOR-swizzled inside each 128-byte segment so that
+// ldmatrix reads of eight consecutive rows hit distinct banks.
+__device__ __forceinline__ uint32_t swz(int r, int c, int row_bytes) {
+  return (uint32_t)(r * row_bytes + ((c >> 3) << 7) + (((c & 7) ^ (r & 7)) << 4));
+}
+
+__device__ __forceinline__ int ld_acquire(const int* ptr) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ uint64_t timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+struct UnitShape {
+  int b, g, cu, t, P;
+};
+
+__device__ __forceinline__ UnitShape unit_shape(const ScoreParams& p, int unit) {
+  UnitShape s;
+  s.b = unit / p.n_kv_heads;
+  s.g = unit % p.n_kv_heads;
+  s.cu = p.cu_seqlens[s.b];
+  s.t = p.cu_seqlens[s.b + 1] - s.cu;
+  s.P = max(s.t - p.window, 0);
+  return s;
+}
+
+template <int D>
+__device__ __forceinline__ void load_q(const ScoreParams& p, const UnitShape& us, uint8_t* q_s) {
+  constexpr int kChunks = D / 8;
+  const __nv_bfloat16* qg = p.q_win + ((size_t)us.b * p.n_q_heads + (size_t)us.g * p.group) * p.window * D;
+  for (int idx = threadIdx.x; idx < p.M * kChunks; idx += kPassThreads) {
+    const int r = idx / kChunks, c = idx % kChunks;
+    cp_async_16(smem_u32(q_s) + swz(r, c, D * 2), qg + (size_t)r * D + c * 8, 16);
+  }
+}
+
+template <int D>
+__device__ __forceinline__ void load_k_tile(const ScoreParams& p, const UnitShape& us, uint8_t* dst, int tile_c0) {
+  constexpr int kChunks = D / 8;
+  const __nv_bfloat16* kg = p.k + (size_t)us.cu * p.stride_token + (size_t)us.g * p.stride_head;
+  for (int idx = threadIdx.x; idx < kKeyTile * kChunks; idx += kPassThreads) {
+    const int r = idx / kChunks, c = idx % kChunks;
+    const int key = tile_c0 + r;
+    const bool in = key < us.t;
+    const __nv_bfloat16* src = kg + (size_t)(in ? key : 0) * p.stride_token + c * 8;
+    cp_async_16(smem_u32(dst) + swz(r, c, D * 2), src, in ? 16 : 0);
+  }
+}
+
+// One 128-key tile against all G*W query rows.  A warp owns 32 keys, keeps their B fragments in
+// registers and sweeps the query rows 16 at a time.
+// PASS 1: online (max, sum of exponentials) per query row in `st` = this warp's [M][2] state.
+// PASS 2: `st` = [M] row normalisers (log2 domain); column sums of the tile go to u for keys < key_end.
 template <int D, int PASS>
-__global__ void __launch_bounds__(kPassThreads) score_pass_kernel(const ScoreParams p) {
-  using C = PassCfg<D>;
-  extern __shared__ __align__(16) uint8_t smem[];
-  const int M = p.M;
-  uint8_t* q_s = smem;
-  uint8_t* k_s = smem + (size_t)M * C::kRowBytes;
-  float* state = reinterpret_cast<float*>(k_s + 2 * C::kTileBytes);   // pass 1: [4][M][2]; pass 2: [M]
-
-  const int unit = blockIdx.x;
-  const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
-  const int cu = p.cu_seqlens[b];
-  const int t = p.cu_seqlens[b + 1] - cu;
-  const int P = max(t - p.window, 0);
-  const int key_end_all = (PASS == 1) ? t : P;
-  const int key_begin = blockIdx.y * p.split_keys;
-  const int key_end = min(key_begin + p.split_keys, key_end_all);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__device__ __forceinline__ void compute_tile(const ScoreParams& p, const UnitShape& us, uint32_t q_base,
+                                             uint32_t k_base, float* st, int tile_c0, int key_end) {
+  constexpr int kRB = D * 2;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int gid = lane >> 2, tig = lane & 3, mat = lane >> 3, mrow_l = lane & 7;
+  const int MT = p.M / 16;
 
-  if (PASS == 1) {
-    float2* out = p.stats_part + ((size_t)unit * p.n_splits + blockIdx.y) * M;
-    if (key_begin >= key_end) {       // empty split: neutral statistics
-      for (int r = tid; r < M; r += kPassThreads) out[r] = make_float2(-INFINITY, 0.f);
-      return;
-    }
-  } else if (key_begin >= key_end) {
-    return;
-  }
-
-  // ---- stage the query rows of the group (G*W x D) and the first key tile
-  const __nv_bfloat16* qg = p.q_win + ((size_t)b * p.n_q_heads + (size_t)g * p.group) * p.window * D;
-  constexpr int kChunksPerRow = D / 8;
-  for (int idx = tid; idx < M * kChunksPerRow; idx += kPassThreads) {
-    const int r = idx / kChunksPerRow, c = idx % kChunksPerRow;
-    cp_async_16(smem_u32(q_s + r * C::kRowBytes + c * 16), qg + (size_t)r * D + c * 8, 16);
-  }
-  const __nv_bfloat16* kg = p.k + (size_t)cu * p.stride_token + (size_t)g * p.stride_head;
-  auto load_tile = [&](int tile_c0, int buf) {
-    uint8_t* dst = k_s + buf * C::kTileBytes;
-    for (int idx = tid; idx < kKeyTile * kChunksPerRow; idx += kPassThreads) {
-      const int r = idx / kChunksPerRow, c = idx % kChunksPerRow;
-      const int key = tile_c0 + r;
-      const bool in = key < t;
-      const __nv_bfloat16* src = kg + (size_t)(in ? key : 0) * p.stride_token + c * 8;
-      cp_async_16(smem_u32(dst + r * C::kRowBytes + c * 16), src, in ? 16 : 0);
-    }
-  };
-  load_tile(key_begin, 0);
-  cp_async_commit();
-
-  if (PASS == 1) {
-    for (int i = tid; i < 4 * M; i += kPassThreads) {
-      state[2 * i] = -INFINITY;
-      state[2 * i + 1] = 0.f;
-    }
-  } else {
-    for (int r = tid; r < M; r += kPassThreads) state[r] = p.mrow[(size_t)unit * M + r];
-  }
-
-  const int n_tiles = (key_end - key_begin + kKeyTile - 1) / kKeyTile;
-  const int MT = M / 16;
-  const uint32_t q_base = smem_u32(q_s);
-  float* my_state = state + (size_t)warp * M * 2;
-
-  for (int ti = 0; ti < n_tiles; ++ti) {
-    const int tile_c0 = key_begin + ti * kKeyTile;
-    if (ti + 1 < n_tiles) {
-      load_tile(tile_c0 + kKeyTile, (ti + 1) & 1);
-      cp_async_commit();
-      cp_async_wait<1>();
-    } else {
-      cp_async_wait<0>();
-    }
-    __syncthreads();
-
-    const uint32_t k_base = smem_u32(k_s + (ti & 1) * C::kTileBytes);
-    uint32_t bf[2][D / 16][4];
+  uint32_t bf[2][D / 16][4];
 #pragma unroll
-    for (int ntp = 0; ntp < 2; ++ntp)
+  for (int ntp = 0; ntp < 2; ++ntp)
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        const int key = 32 * warp + 16 * ntp + (mat >> 1) * 8 + mrow_l;
-        const int col = 16 * ks + (mat & 1) * 8;
-        ldmatrix_x4(bf[ntp][ks], k_base + key * C::kRowBytes + col * 2);
-      }
-
-    float colsum[4][2];
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) colsum[nt][0] = colsum[nt][1] = 0.f;
-    const int c_base = tile_c0 + 32 * warp + 2 * tig;
-
-    for (int mt = 0; mt < MT; ++mt) {
-      float acc[4][4];
-#pragma unroll
-      for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        uint32_t a[4];
-        const int row = 16 * mt + (mat & 1) * 8 + mrow_l;
-        const int col = 16 * ks + (mat >> 1) * 8;
-        ldmatrix_x4(a, q_base + row * C::kRowBytes + col * 2);
-#if XKV_SPLIT_ACC
-        // The tensor core adds into its fp32 accumulator with truncation; summing the per-k-step
-        // partial products with ordinary round-to-nearest adds keeps the logits accurate enough for
-        // the top-k decision.
-        float part[4][4];
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) part[nt][0] = part[nt][1] = part[nt][2] = part[nt][3] = 0.f;
-        mma_bf16_16816(part[0], a, bf[0][ks][0], bf[0][ks][1]);
-        mma_bf16_16816(part[1], a, bf[0][ks][2], bf[0][ks][3]);
-        mma_bf16_16816(part[2], a, bf[1][ks][0], bf[1][ks][1]);
-        mma_bf16_16816(part[3], a, bf[1][ks][2], bf[1][ks][3]);
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[nt][j] += part[nt][j];
-#else
-        mma_bf16_16816(acc[0], a, bf[0][ks][0], bf[0][ks][1]);
-        mma_bf16_16816(acc[1], a, bf[0][ks][2], bf[0][ks][3]);
-        mma_bf16_16816(acc[2], a, bf[1][ks][0], bf[1][ks][1]);
-        mma_bf16_16816(acc[3], a, bf[1][ks][2], bf[1][ks][3]);
-#endif
-      }
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int row = 16 * mt + gid + 8 * half;
-        if (PASS == 1) {
-          const int limit = t - p.window + (row % p.window);   // last visible key of this query row
-          float sv[4][2];
-          float vmax = -INFINITY;
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-              const int c = c_base + 8 * nt + j;
-              sv[nt][j] = (c <= limit) ? acc[nt][2 * half + j] * p.scale_log2 : -INFINITY;
-              vmax = fmaxf(vmax, sv[nt][j]);
-            }
-          vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 1));
-          vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 2));
-          const float m_old = my_state[2 * row], l_old = my_state[2 * row + 1];
-          const float m_new = fmaxf(m_old, vmax);
-          const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-          float sum = 0.f;
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt) sum += fast_exp2(sv[nt][0] - m_ref) + fast_exp2(sv[nt][1] - m_ref);
-          sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-          sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-          const float l_new = l_old * fast_exp2(m_old - m_ref) + sum;
-          __syncwarp();
-          if (tig == 0) {
-            my_state[2 * row] = m_new;
-            my_state[2 * row + 1] = l_new;
-          }
-        } else {
-          const float mr = state[row];
-#pragma unroll
-          for (int nt = 0; nt < 4; ++nt) {
-            colsum[nt][0] += fast_exp2(fmaf(acc[nt][2 * half + 0], p.scale_log2, -mr));
-            colsum[nt][1] += fast_exp2(fmaf(acc[nt][2 * half + 1], p.scale_log2, -mr));
-          }
-        }
-      }
+    for (int ks = 0; ks < D / 16; ++ks) {
+      const int key = 32 * warp + 16 * ntp + (mat >> 1) * 8 + mrow_l;
+      ldmatrix_x4(bf[ntp][ks], k_base + swz(key, 2 * ks + (mat & 1), kRB));
     }
 
-    if (PASS == 2) {
+  float colsum[4][2];
+#pragma unroll
+  for (int nt = 0; nt < 4; ++nt) colsum[nt][0] = colsum[nt][1] = 0.f;
+  const int c_base = tile_c0 + 32 * warp + 2 * tig;
+
+  for (int mt = 0; mt < MT; ++mt) {
+    float acc[4][4];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+      uint32_t a[4];
+      const int row = 16 * mt + (mat & 1) * 8 + mrow_l;
+      ldmatrix_x4(a, q_base + swz(row, 2 * ks + (mat >> 1), kRB));
+      // The tensor core adds into its fp32 accumulator with truncation; summing the per-k-step
+      // partial products with ordinary round-to-nearest adds keeps the logits accurate enough for
+      // the top-k decision.
+      float part[4][4];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt) part[nt][0] = part[nt][1] = part[nt][2] = part[nt][3] = 0.f;
+      mma_bf16_16816(part[0], a, bf[0][ks][0], bf[0][ks][1]);
+      mma_bf16_16816(part[1], a, bf[0][ks][2], bf[0][ks][3]);
+      mma_bf16_16816(part[2], a, bf[1][ks][0], bf[1][ks][1]);
+      mma_bf16_16816(part[3], a, bf[1][ks][2], bf[1][ks][3]);
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          float v = colsum[nt][j];
-          v += __shfl_xor_sync(0xffffffffu, v, 4);
-          v += __shfl_xor_sync(0xffffffffu, v, 8);
-          v += __shfl_xor_sync(0xffffffffu, v, 16);
-          colsum[nt][j] = v;
-        }
-      if (gid == 0) {
-        float* u = p.u + (size_t)g * p.total_tokens + cu;
+        for (int j = 0; j < 4; ++j) acc[nt][j] += part[nt][j];
+    }
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int row = 16 * mt + gid + 8 * half;
+      if (PASS == 1) {
+        const int limit = us.t - p.window + (row % p.window);   // last visible key of this query row
+        float sv[4][2];
+        float vmax = -INFINITY;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const int c = c_base + 8 * nt + j;
-            if (c < key_end) u[c] = colsum[nt][j];
+            sv[nt][j] = (c <= limit) ? acc[nt][2 * half + j] * p.scale_log2 : -INFINITY;
+            vmax = fmaxf(vmax, sv[nt][j]);
           }
+        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 1));
+        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 2));
+        const float m_old = st[2 * row], l_old = st[2 * row + 1];
+        const float m_new = fmaxf(m_old, vmax);
+        const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+        float sum = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) sum += fast_exp2(sv[nt][0] - m_ref) + fast_exp2(sv[nt][1] - m_ref);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        const float l_new = l_old * fast_exp2(m_old - m_ref) + sum;
+        __syncwarp();
+        if (tig == 0) {
+          st[2 * row] = m_new;
+          st[2 * row + 1] = l_new;
+        }
+      } else {
+        const float mr = st[row];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          colsum[nt][0] += fast_exp2(fmaf(acc[nt][2 * half + 0], p.scale_log2, -mr));
+          colsum[nt][1] += fast_exp2(fmaf(acc[nt][2 * half + 1], p.scale_log2, -mr));
+        }
       }
     }
-    __syncthreads();   // the tile buffer is overwritten by the load issued in the next iteration
   }
 
-  if (PASS == 1) {
-    float2* out = p.stats_part + ((size_t)unit * p.n_splits + blockIdx.y) * M;
-    for (int r = tid; r < M; r += kPassThreads) {
-      float m = -INFINITY;
+  if (PASS == 2) {
 #pragma unroll
-      for (int w = 0; w < 4; ++w) m = fmaxf(m, state[((size_t)w * M + r) * 2]);
-      float l = 0.f;
-      if (m > -INFINITY) {
+    for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-        for (int w = 0; w < 4; ++w)
-          l += state[((size_t)w * M + r) * 2 + 1] * fast_exp2(state[((size_t)w * M + r) * 2] - m);
+      for (int j = 0; j < 2; ++j) {
+        float v = colsum[nt][j];
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v += __shfl_xor_sync(0xffffffffu, v, 8);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
+        colsum[nt][j] = v;
       }
-      out[r] = make_float2(m, l);
+    if (gid == 0) {
+      float* u = p.u + (size_t)us.g * p.total_tokens + us.cu;
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int c = c_base + 8 * nt + j;
+          if (c < key_end) u[c] = colsum[nt][j];
+        }
     }
   }
 }
 
-// One CTA per unit: mrow[r] = m_r + log2(l_r) in the log2 domain, +inf for rows without keys.
-__global__ void stats_merge_kernel(const ScoreParams p) {
-  const int unit = blockIdx.x;
-  const int M = p.M;
-  for (int r = threadIdx.x; r < M; r += blockDim.x) {
-    const float2* part = p.stats_part + (size_t)unit * p.n_splits * M + r;
+// Combine the four warps' pass-1 states of a split, publish them, and let the last split of the unit
+// (atomic ticket) merge all splits into mrow[r] = m_r + log2(l_r) (log2 domain; +inf for rows without
+// visible keys) and raise the unit's ready flag.  All threads of the CTA call it.
+__device__ __forceinline__ void publish_stats(const ScoreParams& p, const UnitShape& us, int unit, int split,
+                                              const float* state, int* s_flag) {
+  const int M = p.M, tid = threadIdx.x;
+  float2* out = p.stats_part + ((size_t)unit * p.n_splits + split) * M;
+  for (int r = tid; r < M; r += kPassThreads) {
     float m = -INFINITY;
-    for (int s = 0; s < p.n_splits; ++s) m = fmaxf(m, part[(size_t)s * M].x);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) m = fmaxf(m, state[((size_t)w * M + r) * 2]);
     float l = 0.f;
-    if (m > -INFINITY)
-      for (int s = 0; s < p.n_splits; ++s) {
-        const float2 v = part[(size_t)s * M];
-        l += v.y * exp2f(v.x - m);
+    if (m > -INFINITY) {
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+        l += state[((size_t)w * M + r) * 2 + 1] * fast_exp2(state[((size_t)w * M + r) * 2] - m);
+    }
+    out[r] = make_float2(m, l);
+  }
+  __threadfence();
+  __syncthreads();
+  const int n_splits_u = (us.t + p.split_keys - 1) / p.split_keys;
+  if (tid == 0) *s_flag = (atomicAdd(&p.unit_ticket[unit], 1) == n_splits_u - 1) ? 1 : 0;
+  __syncthreads();
+  if (*s_flag) {
+    __threadfence();
+    for (int r = tid; r < M; r += kPassThreads) {
+      const float2* part = p.stats_part + (size_t)unit * p.n_splits * M + r;
+      float m = -INFINITY;
+      for (int s = 0; s < n_splits_u; ++s) m = fmaxf(m, __ldcg(&part[(size_t)s * M]).x);
+      float l = 0.f;
+      if (m > -INFINITY)
+        for (int s = 0; s < n_splits_u; ++s) {
+          const float2 v = __ldcg(&part[(size_t)s * M]);
+          l += v.y * exp2f(v.x - m);
+        }
+      p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) atomicExch(&p.unit_ready[unit], 1);
+  }
+}
+
+// Bounded wait (two seconds) for a unit's row normalisers.  Thread 0 polls; returns false on expiry.
+__device__ __forceinline__ bool wait_unit_ready(const ScoreParams& p, int unit, int* s_flag) {
+  if (threadIdx.x == 0) {
+    int ok = 1;
+    if (ld_acquire(&p.unit_ready[unit]) == 0) {
+      const uint64_t t0 = timer_ns();
+      while (ld_acquire(&p.unit_ready[unit]) == 0) {
+        __nanosleep(100);
+        if (timer_ns() - t0 > 2000000000ull) {
+          ok = 0;
+          record_status(p.hdr, XKV_ERR_TIMEOUT);
+          break;
+        }
       }
-    p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
+    }
+    *s_flag = ok;
+  }
+  __syncthreads();
+  return *s_flag != 0;
+}
+
+// Resident variant: a work item is (unit, split); the split's keys stay in shared memory between the two
+// passes, so K is read from HBM once.  A CTA runs pass 1 on its split, publishes its row statistics, waits
+// (bounded) until all splits of the unit have done so, and runs pass 2 from shared memory.  Items are
+// handed out in order from a global counter, and a CTA asks for its next item only when it is free: an
+// item that has been handed out is being worked on.  So a waiting CTA depends only on items that are
+// running or will be picked up by the next CTA that finishes, and the host uses this variant only when a
+// unit has far fewer splits than there are resident CTAs.
+template <int D>
+__global__ void __launch_bounds__(kPassThreads) score_resident_kernel(const ScoreParams p) {
+  using C = PassCfg<D>;
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int M = p.M;
+  uint8_t* q_s = smem;
+  uint8_t* k_s = smem + (size_t)M * C::kRowBytes;
+  float* state = reinterpret_cast<float*>(k_s + (size_t)p.slice_tiles * C::kTileBytes);
+  int* s_ctl = reinterpret_cast<int*>(state + (size_t)4 * M * 2);
+  const int tid = threadIdx.x, warp = tid >> 5;
+
+  while (true) {
+    __syncthreads();
+    if (tid == 0) s_ctl[0] = atomicAdd(&p.hdr->work_counter, 1);
+    __syncthreads();
+    const int idx = s_ctl[0];
+    if (idx >= p.n_work) break;
+    const int unit = idx / p.n_splits, split = idx % p.n_splits;
+    const UnitShape us = unit_shape(p, unit);
+    const int key_begin = split * p.split_keys;
+    const int key_end1 = min(key_begin + p.split_keys, us.t);
+    if (key_begin >= key_end1) continue;
+    const int n_tiles = (key_end1 - key_begin + kKeyTile - 1) / kKeyTile;
+
+    load_q<D>(p, us, q_s);
+    for (int ti = 0; ti < n_tiles; ++ti)
+      load_k_tile<D>(p, us, k_s + (size_t)ti * C::kTileBytes, key_begin + ti * kKeyTile);
+    cp_async_commit();
+    for (int i = tid; i < 4 * M; i += kPassThreads) {
+      state[2 * i] = -INFINITY;
+      state[2 * i + 1] = 0.f;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    const uint32_t q_base = smem_u32(q_s);
+    for (int ti = 0; ti < n_tiles; ++ti)
+      compute_tile<D, 1>(p, us, q_base, smem_u32(k_s + (size_t)ti * C::kTileBytes), state + (size_t)warp * M * 2,
+                         key_begin + ti * kKeyTile, 0);
+    __syncthreads();
+    publish_stats(p, us, unit, split, state, &s_ctl[1]);
+
+    const int key_end2 = min(key_end1, us.P);
+    if (key_begin >= key_end2) continue;           // a split that holds window keys only
+    if (!wait_unit_ready(p, unit, &s_ctl[2])) continue;
+    for (int r = tid; r < M; r += kPassThreads) state[r] = __ldcg(&p.mrow[(size_t)unit * M + r]);
+    __syncthreads();
+    const int n_tiles2 = (key_end2 - key_begin + kKeyTile - 1) / kKeyTile;
+    for (int ti = 0; ti < n_tiles2; ++ti)
+      compute_tile<D, 2>(p, us, q_base, smem_u32(k_s + (size_t)ti * C::kTileBytes), state, key_begin + ti * kKeyTile,
+                         key_end2);
+  }
+}
+
+// Streaming variant for sequences too long for the resident one: all pass-1 items, then all pass-2 items,
+// from one global counter; key tiles go through a cp.async ring.  A pass-2 item waits (bounded) for its
+// unit's ready flag, which is long set except right at the boundary between the two phases.  Pass-1 items
+// never wait, and every pass-1 item has a lower index than every pass-2 item, so fetching the next index
+// early cannot hold back an item somebody waits for.
+template <int D>
+__global__ void __launch_bounds__(kPassThreads) score_stream_kernel(const ScoreParams p) {
+  using C = PassCfg<D>;
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int M = p.M;
+  uint8_t* q_s = smem;
+  uint8_t* k_s = smem + (size_t)M * C::kRowBytes;
+  float* state = reinterpret_cast<float*>(k_s + (size_t)kPassStages * C::kTileBytes);
+  int* s_ctl = reinterpret_cast<int*>(state + (size_t)4 * M * 2);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int half_work = p.n_work / 2;
+
+  int next = 0;
+  if (tid == 0) next = atomicAdd(&p.hdr->work_counter, 1);
+  while (true) {
+    __syncthreads();
+    if (tid == 0) {
+      s_ctl[0] = next;
+      next = atomicAdd(&p.hdr->work_counter, 1);      // fetched now, used after this item
+    }
+    __syncthreads();
+    const int idx = s_ctl[0];
+    if (idx >= p.n_work) break;
+    const int pass = idx < half_work ? 1 : 2;
+    const int rem = idx < half_work ? idx : idx - half_work;
+    const int unit = rem / p.n_splits, split = rem % p.n_splits;
+    const UnitShape us = unit_shape(p, unit);
+    const int key_begin = split * p.split_keys;
+    const int key_end = min(key_begin + p.split_keys, pass == 1 ? us.t : us.P);
+    if (key_begin >= key_end) continue;
+    if (pass == 2) {
+      if (!wait_unit_ready(p, unit, &s_ctl[2])) continue;
+      for (int r = tid; r < M; r += kPassThreads) state[r] = __ldcg(&p.mrow[(size_t)unit * M + r]);
+    } else {
+      for (int i = tid; i < 4 * M; i += kPassThreads) {
+        state[2 * i] = -INFINITY;
+        state[2 * i + 1] = 0.f;
+      }
+    }
+
+    const int n_tiles = (key_end - key_begin + kKeyTile - 1) / kKeyTile;
+    load_q<D>(p, us, q_s);
+#pragma unroll
+    for (int s = 0; s < kPassStages - 1; ++s) {
+      if (s < n_tiles) load_k_tile<D>(p, us, k_s + (size_t)s * C::kTileBytes, key_begin + s * kKeyTile);
+      cp_async_commit();
+    }
+    const uint32_t q_base = smem_u32(q_s);
+    for (int ti = 0; ti < n_tiles; ++ti) {
+      cp_async_wait<kPassStages - 2>();
+      __syncthreads();          // tile ti has landed for everyone; the buffer of tile ti-1 is free
+      if (ti + kPassStages - 1 < n_tiles)
+        load_k_tile<D>(p, us, k_s + (size_t)((ti + kPassStages - 1) % kPassStages) * C::kTileBytes,
+                       key_begin + (ti + kPassStages - 1) * kKeyTile);
+      cp_async_commit();
+      const uint32_t k_base = smem_u32(k_s + (size_t)(ti % kPassStages) * C::kTileBytes);
+      if (pass == 1)
+        compute_tile<D, 1>(p, us, q_base, k_base, state + (size_t)warp * M * 2, key_begin + ti * kKeyTile, 0);
+      else
+        compute_tile<D, 2>(p, us, q_base, k_base, state, key_begin + ti * kKeyTile, key_end);
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    if (pass == 1) publish_stats(p, us, unit, split, state, &s_ctl[1]);
   }
 }
 
@@ -486,52 +636,74 @@ __global__ void __launch_bounds__(1024) mass_kernel(const ScoreParams p) {
 }
 
 struct ScoreLayout {
-  size_t u, tmp_sorted, stats_part, mrow, part_sum, total;
-  int split_keys, n_splits, n_chunks;
+  size_t flags, u, tmp_sorted, stats_part, mrow, part_sum, total;
+  int split_keys, n_splits, n_chunks, slice_tiles, ctas_per_sm;
+  bool resident;
 };
 
 void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) {
   const int units = d->batch * d->n_kv_heads;
   const int M = (d->n_q_heads / d->n_kv_heads) * d->window;
-  int split = 1024;
-  while (split > kKeyTile && (int64_t)units * ((max_seqlen + split - 1) / split) < 2 * 148) split >>= 1;
-  L->split_keys = split;
-  L->n_splits = (max_seqlen + split - 1) / split;
+  const int sms = sm_count();
+  // Resident variant: key tiles per split chosen so that two CTAs fit on an SM (one for G*W = 256).
+  int tiles = M <= 64 ? 3 : (M <= 128 ? 2 : 4);
+  while (tiles > 1 && (int64_t)units * ((max_seqlen + tiles * kKeyTile - 1) / (tiles * kKeyTile)) < 2 * sms) --tiles;
+  const size_t tile_bytes = (size_t)kKeyTile * d->head_dim * 2;
+  const size_t fixed = (size_t)M * d->head_dim * 2 + (size_t)4 * M * 8 + 64;
+  auto ctas_for = [&](size_t smem) {
+    int c = (int)((227u * 1024u) / (smem + 1024));
+    return c < 1 ? 1 : (c > 3 ? 3 : c);
+  };
+  const int res_ctas = ctas_for(fixed + tiles * tile_bytes);
+  const int res_splits = (max_seqlen + tiles * kKeyTile - 1) / (tiles * kKeyTile);
+  // every split of a unit must be in flight at once with room to spare (CTAs of a unit wait for each other)
+  L->resident = res_splits * 4 <= sms * (res_ctas < 2 ? res_ctas : 2);
+  if (L->resident) {
+    L->slice_tiles = tiles;
+    L->split_keys = tiles * kKeyTile;
+    L->ctas_per_sm = res_ctas;
+  } else {
+    int split = 1024;
+    while (split > kKeyTile && (int64_t)units * ((max_seqlen + split - 1) / split) < 2 * sms) split >>= 1;
+    L->slice_tiles = kPassStages;
+    L->split_keys = split;
+    L->ctas_per_sm = ctas_for(fixed + kPassStages * tile_bytes);
+  }
+  L->n_splits = (max_seqlen + L->split_keys - 1) / L->split_keys;
   L->n_chunks = (max_seqlen + kSortChunk - 1) / kSortChunk;
   size_t off = kHeaderBytes;
+  L->flags = off;      off = align_up(off + (size_t)units * 8, 256);
   L->u = off;          off = align_up(off + (size_t)d->n_kv_heads * T * 4, 256);
   L->tmp_sorted = off; off = align_up(off + (size_t)d->n_kv_heads * T * 4, 256);
-  L->stats_part = off; off = align_up(off + (size_t)units * L->n_splits * M * 8, 256);
+  // sized for the smallest split either variant may choose, so the size does not depend on the device
+  L->stats_part = off; off = align_up(off + (size_t)units * ((max_seqlen + kKeyTile - 1) / kKeyTile) * M * 8, 256);
   L->mrow = off;       off = align_up(off + (size_t)units * M * 4, 256);
   L->part_sum = off;   off = align_up(off + (size_t)units * L->n_chunks * 4, 256);
   L->total = off;
 }
 
 template <int D>
-xkv_status launch_passes(const ScoreParams& p, int units, cudaStream_t st) {
-  const size_t smem = PassCfg<D>::smem_bytes(p.M);
+xkv_status launch_passes(const ScoreParams& p, const ScoreLayout& L, cudaStream_t st) {
+  const size_t smem = PassCfg<D>::smem_bytes(p.M, L.slice_tiles);
   static bool done[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(score_pass_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)PassCfg<D>::smem_bytes(256)) != cudaSuccess ||
-        cudaFuncSetAttribute(score_pass_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)PassCfg<D>::smem_bytes(256)) != cudaSuccess)
+    const int max_smem = 227 * 1024;
+    if (cudaFuncSetAttribute(score_stream_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(score_resident_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) !=
+            cudaSuccess)
       return XKV_ERR_CUDA;
     done[dev] = true;
   }
-  dim3 grid(units, p.n_splits);
-  score_pass_kernel<D, 1><<<grid, kPassThreads, smem, st>>>(p);
-  count_launch();
-  xkv_status s = check_launch();
-  if (s != XKV_OK) return s;
-  stats_merge_kernel<<<units, 256, 0, st>>>(p);
-  count_launch();
-  s = check_launch();
-  if (s != XKV_OK) return s;
-  score_pass_kernel<D, 2><<<grid, kPassThreads, smem, st>>>(p);
+  int grid = sm_count() * L.ctas_per_sm;
+  if (grid > p.n_work) grid = p.n_work;
+  if (L.resident)
+    score_resident_kernel<D><<<grid, kPassThreads, smem, st>>>(p);
+  else
+    score_stream_kernel<D><<<grid, kPassThreads, smem, st>>>(p);
   count_launch();
   return check_launch();
 }
@@ -581,11 +753,16 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
   p.n_splits = L.n_splits;
   p.n_chunks = L.n_chunks;
   p.curve_len = curve_len;
+  p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  p.unit_ticket = reinterpret_cast<int32_t*>(ws + L.flags);
+  p.unit_ready = p.unit_ticket + units;
+  p.slice_tiles = L.slice_tiles;
+  p.n_work = (L.resident ? 1 : 2) * units * L.n_splits;
   const float scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
 
-  if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;
-  xkv_status s = d->head_dim == 128 ? launch_passes<128>(p, units, st) : launch_passes<64>(p, units, st);
+  if (cudaMemsetAsync(ws, 0, L.u, st) != cudaSuccess) return XKV_ERR_CUDA;   // header, tickets, ready flags
+  xkv_status s = d->head_dim == 128 ? launch_passes<128>(p, L, st) : launch_passes<64>(p, L, st);
   if (s != XKV_OK) return s;
 
   // chunk sort, then log2(n_chunks) merge passes ping-ponging so that the last one lands in `sorted`
