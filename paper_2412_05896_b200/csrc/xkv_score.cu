@@ -12,7 +12,8 @@
 //                           passes (K is read from HBM once); the streaming variant, for sequences
 //                           too long for that, runs all pass-1 items and then all pass-2 items.
 //   pool_sort_kernel        1-D pooling (max or zero-padded average) of u into the scores w, and a
-//                           descending bitonic sort of each 4096-score chunk in shared memory
+//                           descending bitonic sort of each 4096-score chunk (registers, warp
+//                           shuffles, shared memory only for the longest exchanges)
 //   merge_kernel            merge-path passes that combine the sorted chunks of a segment
 //   gains_kernel / mass_kernel  the per-sequence retained-importance curve of the layer
 //
@@ -32,7 +33,8 @@ namespace {
 constexpr int kPassThreads = 128;     // 4 warps
 constexpr int kKeyTile = 128;         // keys per tile, 32 per warp
 constexpr int kSortChunk = 4096;      // scores sorted per CTA
-constexpr int kSortThreads = 1024;
+constexpr int kSortThreads = 512;
+constexpr int kSortItems = kSortChunk / kSortThreads;   // 8 scores per thread, kept in registers
 constexpr int kMergeTile = 2048;
 constexpr int kMergeThreads = 256;
 constexpr int kMergeItems = kMergeTile / kMergeThreads;
@@ -445,7 +447,7 @@ __global__ void __launch_bounds__(kPassThreads) score_stream_kernel(const ScoreP
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSortThreads) pool_sort_kernel(const ScoreParams p, float* sort_out) {
   __shared__ float s_u[kSortChunk + 64];
-  __shared__ float s_key[kSortChunk];
+  __shared__ __align__(16) float s_key[kSortChunk];
   __shared__ float s_red[32];
   const int unit = blockIdx.x, chunk = blockIdx.y;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
@@ -494,29 +496,66 @@ __global__ void __launch_bounds__(kSortThreads) pool_sort_kernel(const ScorePara
   if ((tid & 31) == 0) s_red[tid >> 5] = local;
   __syncthreads();
   if (tid < 32) {
-    float v = s_red[tid];
+    float v = tid < kSortThreads / 32 ? s_red[tid] : 0.f;
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     if (tid == 0) p.part_sum[(size_t)unit * p.n_chunks + chunk] = v;
   }
   if (sort_out == nullptr) return;
   if (c0 >= P) return;
 
-  // bitonic sort, descending; absent entries (-1) end up last
+  // Bitonic sort, descending; absent entries (-1) end up last.  Thread t holds elements 8t..8t+7 in
+  // registers: exchanges at distance < 8 stay in the thread, distances 8..128 are warp shuffles, and
+  // only the ten steps at distance >= 256 go through shared memory.
+  static_assert(kSortItems == 8, "the exchange pattern below assumes 8 scores per thread");
+  __syncthreads();
+  float e[kSortItems];
+  {
+    const float4 lo = *reinterpret_cast<const float4*>(&s_key[8 * tid]);
+    const float4 hi = *reinterpret_cast<const float4*>(&s_key[8 * tid + 4]);
+    e[0] = lo.x; e[1] = lo.y; e[2] = lo.z; e[3] = lo.w;
+    e[4] = hi.x; e[5] = hi.y; e[6] = hi.z; e[7] = hi.w;
+  }
+#pragma unroll
   for (int k = 2; k <= kSortChunk; k <<= 1) {
+#pragma unroll
     for (int j = k >> 1; j > 0; j >>= 1) {
-      __syncthreads();
-      for (int x = tid; x < kSortChunk / 2; x += kSortThreads) {
-        const int i = ((x & ~(j - 1)) << 1) | (x & (j - 1));   // index with bit j clear
-        const int l = i | j;
-        const float a = s_key[i], c = s_key[l];
-        const bool desc = (i & k) == 0;
-        if (desc ? (a < c) : (a > c)) {
-          s_key[i] = c;
-          s_key[l] = a;
+      if (j >= 8) {
+        const int m = j >> 3;                                   // partner thread = tid ^ m
+        const bool lower = (tid & m) == 0;
+        const bool desc = (tid & (k >> 3)) == 0;
+        const bool want_max = lower == desc;
+        float o[kSortItems];
+        if (m >= 32) {
+          __syncthreads();
+          *reinterpret_cast<float4*>(&s_key[8 * tid]) = make_float4(e[0], e[1], e[2], e[3]);
+          *reinterpret_cast<float4*>(&s_key[8 * tid + 4]) = make_float4(e[4], e[5], e[6], e[7]);
+          __syncthreads();
+          const float4 lo = *reinterpret_cast<const float4*>(&s_key[8 * (tid ^ m)]);
+          const float4 hi = *reinterpret_cast<const float4*>(&s_key[8 * (tid ^ m) + 4]);
+          o[0] = lo.x; o[1] = lo.y; o[2] = lo.z; o[3] = lo.w;
+          o[4] = hi.x; o[5] = hi.y; o[6] = hi.z; o[7] = hi.w;
+        } else {
+#pragma unroll
+          for (int r = 0; r < kSortItems; ++r) o[r] = __shfl_xor_sync(0xffffffffu, e[r], m);
+        }
+#pragma unroll
+        for (int r = 0; r < kSortItems; ++r) e[r] = want_max ? fmaxf(e[r], o[r]) : fminf(e[r], o[r]);
+      } else {
+#pragma unroll
+        for (int r = 0; r < kSortItems; ++r) {
+          if ((r & j) == 0) {
+            const bool desc = k < 8 ? ((r & k) == 0) : ((tid & (k >> 3)) == 0);
+            const float hi = fmaxf(e[r], e[r | j]), lo = fminf(e[r], e[r | j]);
+            e[r] = desc ? hi : lo;
+            e[r | j] = desc ? lo : hi;
+          }
         }
       }
     }
   }
+  __syncthreads();
+  *reinterpret_cast<float4*>(&s_key[8 * tid]) = make_float4(e[0], e[1], e[2], e[3]);
+  *reinterpret_cast<float4*>(&s_key[8 * tid + 4]) = make_float4(e[4], e[5], e[6], e[7]);
   __syncthreads();
   const int n_valid = min(kSortChunk, P - c0);
   for (int i = tid; i < n_valid; i += kSortThreads) sort_out[seg + c0 + i] = s_key[i];
