@@ -1,0 +1,37 @@
+// Parameters shared by the scoring kernels (xkv_score.cu, xkv_score_tc.cu).
+#pragma once
+
+#include "common.cuh"
+
+namespace xkv {
+
+struct ScoreParams {
+  const __nv_bfloat16* q_win;
+  const __nv_bfloat16* k;
+  const int32_t* cu_seqlens;
+  float* scores;
+  float* sorted;
+  float* gains;
+  float* mass;
+  float* u;            // [Hkv][T] un-pooled column sums
+  float* tmp_sorted;   // [Hkv][T] ping-pong buffer of the merge passes
+  float2* stats_part;  // [units][n_splits][M]
+  float* mrow;         // [units][M]
+  float* part_sum;     // [units][n_chunks]
+  WorkspaceHeader* hdr;
+  int32_t* unit_ticket;  // [units] pass-1 items of the unit that have finished
+  int32_t* unit_ready;   // [units] 1 once mrow of the unit is final
+  int32_t slice_tiles, n_work;
+  int64_t total_tokens, stride_token, stride_head;
+  int32_t batch, n_q_heads, n_kv_heads, group, window, M, pool_kernel, pool_mode;
+  int32_t split_keys, n_splits, n_chunks, curve_len;
+  float scale_log2;
+};
+
+// tcgen05 variant of the two logit passes (xkv_score_tc.cu).  Returns XKV_ERR_UNSUPPORTED when the shape
+// is outside what it covers; the caller then uses the mma.sync kernels.
+xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st);
+// Key split the tcgen05 variant uses (0 if it does not cover the shape).
+int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen);
+
+}  // namespace xkv

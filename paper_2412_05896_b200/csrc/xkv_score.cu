@@ -26,6 +26,7 @@
 
 #include "common.cuh"
 #include "ops.h"
+#include "score_params.h"
 
 namespace xkv {
 namespace {
@@ -39,28 +40,6 @@ constexpr int kMergeTile = 2048;
 constexpr int kMergeThreads = 256;
 constexpr int kMergeItems = kMergeTile / kMergeThreads;
 
-struct ScoreParams {
-  const __nv_bfloat16* q_win;
-  const __nv_bfloat16* k;
-  const int32_t* cu_seqlens;
-  float* scores;
-  float* sorted;
-  float* gains;
-  float* mass;
-  float* u;            // [Hkv][T] un-pooled column sums
-  float* tmp_sorted;   // [Hkv][T] ping-pong buffer of the merge passes
-  float2* stats_part;  // [units][n_splits][M]
-  float* mrow;         // [units][M]
-  float* part_sum;     // [units][n_chunks]
-  WorkspaceHeader* hdr;
-  int32_t* unit_ticket;  // [units] pass-1 items of the unit that have finished
-  int32_t* unit_ready;   // [units] 1 once mrow of the unit is final
-  int32_t slice_tiles, n_work;
-  int64_t total_tokens, stride_token, stride_head;
-  int32_t batch, n_q_heads, n_kv_heads, group, window, M, pool_kernel, pool_mode;
-  int32_t split_keys, n_splits, n_chunks, curve_len;
-  float scale_log2;
-};
 
 constexpr int kPassStages = 3;        // cp.async ring of key tiles (streaming variant)
 
@@ -677,7 +656,7 @@ __global__ void __launch_bounds__(1024) mass_kernel(const ScoreParams p) {
 struct ScoreLayout {
   size_t flags, u, tmp_sorted, stats_part, mrow, part_sum, total;
   int split_keys, n_splits, n_chunks, slice_tiles, ctas_per_sm;
-  bool resident;
+  bool resident, use_tc;
 };
 
 void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) {
@@ -707,6 +686,14 @@ void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) 
     L->slice_tiles = kPassStages;
     L->split_keys = split;
     L->ctas_per_sm = ctas_for(fixed + kPassStages * tile_bytes);
+  }
+  // the tcgen05 kernel takes the passes over when it covers the shape (it is a resident variant too)
+  const int tc_split = score_tc_split_keys(M, d->head_dim, units, max_seqlen);
+  L->use_tc = tc_split > 0;
+  if (L->use_tc) {
+    L->resident = true;
+    L->split_keys = tc_split;
+    L->slice_tiles = tc_split / kKeyTile;
   }
   L->n_splits = (max_seqlen + L->split_keys - 1) / L->split_keys;
   L->n_chunks = (max_seqlen + kSortChunk - 1) / kSortChunk;
@@ -801,7 +788,12 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
   p.scale_log2 = scale * 1.4426950408889634f;
 
   if (cudaMemsetAsync(ws, 0, L.u, st) != cudaSuccess) return XKV_ERR_CUDA;   // header, tickets, ready flags
-  xkv_status s = d->head_dim == 128 ? launch_passes<128>(p, L, st) : launch_passes<64>(p, L, st);
+  xkv_status s;
+  if (L.use_tc) {
+    s = score_tc_passes(p, d->head_dim, max_seqlen, st);
+  } else {
+    s = d->head_dim == 128 ? launch_passes<128>(p, L, st) : launch_passes<64>(p, L, st);
+  }
   if (s != XKV_OK) return s;
 
   // chunk sort, then log2(n_chunks) merge passes ping-ponging so that the last one lands in `sorted`
