@@ -691,7 +691,7 @@ void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) 
   const int tc_split = score_tc_split_keys(M, d->head_dim, units, max_seqlen);
   L->use_tc = tc_split > 0;
   if (L->use_tc) {
-    L->resident = true;
+    L->resident = true;            // one work item per (unit, split); the kernel runs as two launches
     L->split_keys = tc_split;
     L->slice_tiles = tc_split / kKeyTile;
   }

@@ -1,16 +1,19 @@
 // Window-logit passes of xkv_score on the 5th-generation tensor cores (tcgen05) with TMEM accumulators.
 //
-// A work item is (unit = (sequence, KV head), split of the key axis).  Its keys are brought into shared
-// memory once by TMA (128-byte swizzled, K-major tiles of 128 keys) and stay there for both passes:
+// A work item is (unit = (sequence, KV head), split of the key axis).  Persistent CTAs take items from a
+// global counter and stream the item's keys through a two-stage shared-memory ring filled by TMA
+// (128-byte swizzled, K-major tiles of 128 keys); one thread issues the MMAs of a tile into one of two TMEM
+// accumulator buffers while all threads reduce the previous tile out of the other; completion comes back
+// through tcgen05.commit on an mbarrier.  Two launches:
 //   pass 1  D[query rows x keys] = Q K^T with the G*W query rows on the MMA's M axis: a thread owns one
 //           TMEM lane = one query row, so the running (max, sum of exponentials) of the softmax is two
 //           registers and needs no cross-lane traffic.  With fewer than 128 query rows the rows are
 //           replicated over the four lane quarters and every warp takes a quarter of the key columns.
+//           The last split of a unit to finish (atomic ticket) merges the unit's statistics.
 //   pass 2  D[keys x query rows] = K Q^T with the keys on M: a thread owns one key and sums
 //           exp2(s*c - normaliser[row]) over the query rows straight out of TMEM -> column score u[key].
-// Between the passes the splits of a unit exchange their row statistics through global memory: the last
-// split to publish (atomic ticket) merges them and raises the unit's ready flag; the others wait for it
-// (bounded).  One thread issues the MMAs; completion comes back through tcgen05.commit on an mbarrier.
+//           Items are walked in reverse so that the keys pass 1 streamed last are re-read from L2.
+// No CTA ever waits for another one; every mbarrier wait is bounded.
 #include <cuda.h>
 
 #include <cmath>
@@ -24,8 +27,6 @@ namespace {
 
 constexpr int kTcThreads = 128;
 constexpr int kTcKeyTile = 128;                 // keys per MMA tile
-constexpr int kTcMaxTiles = 4;                  // key tiles a split may hold
-constexpr uint32_t kTmemCols = 256;             // TMEM columns a CTA allocates (two CTAs fit on an SM)
 
 // ---------------------------------------------------------------------------------------------
 // tcgen05 / TMEM wrappers
@@ -131,6 +132,8 @@ __device__ __forceinline__ int tc_ld_acquire(const int* ptr) {
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
+constexpr int kTcStages = 2;       // shared-memory ring of key tiles, and TMEM accumulator buffers
+
 template <int D, int M>
 struct TcCfg {
   static constexpr int kHalves = D / 64;                         // 128-byte swizzled K segments per row
@@ -141,12 +144,12 @@ struct TcCfg {
   static constexpr int kQBytes = kHalves * kQHalfBytes;
   static constexpr int kKHalfBytes = kTcKeyTile * 128;
   static constexpr int kKTileBytes = kHalves * kKHalfBytes;
-  static constexpr int kBufs = M == 256 ? 1 : 2;                 // TMEM accumulator buffers of 128 (256) columns
+  static constexpr uint32_t kBufCols = M == 256 ? 256 : 128;     // TMEM columns of one accumulator buffer
+  static constexpr uint32_t kTmemCols = kTcStages * kBufCols;    // 256 (two CTAs per SM) or 512
   static constexpr int kColsPerThread = M < 128 ? M : 128;       // pass-1 key columns a thread reduces per tile
   static constexpr uint32_t kQTxBytes = (uint32_t)(kRep * kHalves * (M < 128 ? M : kQRows) * 128);
-  static size_t smem_bytes(int tiles) {
-    return 1024 + (size_t)kQBytes + (size_t)tiles * kKTileBytes + 256 * 4 /*mrow*/ + 256 * 8 /*stats*/ + 128;
-  }
+  static constexpr size_t kSmemBytes =
+      1024 + (size_t)kQBytes + (size_t)kTcStages * kKTileBytes + 256 * 4 /*mrow*/ + 256 * 8 /*stats*/ + 128;
 };
 
 __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
@@ -167,7 +170,10 @@ __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int
   m = m_new;
 }
 
-template <int D, int M>
+// PASS 1: row statistics of every (unit, split) item, merged per unit by the last split to finish.
+// PASS 2: column sums u, launched after pass 1 has completed; items are taken in reverse order so that the
+//         keys pass 1 streamed last are still in L2.
+template <int D, int M, int PASS>
 __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                                                              const __grid_constant__ CUtensorMap tmap_k,
                                                              const ScoreParams p) {
@@ -176,24 +182,27 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
   uint8_t* k_s = q_s + C::kQBytes;
-  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)p.slice_tiles * C::kKTileBytes);   // [256]
-  float2* s_stat = reinterpret_cast<float2*>(s_mrow + 256);                                  // [256]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_stat + 256);                            // [kTcMaxTiles]
-  uint64_t* mma_bar = full_bar + kTcMaxTiles;                                                // [2]
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(mma_bar + 2);
-  int* s_ctl = reinterpret_cast<int*>(s_tmem + 1);                                           // [0] item [1] flag [2] ok
+  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)kTcStages * C::kKTileBytes);   // [256]
+  float2* s_stat = reinterpret_cast<float2*>(s_mrow + 256);                              // [256]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_stat + 256);                        // [kTcStages]
+  uint64_t* mma_bar = full_bar + kTcStages;                                              // [kTcStages]
+  uint64_t* q_bar = mma_bar + kTcStages;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(q_bar + 1);
+  int* s_ctl = reinterpret_cast<int*>(s_tmem + 1);                                       // [0] item [1] flag
 
   const int tid = threadIdx.x, warp = tid >> 5;
   if (tid == 0) {
-    for (int i = 0; i < kTcMaxTiles; ++i) mbar_init(&full_bar[i], 1);
-    mbar_init(&mma_bar[0], 1);
-    mbar_init(&mma_bar[1], 1);
+    for (int i = 0; i < kTcStages; ++i) {
+      mbar_init(&full_bar[i], 1);
+      mbar_init(&mma_bar[i], 1);
+    }
+    mbar_init(q_bar, 1);
     fence_mbar_init();
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_k);
   }
   if (warp == 0) {
-    tmem_alloc(s_tmem, kTmemCols);
+    tmem_alloc(s_tmem, C::kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -202,57 +211,54 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
   const uint32_t tmem_base = *s_tmem;
   const uint32_t tmem_lane = tmem_base + ((uint32_t)(32 * warp) << 16);   // this warp's quarter of the lanes
 
-  uint32_t item_parity = 0;          // phase of the TMA barriers (every item flips all of them)
-  uint32_t mma_cnt[2] = {0, 0};      // uses of each accumulator buffer so far
+  uint32_t gt = 0;            // key tiles this CTA has processed: stage, accumulator buffer and phases follow it
+  uint32_t q_parity = 0;      // phase of the query barrier (one use per item)
   bool aborted = false;
   const uint32_t q_base = smem_u32(q_s), k_base = smem_u32(k_s);
+  int* counter = PASS == 1 ? &p.hdr->work_counter : &p.hdr->prep_ticket;
 
+  int next = 0;
+  if (tid == 0) next = atomicAdd(counter, 1);
   while (!aborted) {
     __syncthreads();
-    if (tid == 0) s_ctl[0] = atomicAdd(&p.hdr->work_counter, 1);
+    if (tid == 0) {
+      s_ctl[0] = next;
+      next = atomicAdd(counter, 1);      // fetched now, used after this item (no item ever waits for another)
+    }
     __syncthreads();
-    const int idx = s_ctl[0];
+    int idx = s_ctl[0];
     if (idx >= p.n_work) break;
+    if (PASS == 2) idx = p.n_work - 1 - idx;
     const int unit = idx / p.n_splits, split = idx % p.n_splits;
     const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
     const int cu = p.cu_seqlens[b];
     const int t = p.cu_seqlens[b + 1] - cu;
     const int P = max(t - p.window, 0);
     const int key_begin = split * p.split_keys;
-    const int key_end1 = min(key_begin + p.split_keys, t);
-    if (key_begin >= key_end1) continue;
-    const int n_tiles = (key_end1 - key_begin + kTcKeyTile - 1) / kTcKeyTile;
+    const int key_end = min(key_begin + p.split_keys, PASS == 1 ? t : P);
+    if (key_begin >= key_end) continue;
+    const int n_tiles = (key_end - key_begin + kTcKeyTile - 1) / kTcKeyTile;
 
-    // ---- bring the query rows (replicated) and the split's key tiles into shared memory
-    if (tid == 0) {
-      for (int ti = 0; ti < kTcMaxTiles; ++ti) {
-        const uint32_t bytes = (ti < n_tiles ? (uint32_t)C::kKTileBytes : 0u) + (ti == 0 ? C::kQTxBytes : 0u);
-        mbar_arrive_expect_tx(&full_bar[ti], bytes);
-      }
-      const int qrow0 = (b * p.n_q_heads + g * p.group) * p.window;
+    auto load_tile = [&](int ti) {           // thread 0: arm the stage's barrier and start the copy
+      const uint32_t s = (gt + ti) % kTcStages;
+      mbar_arrive_expect_tx(&full_bar[s], (uint32_t)C::kKTileBytes);
 #pragma unroll
-      for (int rep = 0; rep < C::kRep; ++rep)
-#pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_2d(q_s + hf * C::kQHalfBytes + rep * M * 128, &tmap_q, hf * 64, qrow0, &full_bar[0]);
-      for (int ti = 0; ti < n_tiles; ++ti)
-#pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_3d(k_s + (size_t)ti * C::kKTileBytes + hf * C::kKHalfBytes, &tmap_k, hf * 64, g,
-                      cu + key_begin + ti * kTcKeyTile, &full_bar[ti]);
-    }
-
-    // One thread issues the MMAs of a tile once its keys have landed.
-    auto issue = [&](int pass, int ti, int buf) -> bool {
-      if (!tc_mbar_wait(&full_bar[ti], item_parity)) return false;
+      for (int hf = 0; hf < C::kHalves; ++hf)
+        tma_load_3d(k_s + (size_t)s * C::kKTileBytes + hf * C::kKHalfBytes, &tmap_k, hf * 64, g,
+                    cu + key_begin + ti * kTcKeyTile, &full_bar[s]);
+    };
+    // thread 0: once tile ti has landed, issue its MMAs into accumulator buffer (gt+ti) % 2
+    auto issue = [&](int ti) -> bool {
+      const uint32_t gi = gt + ti, s = gi % kTcStages;
+      if (!tc_mbar_wait(&full_bar[s], (gi / kTcStages) & 1u)) return false;
       tc_fence_after_sync();
-      const uint32_t kt = k_base + (uint32_t)ti * C::kKTileBytes;
-      const uint32_t d_tmem = tmem_base + (uint32_t)buf * 128u;
+      const uint32_t kt = k_base + s * C::kKTileBytes;
+      const uint32_t d_tmem = tmem_base + s * C::kBufCols;
 #pragma unroll
       for (int k = 0; k < C::kSteps; ++k) {
-        const uint32_t ko = (uint32_t)(k / 4) * 0u + (uint32_t)(k % 4) * 32u;
+        const uint32_t ko = (uint32_t)(k % 4) * 32u;          // 16 bf16 along K inside the swizzled 128-byte row
         const uint64_t kd = umma_desc_k128(kt + (k / 4) * C::kKHalfBytes + ko);
-        if (pass == 1) {
+        if (PASS == 1) {
 #pragma unroll
           for (int rb = 0; rb < (M == 256 ? 2 : 1); ++rb) {
             const uint64_t qd = umma_desc_k128(q_base + (k / 4) * C::kQHalfBytes + rb * 128 * 128 + ko);
@@ -263,54 +269,87 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
           umma_bf16(d_tmem, kd, qd, umma_idesc(kTcKeyTile, M), k > 0 ? 1u : 0u);
         }
       }
-      umma_commit(&mma_bar[buf]);
+      umma_commit(&mma_bar[s]);
       return true;
     };
 
-    // ---- pass 1: running (max, sum) of this thread's query row(s) over its key columns
+    // ---- prologue of the item: query rows (replicated across lane quarters) and the first key tiles
+    bool issue_ok = true;
+    if (tid == 0) {
+      mbar_arrive_expect_tx(q_bar, C::kQTxBytes);
+      const int qrow0 = (b * p.n_q_heads + g * p.group) * p.window;
+#pragma unroll
+      for (int rep = 0; rep < C::kRep; ++rep)
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf)
+          tma_load_2d(q_s + hf * C::kQHalfBytes + rep * M * 128, &tmap_q, hf * 64, qrow0, q_bar);
+      for (int ti = 0; ti < min(n_tiles, kTcStages); ++ti) load_tile(ti);
+      issue_ok = tc_mbar_wait(q_bar, q_parity);
+      if (issue_ok) issue_ok = issue(0);
+    }
+    q_parity ^= 1u;
+    if (PASS == 2) {
+      for (int r = tid; r < M; r += kTcThreads) s_mrow[r] = __ldcg(&p.mrow[(size_t)unit * M + r]);
+      __syncthreads();
+    }
+
+    // ---- the item's tiles: MMA of tile ti+1 runs while tile ti is reduced out of TMEM
     float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // second pair: row tid+128 when M == 256
-    const int row0 = tid % M;
-    const int limit0 = t - p.window + (row0 % p.window);
+    const int limit0 = t - p.window + ((tid % M) % p.window);
     const int limit1 = t - p.window + ((tid + 128) % p.window);
     const int col_begin = M < 128 ? (tid / M) * C::kColsPerThread : 0;
-    bool issue_ok = true;
-    if (tid == 0) issue_ok = issue(1, 0, 0);
+    float* u = p.u + (size_t)g * p.total_tokens + cu;
     for (int ti = 0; ti < n_tiles; ++ti) {
-      const int buf = C::kBufs == 2 ? (ti & 1) : 0;
-      if (C::kBufs == 2 && tid == 0 && ti + 1 < n_tiles && issue_ok) issue_ok = issue(1, ti + 1, (ti + 1) & 1);
-      bool ok = issue_ok && tc_mbar_wait(&mma_bar[buf], mma_cnt[buf] & 1u);
-      ++mma_cnt[buf];
+      const uint32_t gi = gt + ti, s = gi % kTcStages;
+      if (tid == 0 && ti + 1 < n_tiles && issue_ok) issue_ok = issue(ti + 1);
+      const bool ok = issue_ok && tc_mbar_wait(&mma_bar[s], (gi / kTcStages) & 1u);
       tc_fence_after_sync();
+      if (tid == 0 && ok && ti + kTcStages < n_tiles) load_tile(ti + kTcStages);   // the MMA is done with stage s
       if (ok) {
         const int tile_c0 = key_begin + ti * kTcKeyTile;
-        const bool masked = tile_c0 + kTcKeyTile > t - p.window;
+        const uint32_t acc_addr = tmem_lane + s * C::kBufCols;
+        if (PASS == 1) {
+          const bool masked = tile_c0 + kTcKeyTile > t - p.window;
 #pragma unroll
-        for (int cc = 0; cc < C::kColsPerThread; cc += 32) {
-          float v[32];
-          tmem_ld32(tmem_lane + (uint32_t)buf * 128u + (uint32_t)(col_begin + cc), v);
-          p1_update(v, masked, tile_c0 + col_begin + cc, limit0, p.scale_log2, m0, l0);
-        }
-        if (M == 256) {
-#pragma unroll
-          for (int cc = 0; cc < 128; cc += 32) {
+          for (int cc = 0; cc < C::kColsPerThread; cc += 32) {
             float v[32];
-            tmem_ld32(tmem_lane + 128u + (uint32_t)cc, v);
-            p1_update(v, masked, tile_c0 + cc, limit1, p.scale_log2, m1, l1);
+            tmem_ld32(acc_addr + (uint32_t)(col_begin + cc), v);
+            p1_update(v, masked, tile_c0 + col_begin + cc, limit0, p.scale_log2, m0, l0);
           }
+          if (M == 256) {
+#pragma unroll
+            for (int cc = 0; cc < 128; cc += 32) {
+              float v[32];
+              tmem_ld32(acc_addr + 128u + (uint32_t)cc, v);
+              p1_update(v, masked, tile_c0 + cc, limit1, p.scale_log2, m1, l1);
+            }
+          }
+        } else {
+          float acc = 0.f;
+#pragma unroll
+          for (int cc = 0; cc < M; cc += 32) {
+            float v[32];
+            tmem_ld32(acc_addr + (uint32_t)cc, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) acc += fast_exp2(fmaf(v[i], p.scale_log2, -s_mrow[cc + i]));
+          }
+          const int key = tile_c0 + tid;
+          if (key < key_end) u[key] = acc;
         }
       }
       tc_fence_before_sync();
       aborted = __syncthreads_or(ok ? 0 : 1) != 0;
       if (aborted) break;
-      if (C::kBufs == 1 && tid == 0 && ti + 1 < n_tiles) issue_ok = issue(1, ti + 1, 0);
     }
     if (aborted) break;
+    gt += (uint32_t)n_tiles;
 
-    // ---- publish this split's row statistics; the last split of the unit merges them
-    s_stat[tid] = make_float2(m0, l0);
-    if (M == 256) s_stat[128 + tid] = make_float2(m1, l1);
-    __syncthreads();
-    {
+    if (PASS == 1) {
+      // ---- publish this split's row statistics; the last split of the unit merges them into
+      //      mrow[r] = m_r + log2(l_r) (log2 domain; +inf for rows without visible keys)
+      s_stat[tid] = make_float2(m0, l0);
+      if (M == 256) s_stat[128 + tid] = make_float2(m1, l1);
+      __syncthreads();
       float2* out = p.stats_part + ((size_t)unit * p.n_splits + split) * M;
       for (int r = tid; r < M; r += kTcThreads) {
         float m = -INFINITY;
@@ -323,86 +362,27 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
         }
         out[r] = make_float2(m, l);
       }
-    }
-    __threadfence();
-    __syncthreads();
-    const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
-    if (tid == 0) s_ctl[1] = (atomicAdd(&p.unit_ticket[unit], 1) == n_splits_u - 1) ? 1 : 0;
-    __syncthreads();
-    if (s_ctl[1]) {
-      // mrow[r] = m_r + log2(l_r) in the log2 domain, +inf for rows without visible keys
-      __threadfence();
-      for (int r = tid; r < M; r += kTcThreads) {
-        const float2* part = p.stats_part + (size_t)unit * p.n_splits * M + r;
-        float m = -INFINITY;
-        for (int s = 0; s < n_splits_u; ++s) m = fmaxf(m, __ldcg(&part[(size_t)s * M]).x);
-        float l = 0.f;
-        if (m > -INFINITY)
-          for (int s = 0; s < n_splits_u; ++s) {
-            const float2 v = __ldcg(&part[(size_t)s * M]);
-            l += v.y * exp2f(v.x - m);
-          }
-        p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
-      }
       __threadfence();
       __syncthreads();
-      if (tid == 0) atomicExch(&p.unit_ready[unit], 1);
-    }
-
-    // ---- pass 2 over the prefix keys of this split, from the tiles still in shared memory
-    const int key_end2 = min(key_end1, P);
-    if (key_begin < key_end2) {
-      if (tid == 0) {
-        int ok = 1;
-        if (tc_ld_acquire(&p.unit_ready[unit]) == 0) {
-          const uint64_t t0 = tc_timer_ns();
-          while (tc_ld_acquire(&p.unit_ready[unit]) == 0) {
-            __nanosleep(100);
-            if (tc_timer_ns() - t0 > 2000000000ull) {
-              ok = 0;
-              break;
+      const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
+      if (tid == 0) s_ctl[1] = (atomicAdd(&p.unit_ticket[unit], 1) == n_splits_u - 1) ? 1 : 0;
+      __syncthreads();
+      if (s_ctl[1]) {
+        __threadfence();
+        for (int r = tid; r < M; r += kTcThreads) {
+          const float2* part = p.stats_part + (size_t)unit * p.n_splits * M + r;
+          float m = -INFINITY;
+          for (int sp = 0; sp < n_splits_u; ++sp) m = fmaxf(m, __ldcg(&part[(size_t)sp * M]).x);
+          float l = 0.f;
+          if (m > -INFINITY)
+            for (int sp = 0; sp < n_splits_u; ++sp) {
+              const float2 v = __ldcg(&part[(size_t)sp * M]);
+              l += v.y * exp2f(v.x - m);
             }
-          }
+          p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
         }
-        s_ctl[2] = ok;
       }
-      __syncthreads();
-      if (!s_ctl[2]) {
-        aborted = true;
-        break;
-      }
-      for (int r = tid; r < M; r += kTcThreads) s_mrow[r] = __ldcg(&p.mrow[(size_t)unit * M + r]);
-      __syncthreads();
-      const int n_tiles2 = (key_end2 - key_begin + kTcKeyTile - 1) / kTcKeyTile;
-      float* u = p.u + (size_t)g * p.total_tokens + cu;
-      issue_ok = true;
-      if (tid == 0) issue_ok = issue(2, 0, 0);
-      for (int ti = 0; ti < n_tiles2; ++ti) {
-        const int buf = C::kBufs == 2 ? (ti & 1) : 0;
-        if (C::kBufs == 2 && tid == 0 && ti + 1 < n_tiles2 && issue_ok) issue_ok = issue(2, ti + 1, (ti + 1) & 1);
-        bool ok = issue_ok && tc_mbar_wait(&mma_bar[buf], mma_cnt[buf] & 1u);
-        ++mma_cnt[buf];
-        tc_fence_after_sync();
-        if (ok) {
-          float acc = 0.f;
-#pragma unroll
-          for (int cc = 0; cc < M; cc += 32) {
-            float v[32];
-            tmem_ld32(tmem_lane + (uint32_t)buf * 128u + (uint32_t)cc, v);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc += fast_exp2(fmaf(v[i], p.scale_log2, -s_mrow[cc + i]));
-          }
-          const int key = key_begin + ti * kTcKeyTile + tid;
-          if (key < key_end2) u[key] = acc;
-        }
-        tc_fence_before_sync();
-        aborted = __syncthreads_or(ok ? 0 : 1) != 0;
-        if (aborted) break;
-        if (C::kBufs == 1 && tid == 0 && ti + 1 < n_tiles2) issue_ok = issue(2, ti + 1, 0);
-      }
-      if (aborted) break;
     }
-    item_parity ^= 1u;
   }
 
   // ---- teardown: every MMA has completed (its barrier was waited on) before TMEM goes back
@@ -412,7 +392,7 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == 0) tmem_dealloc(tmem_base, C::kTmemCols);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -445,26 +425,24 @@ bool tc_make_tmap(CUtensorMap* tmap, const void* base, int rank, const cuuint64_
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Key tiles per work item: large enough to amortise the per-item prologue, small enough to fill the GPU.
 int tc_tiles(int M, int head_dim, int units, int max_seqlen, int* ctas_per_sm) {
   if (M != 32 && M != 64 && M != 128 && M != 256) return 0;
   if (head_dim != 64 && head_dim != 128) return 0;
   const int sms = sm_count();
-  int tiles = M == 256 ? 4 : 2;
-  while (tiles > 1 && (int64_t)units * ((max_seqlen + tiles * kTcKeyTile - 1) / (tiles * kTcKeyTile)) < 2 * sms) --tiles;
-  const int ctas = M == 256 ? 1 : 2;
-  const int splits = (max_seqlen + tiles * kTcKeyTile - 1) / (tiles * kTcKeyTile);
-  // splits of a unit wait for each other: all of them must be in flight at once, with room to spare
-  if (splits * 4 > sms * ctas) return 0;
-  *ctas_per_sm = ctas;
+  int tiles = 8;
+  while (tiles > 1 && (int64_t)units * ((max_seqlen + tiles * kTcKeyTile - 1) / (tiles * kTcKeyTile)) < 4 * sms)
+    tiles >>= 1;
+  *ctas_per_sm = M == 256 ? 1 : 2;
   return tiles;
 }
 
-template <int D, int M>
+template <int D, int M, int PASS>
 xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int ctas_per_sm,
                      cudaStream_t st) {
   using C = TcCfg<D, M>;
-  size_t smem = C::smem_bytes(p.slice_tiles);
-  // keep a third CTA off the SM: each CTA holds 256 of the 512 TMEM columns
+  size_t smem = C::kSmemBytes;
+  // keep further CTAs off the SM: the resident ones hold all 512 TMEM columns between them
   const size_t floor_bytes = ctas_per_sm == 2 ? 80 * 1024 : 120 * 1024;
   if (smem < floor_bytes) smem = floor_bytes;
   static bool done[64] = {};
@@ -472,16 +450,24 @@ xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScorePa
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
   if (!done[dev]) {
-    if (cudaFuncSetAttribute(score_tc_kernel<D, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(score_tc_kernel<D, M, PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024) != cudaSuccess)
       return XKV_ERR_CUDA;
     done[dev] = true;
   }
   int grid = sm_count() * ctas_per_sm;
   if (grid > p.n_work) grid = p.n_work;
-  score_tc_kernel<D, M><<<grid, kTcThreads, smem, st>>>(tq, tk, p);
+  score_tc_kernel<D, M, PASS><<<grid, kTcThreads, smem, st>>>(tq, tk, p);
   count_launch();
   return check_launch();
+}
+
+template <int D, int M>
+xkv_status tc_launch_both(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int ctas_per_sm,
+                          cudaStream_t st) {
+  xkv_status s = tc_launch<D, M, 1>(tq, tk, p, ctas_per_sm, st);
+  if (s != XKV_OK) return s;
+  return tc_launch<D, M, 2>(tq, tk, p, ctas_per_sm, st);
 }
 
 }  // namespace
@@ -499,7 +485,7 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
   const int units = p.batch * p.n_kv_heads;
   int ctas = 1;
   const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen, &ctas);
-  if (tiles == 0 || tiles != p.slice_tiles) return XKV_ERR_UNSUPPORTED;
+  if (tiles == 0 || tiles * kTcKeyTile != p.split_keys) return XKV_ERR_UNSUPPORTED;
   CUtensorMap tq, tk;
   {
     const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)p.batch * p.n_q_heads * p.window};
@@ -514,7 +500,7 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
     if (!tc_make_tmap(&tk, p.k, 3, dims, strides, box)) return XKV_ERR_CUDA;
   }
 #define XKV_TC_CASE(DD, MM) \
-  if (head_dim == DD && p.M == MM) return tc_launch<DD, MM>(tq, tk, p, ctas, st);
+  if (head_dim == DD && p.M == MM) return tc_launch_both<DD, MM>(tq, tk, p, ctas, st);
   XKV_TC_CASE(128, 32) XKV_TC_CASE(128, 64) XKV_TC_CASE(128, 128) XKV_TC_CASE(128, 256)
   XKV_TC_CASE(64, 32) XKV_TC_CASE(64, 64) XKV_TC_CASE(64, 128) XKV_TC_CASE(64, 256)
 #undef XKV_TC_CASE
