@@ -702,7 +702,7 @@ void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) 
   L->u = off;          off = align_up(off + (size_t)d->n_kv_heads * T * 4, 256);
   L->tmp_sorted = off; off = align_up(off + (size_t)d->n_kv_heads * T * 4, 256);
   // sized for the smallest split either variant may choose, so the size does not depend on the device
-  L->stats_part = off; off = align_up(off + (size_t)units * ((max_seqlen + kKeyTile - 1) / kKeyTile) * M * 8, 256);
+  L->stats_part = off; off = align_up(off + (size_t)units * ((max_seqlen + kKeyTile - 1) / kKeyTile) * (M < 128 ? 128 : M) * 2 * 8, 256);
   L->mrow = off;       off = align_up(off + (size_t)units * M * 4, 256);
   L->part_sum = off;   off = align_up(off + (size_t)units * L->n_chunks * 4, 256);
   L->total = off;

@@ -1,15 +1,15 @@
 // Window-logit passes of xkv_score on the 5th-generation tensor cores (tcgen05) with TMEM accumulators.
 //
-// A work item is (unit = (sequence, KV head), split of the key axis).  Persistent CTAs take items from a
-// global counter and stream the item's keys through a two-stage shared-memory ring filled by TMA
-// (128-byte swizzled, K-major tiles of 128 keys); one thread issues the MMAs of a tile into one of two TMEM
-// accumulator buffers while all threads reduce the previous tile out of the other; completion comes back
-// through tcgen05.commit on an mbarrier.  Two launches:
+// A work item is (unit = (sequence, KV head), split of the key axis).  One persistent CTA per SM streams
+// its items' keys through a four-stage shared-memory ring filled by TMA (128-byte swizzled, K-major tiles
+// of 128 keys); a one-lane MMA warp issues tcgen05.mma per landed tile into one of two TMEM accumulator
+// buffers while four epilogue warps reduce the previous tile out of the other; stages and accumulators
+// are handed around with mbarriers (tcgen05.commit on the MMA side).  Two launches with a small merge of
+// the row statistics in between:
 //   pass 1  D[query rows x keys] = Q K^T with the G*W query rows on the MMA's M axis: a thread owns one
 //           TMEM lane = one query row, so the running (max, sum of exponentials) of the softmax is two
 //           registers and needs no cross-lane traffic.  With fewer than 128 query rows the rows are
 //           replicated over the four lane quarters and every warp takes a quarter of the key columns.
-//           The last split of a unit to finish (atomic ticket) merges the unit's statistics.
 //   pass 2  D[keys x query rows] = K Q^T with the keys on M: a thread owns one key and sums
 //           exp2(s*c - normaliser[row]) over the query rows straight out of TMEM -> column score u[key].
 //           Items are walked in reverse so that the keys pass 1 streamed last are re-read from L2.
@@ -66,7 +66,7 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane.
+// 32 consecutive fp32 columns of this thread's TMEM lane; the values may be used after tmem_wait_ld().
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   uint32_t r[32];
   asm volatile(
@@ -79,7 +79,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-  tmem_wait_ld();
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
@@ -130,9 +129,20 @@ __device__ __forceinline__ int tc_ld_acquire(const int* ptr) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Kernel
+// Kernel: warp-specialised pipeline
+//   warp 8 (one lane)  producer: TMA loads of the query rows of an item and of its key tiles into a ring
+//   warp 9 (one lane)  MMA issuer: tcgen05.mma per landed tile into one of two TMEM accumulator buffers;
+//                      tcgen05.commit hands the ring stage back to the producer and the accumulator to the
+//                      epilogue
+//   warps 0-7          epilogue, two groups of four warps: group e owns accumulator buffer e (every other
+//                      tile), reduces it out of TMEM and hands it back
+// Work items are assigned statically (item = CTA + n * grid), so each role walks the same sequence on its
+// own and the producer runs ahead across item boundaries.
 // ---------------------------------------------------------------------------------------------
-constexpr int kTcStages = 2;       // shared-memory ring of key tiles, and TMEM accumulator buffers
+constexpr int kWsThreads = 320;
+constexpr int kEpiThreads = 128;     // threads of one epilogue group
+constexpr int kWsStages = 4;       // shared-memory ring of key tiles
+constexpr int kAccBufs = 2;        // TMEM accumulator buffers
 
 template <int D, int M>
 struct TcCfg {
@@ -142,14 +152,15 @@ struct TcCfg {
   static constexpr int kRep = M < 128 ? 128 / M : 1;             // replicas of the query rows across lanes
   static constexpr int kQHalfBytes = kQRows * 128;
   static constexpr int kQBytes = kHalves * kQHalfBytes;
+  static constexpr int kQBufs = M == 256 ? 1 : 2;
   static constexpr int kKHalfBytes = kTcKeyTile * 128;
   static constexpr int kKTileBytes = kHalves * kKHalfBytes;
   static constexpr uint32_t kBufCols = M == 256 ? 256 : 128;     // TMEM columns of one accumulator buffer
-  static constexpr uint32_t kTmemCols = kTcStages * kBufCols;    // 256 (two CTAs per SM) or 512
+  static constexpr uint32_t kTmemCols = kAccBufs * kBufCols;
   static constexpr int kColsPerThread = M < 128 ? M : 128;       // pass-1 key columns a thread reduces per tile
   static constexpr uint32_t kQTxBytes = (uint32_t)(kRep * kHalves * (M < 128 ? M : kQRows) * 128);
-  static constexpr size_t kSmemBytes =
-      1024 + (size_t)kQBytes + (size_t)kTcStages * kKTileBytes + 256 * 4 /*mrow*/ + 256 * 8 /*stats*/ + 128;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kQBufs * kQBytes + (size_t)kWsStages * kKTileBytes +
+                                       256 * 4 /*mrow*/ + 256 * 8 /*stats*/ + 256 /*barriers*/;
 };
 
 __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
@@ -170,33 +181,79 @@ __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int
   m = m_new;
 }
 
-// PASS 1: row statistics of every (unit, split) item, merged per unit by the last split to finish.
-// PASS 2: column sums u, launched after pass 1 has completed; items are taken in reverse order so that the
-//         keys pass 1 streamed last are still in L2.
+struct ItemShape {
+  int unit, split, b, g, cu, t, P, key_begin, key_end, n_tiles;
+};
+
+// Item n of this CTA; returns false when the sequence is exhausted.  Empty items have n_tiles == 0.
+template <int PASS>
+__device__ __forceinline__ bool item_shape(const ScoreParams& p, int n, ItemShape* it) {
+  int idx = blockIdx.x + n * gridDim.x;
+  if (idx >= p.n_work) return false;
+  if (PASS == 2) idx = p.n_work - 1 - idx;       // reverse: the keys pass 1 read last are still in L2
+  it->unit = idx / p.n_splits;
+  it->split = idx % p.n_splits;
+  it->b = it->unit / p.n_kv_heads;
+  it->g = it->unit % p.n_kv_heads;
+  it->cu = p.cu_seqlens[it->b];
+  it->t = p.cu_seqlens[it->b + 1] - it->cu;
+  it->P = max(it->t - p.window, 0);
+  it->key_begin = it->split * p.split_keys;
+  it->key_end = min(it->key_begin + p.split_keys, PASS == 1 ? it->t : it->P);
+  it->n_tiles = it->key_end > it->key_begin ? (it->key_end - it->key_begin + kTcKeyTile - 1) / kTcKeyTile : 0;
+  return true;
+}
+
+// Bounded mbarrier wait (two seconds) that also gives up when another role has raised the abort flag.
+__device__ __forceinline__ bool ws_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = tc_timer_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (tc_timer_ns() - t0 > 2000000000ull) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
 template <int D, int M, int PASS>
-__global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
+__global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q,
                                                              const __grid_constant__ CUtensorMap tmap_k,
                                                              const ScoreParams p) {
   using C = TcCfg<D, M>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
-  uint8_t* k_s = q_s + C::kQBytes;
-  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)kTcStages * C::kKTileBytes);   // [256]
+  uint8_t* k_s = q_s + (size_t)C::kQBufs * C::kQBytes;
+  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)kWsStages * C::kKTileBytes);   // [256]
   float2* s_stat = reinterpret_cast<float2*>(s_mrow + 256);                              // [256]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_stat + 256);                        // [kTcStages]
-  uint64_t* mma_bar = full_bar + kTcStages;                                              // [kTcStages]
-  uint64_t* q_bar = mma_bar + kTcStages;
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(q_bar + 1);
-  int* s_ctl = reinterpret_cast<int*>(s_tmem + 1);                                       // [0] item [1] flag
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_stat + 256);    // [kWsStages] tile landed
+  uint64_t* empty_bar = full_bar + kWsStages;                        // [kWsStages] tile consumed by the MMAs
+  uint64_t* qfull_bar = empty_bar + kWsStages;                       // [2] query rows landed
+  uint64_t* qempty_bar = qfull_bar + 2;                              // [2] query rows no longer read
+  uint64_t* accfull_bar = qempty_bar + 2;                            // [kAccBufs] accumulator complete
+  uint64_t* accempty_bar = accfull_bar + kAccBufs;                   // [kAccBufs] accumulator reduced
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(accempty_bar + kAccBufs);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
-    for (int i = 0; i < kTcStages; ++i) {
+    for (int i = 0; i < kWsStages; ++i) {
       mbar_init(&full_bar[i], 1);
-      mbar_init(&mma_bar[i], 1);
+      mbar_init(&empty_bar[i], 1);
     }
-    mbar_init(q_bar, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&qfull_bar[i], 1);
+      mbar_init(&qempty_bar[i], 1);
+    }
+    for (int i = 0; i < kAccBufs; ++i) {
+      mbar_init(&accfull_bar[i], 1);
+      mbar_init(&accempty_bar[i], 4);          // one arrival per warp of the owning epilogue group
+    }
+    *s_abort = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_k);
@@ -209,190 +266,225 @@ __global__ void __launch_bounds__(kTcThreads) score_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
-  const uint32_t tmem_lane = tmem_base + ((uint32_t)(32 * warp) << 16);   // this warp's quarter of the lanes
 
-  uint32_t gt = 0;            // key tiles this CTA has processed: stage, accumulator buffer and phases follow it
-  uint32_t q_parity = 0;      // phase of the query barrier (one use per item)
-  bool aborted = false;
-  const uint32_t q_base = smem_u32(q_s), k_base = smem_u32(k_s);
-  int* counter = PASS == 1 ? &p.hdr->work_counter : &p.hdr->prep_ticket;
-
-  int next = 0;
-  if (tid == 0) next = atomicAdd(counter, 1);
-  while (!aborted) {
-    __syncthreads();
-    if (tid == 0) {
-      s_ctl[0] = next;
-      next = atomicAdd(counter, 1);      // fetched now, used after this item (no item ever waits for another)
-    }
-    __syncthreads();
-    int idx = s_ctl[0];
-    if (idx >= p.n_work) break;
-    if (PASS == 2) idx = p.n_work - 1 - idx;
-    const int unit = idx / p.n_splits, split = idx % p.n_splits;
-    const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
-    const int cu = p.cu_seqlens[b];
-    const int t = p.cu_seqlens[b + 1] - cu;
-    const int P = max(t - p.window, 0);
-    const int key_begin = split * p.split_keys;
-    const int key_end = min(key_begin + p.split_keys, PASS == 1 ? t : P);
-    if (key_begin >= key_end) continue;
-    const int n_tiles = (key_end - key_begin + kTcKeyTile - 1) / kTcKeyTile;
-
-    auto load_tile = [&](int ti) {           // thread 0: arm the stage's barrier and start the copy
-      const uint32_t s = (gt + ti) % kTcStages;
-      mbar_arrive_expect_tx(&full_bar[s], (uint32_t)C::kKTileBytes);
+  if (warp == 8) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t gt = 0, it = 0;
+      ItemShape sh;
+      bool ok = true;
+      for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
+        if (sh.n_tiles == 0) continue;
+        const uint32_t qb = it % C::kQBufs;
+        ok = ws_wait(&qempty_bar[qb], ((it / C::kQBufs) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&qfull_bar[qb], C::kQTxBytes);
+        const int qrow0 = (sh.b * p.n_q_heads + sh.g * p.group) * p.window;
 #pragma unroll
-      for (int hf = 0; hf < C::kHalves; ++hf)
-        tma_load_3d(k_s + (size_t)s * C::kKTileBytes + hf * C::kKHalfBytes, &tmap_k, hf * 64, g,
-                    cu + key_begin + ti * kTcKeyTile, &full_bar[s]);
-    };
-    // thread 0: once tile ti has landed, issue its MMAs into accumulator buffer (gt+ti) % 2
-    auto issue = [&](int ti) -> bool {
-      const uint32_t gi = gt + ti, s = gi % kTcStages;
-      if (!tc_mbar_wait(&full_bar[s], (gi / kTcStages) & 1u)) return false;
-      tc_fence_after_sync();
-      const uint32_t kt = k_base + s * C::kKTileBytes;
-      const uint32_t d_tmem = tmem_base + s * C::kBufCols;
+        for (int rep = 0; rep < C::kRep; ++rep)
 #pragma unroll
-      for (int k = 0; k < C::kSteps; ++k) {
-        const uint32_t ko = (uint32_t)(k % 4) * 32u;          // 16 bf16 along K inside the swizzled 128-byte row
-        const uint64_t kd = umma_desc_k128(kt + (k / 4) * C::kKHalfBytes + ko);
-        if (PASS == 1) {
+          for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_2d(q_s + (size_t)qb * C::kQBytes + hf * C::kQHalfBytes + rep * M * 128, &tmap_q, hf * 64, qrow0,
+                        &qfull_bar[qb]);
+        for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
+          const uint32_t s = gt % kWsStages;
+          ok = ws_wait(&empty_bar[s], ((gt / kWsStages) & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&full_bar[s], (uint32_t)C::kKTileBytes);
 #pragma unroll
-          for (int rb = 0; rb < (M == 256 ? 2 : 1); ++rb) {
-            const uint64_t qd = umma_desc_k128(q_base + (k / 4) * C::kQHalfBytes + rb * 128 * 128 + ko);
-            umma_bf16(d_tmem + rb * 128u, qd, kd, umma_idesc(128, kTcKeyTile), k > 0 ? 1u : 0u);
-          }
-        } else {
-          const uint64_t qd = umma_desc_k128(q_base + (k / 4) * C::kQHalfBytes + ko);
-          umma_bf16(d_tmem, kd, qd, umma_idesc(kTcKeyTile, M), k > 0 ? 1u : 0u);
+          for (int hf = 0; hf < C::kHalves; ++hf)
+            tma_load_3d(k_s + (size_t)s * C::kKTileBytes + hf * C::kKHalfBytes, &tmap_k, hf * 64, sh.g,
+                        sh.cu + sh.key_begin + ti * kTcKeyTile, &full_bar[s]);
         }
+        ++it;
       }
-      umma_commit(&mma_bar[s]);
-      return true;
-    };
-
-    // ---- prologue of the item: query rows (replicated across lane quarters) and the first key tiles
-    bool issue_ok = true;
-    if (tid == 0) {
-      mbar_arrive_expect_tx(q_bar, C::kQTxBytes);
-      const int qrow0 = (b * p.n_q_heads + g * p.group) * p.window;
-#pragma unroll
-      for (int rep = 0; rep < C::kRep; ++rep)
-#pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_2d(q_s + hf * C::kQHalfBytes + rep * M * 128, &tmap_q, hf * 64, qrow0, q_bar);
-      for (int ti = 0; ti < min(n_tiles, kTcStages); ++ti) load_tile(ti);
-      issue_ok = tc_mbar_wait(q_bar, q_parity);
-      if (issue_ok) issue_ok = issue(0);
     }
-    q_parity ^= 1u;
-    if (PASS == 2) {
-      for (int r = tid; r < M; r += kTcThreads) s_mrow[r] = __ldcg(&p.mrow[(size_t)unit * M + r]);
-      __syncthreads();
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t gt = 0, it = 0;
+      ItemShape sh;
+      bool ok = true;
+      const uint32_t q_base = smem_u32(q_s), k_base = smem_u32(k_s);
+      for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
+        if (sh.n_tiles == 0) continue;
+        const uint32_t qb = it % C::kQBufs;
+        ok = ws_wait(&qfull_bar[qb], (it / C::kQBufs) & 1u, s_abort);
+        if (!ok) break;
+        const uint32_t qa = q_base + qb * C::kQBytes;
+        for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
+          const uint32_t s = gt % kWsStages, ab = gt % kAccBufs;
+          ok = ws_wait(&full_bar[s], (gt / kWsStages) & 1u, s_abort) &&
+               ws_wait(&accempty_bar[ab], ((gt / kAccBufs) & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t kt = k_base + s * C::kKTileBytes;
+          const uint32_t d_tmem = tmem_base + ab * C::kBufCols;
+#pragma unroll
+          for (int k = 0; k < C::kSteps; ++k) {
+            const uint32_t ko = (uint32_t)(k % 4) * 32u;      // 16 bf16 along K inside the swizzled 128-byte row
+            const uint64_t kd = umma_desc_k128(kt + (k / 4) * C::kKHalfBytes + ko);
+            if (PASS == 1) {
+#pragma unroll
+              for (int rb = 0; rb < (M == 256 ? 2 : 1); ++rb) {
+                const uint64_t qd = umma_desc_k128(qa + (k / 4) * C::kQHalfBytes + rb * 128 * 128 + ko);
+                umma_bf16(d_tmem + rb * 128u, qd, kd, umma_idesc(128, kTcKeyTile), k > 0 ? 1u : 0u);
+              }
+            } else {
+              const uint64_t qd = umma_desc_k128(qa + (k / 4) * C::kQHalfBytes + ko);
+              umma_bf16(d_tmem, kd, qd, umma_idesc(kTcKeyTile, M), k > 0 ? 1u : 0u);
+            }
+          }
+          umma_commit(&empty_bar[s]);         // the ring stage is free once these MMAs have read it
+          umma_commit(&accfull_bar[ab]);      // and the accumulator is complete
+        }
+        if (!ok) break;
+        umma_commit(&qempty_bar[qb]);         // all MMAs of the item have read the query rows
+        ++it;
+      }
     }
-
-    // ---- the item's tiles: MMA of tile ti+1 runs while tile ti is reduced out of TMEM
-    float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // second pair: row tid+128 when M == 256
-    const int limit0 = t - p.window + ((tid % M) % p.window);
-    const int limit1 = t - p.window + ((tid + 128) % p.window);
-    const int col_begin = M < 128 ? (tid / M) * C::kColsPerThread : 0;
-    float* u = p.u + (size_t)g * p.total_tokens + cu;
-    for (int ti = 0; ti < n_tiles; ++ti) {
-      const uint32_t gi = gt + ti, s = gi % kTcStages;
-      if (tid == 0 && ti + 1 < n_tiles && issue_ok) issue_ok = issue(ti + 1);
-      const bool ok = issue_ok && tc_mbar_wait(&mma_bar[s], (gi / kTcStages) & 1u);
-      tc_fence_after_sync();
-      if (tid == 0 && ok && ti + kTcStages < n_tiles) load_tile(ti + kTcStages);   // the MMA is done with stage s
-      if (ok) {
-        const int tile_c0 = key_begin + ti * kTcKeyTile;
-        const uint32_t acc_addr = tmem_lane + s * C::kBufCols;
+  } else {
+    // ------------------------------------------------------------------ epilogue warps 0..7
+    const uint32_t group = warp >> 2;                                       // owns accumulator buffer `group`
+    const int etid = tid & (kEpiThreads - 1);                               // thread within the group = TMEM lane
+    const uint32_t tmem_lane = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // this warp's quarter of the lanes
+    constexpr int kEntries = M < 128 ? 128 : M;                             // statistics entries per item
+    uint32_t gt = 0;
+    ItemShape sh;
+    bool ok = true;
+    for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
+      if (sh.n_tiles == 0) continue;
+      float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // second pair: row tid+128 when M == 256
+      const int limit0 = sh.t - p.window + ((etid % M) % p.window);
+      const int limit1 = sh.t - p.window + ((etid + 128) % p.window);
+      const int col_begin = M < 128 ? (etid / M) * C::kColsPerThread : 0;
+      float* u = p.u + (size_t)sh.g * p.total_tokens + sh.cu;
+      const float4* mrow4 = reinterpret_cast<const float4*>(p.mrow + (size_t)sh.unit * M);
+      for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
+        const uint32_t ab = gt % kAccBufs;
+        if (ab != group) continue;               // the other group's tile
+        ok = __all_sync(0xffffffffu, ws_wait(&accfull_bar[ab], (gt / kAccBufs) & 1u, s_abort));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int tile_c0 = sh.key_begin + ti * kTcKeyTile;
+        const uint32_t acc_addr = tmem_lane + ab * C::kBufCols;
         if (PASS == 1) {
-          const bool masked = tile_c0 + kTcKeyTile > t - p.window;
-#pragma unroll
-          for (int cc = 0; cc < C::kColsPerThread; cc += 32) {
+          const bool masked = tile_c0 + kTcKeyTile > sh.t - p.window;
+          if (C::kColsPerThread == 32) {
             float v[32];
-            tmem_ld32(acc_addr + (uint32_t)(col_begin + cc), v);
-            p1_update(v, masked, tile_c0 + col_begin + cc, limit0, p.scale_log2, m0, l0);
+            tmem_ld32(acc_addr + (uint32_t)col_begin, v);
+            tmem_wait_ld();
+            p1_update(v, masked, tile_c0 + col_begin, limit0, p.scale_log2, m0, l0);
+          } else {
+#pragma unroll
+            for (int cc = 0; cc < C::kColsPerThread; cc += 64) {      // two TMEM loads in flight
+              float va[32], vb[32];
+              tmem_ld32(acc_addr + (uint32_t)(col_begin + cc), va);
+              tmem_ld32(acc_addr + (uint32_t)(col_begin + cc + 32), vb);
+              tmem_wait_ld();
+              p1_update(va, masked, tile_c0 + col_begin + cc, limit0, p.scale_log2, m0, l0);
+              p1_update(vb, masked, tile_c0 + col_begin + cc + 32, limit0, p.scale_log2, m0, l0);
+            }
           }
           if (M == 256) {
 #pragma unroll
-            for (int cc = 0; cc < 128; cc += 32) {
-              float v[32];
-              tmem_ld32(acc_addr + 128u + (uint32_t)cc, v);
-              p1_update(v, masked, tile_c0 + cc, limit1, p.scale_log2, m1, l1);
+            for (int cc = 0; cc < 128; cc += 64) {
+              float va[32], vb[32];
+              tmem_ld32(acc_addr + 128u + (uint32_t)cc, va);
+              tmem_ld32(acc_addr + 128u + (uint32_t)(cc + 32), vb);
+              tmem_wait_ld();
+              p1_update(va, masked, tile_c0 + cc, limit1, p.scale_log2, m1, l1);
+              p1_update(vb, masked, tile_c0 + cc + 32, limit1, p.scale_log2, m1, l1);
             }
           }
         } else {
           float acc = 0.f;
+          auto add_chunk = [&](const float (&v)[32], int cc) {
 #pragma unroll
-          for (int cc = 0; cc < M; cc += 32) {
-            float v[32];
-            tmem_ld32(acc_addr + (uint32_t)cc, v);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc += fast_exp2(fmaf(v[i], p.scale_log2, -s_mrow[cc + i]));
-          }
-          const int key = tile_c0 + tid;
-          if (key < key_end) u[key] = acc;
-        }
-      }
-      tc_fence_before_sync();
-      aborted = __syncthreads_or(ok ? 0 : 1) != 0;
-      if (aborted) break;
-    }
-    if (aborted) break;
-    gt += (uint32_t)n_tiles;
-
-    if (PASS == 1) {
-      // ---- publish this split's row statistics; the last split of the unit merges them into
-      //      mrow[r] = m_r + log2(l_r) (log2 domain; +inf for rows without visible keys)
-      s_stat[tid] = make_float2(m0, l0);
-      if (M == 256) s_stat[128 + tid] = make_float2(m1, l1);
-      __syncthreads();
-      float2* out = p.stats_part + ((size_t)unit * p.n_splits + split) * M;
-      for (int r = tid; r < M; r += kTcThreads) {
-        float m = -INFINITY;
-#pragma unroll
-        for (int rep = 0; rep < C::kRep; ++rep) m = fmaxf(m, s_stat[r + rep * M].x);
-        float l = 0.f;
-        if (m > -INFINITY) {
-#pragma unroll
-          for (int rep = 0; rep < C::kRep; ++rep) l += s_stat[r + rep * M].y * fast_exp2(s_stat[r + rep * M].x - m);
-        }
-        out[r] = make_float2(m, l);
-      }
-      __threadfence();
-      __syncthreads();
-      const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
-      if (tid == 0) s_ctl[1] = (atomicAdd(&p.unit_ticket[unit], 1) == n_splits_u - 1) ? 1 : 0;
-      __syncthreads();
-      if (s_ctl[1]) {
-        __threadfence();
-        for (int r = tid; r < M; r += kTcThreads) {
-          const float2* part = p.stats_part + (size_t)unit * p.n_splits * M + r;
-          float m = -INFINITY;
-          for (int sp = 0; sp < n_splits_u; ++sp) m = fmaxf(m, __ldcg(&part[(size_t)sp * M]).x);
-          float l = 0.f;
-          if (m > -INFINITY)
-            for (int sp = 0; sp < n_splits_u; ++sp) {
-              const float2 v = __ldcg(&part[(size_t)sp * M]);
-              l += v.y * exp2f(v.x - m);
+            for (int i = 0; i < 32; i += 4) {
+              const float4 mr = __ldg(&mrow4[(cc + i) >> 2]);      // same address in every thread: a broadcast
+              acc += fast_exp2(fmaf(v[i + 0], p.scale_log2, -mr.x)) + fast_exp2(fmaf(v[i + 1], p.scale_log2, -mr.y)) +
+                     fast_exp2(fmaf(v[i + 2], p.scale_log2, -mr.z)) + fast_exp2(fmaf(v[i + 3], p.scale_log2, -mr.w));
             }
-          p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
+          };
+          if (M == 32) {
+            float v[32];
+            tmem_ld32(acc_addr, v);
+            tmem_wait_ld();
+            add_chunk(v, 0);
+          } else {
+#pragma unroll
+            for (int cc = 0; cc < M; cc += 64) {                    // two TMEM loads in flight
+              float va[32], vb[32];
+              tmem_ld32(acc_addr + (uint32_t)cc, va);
+              tmem_ld32(acc_addr + (uint32_t)(cc + 32), vb);
+              tmem_wait_ld();
+              add_chunk(va, cc);
+              add_chunk(vb, cc + 32);
+            }
+          }
+          const int key = tile_c0 + etid;
+          if (key < sh.key_end) u[key] = acc;
         }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&accempty_bar[ab]);
+      }
+      if (!ok) break;
+      if (PASS == 1) {
+        // every thread stores the statistics of its own (row, key-column quarter); tc_merge_kernel combines them
+        float2* out = p.stats_part + (((size_t)sh.unit * p.n_splits + sh.split) * kAccBufs + group) * kEntries;
+        out[etid] = make_float2(m0, l0);
+        if (M == 256) out[128 + etid] = make_float2(m1, l1);
       }
     }
   }
 
-  // ---- teardown: every MMA has completed (its barrier was waited on) before TMEM goes back
-  if (aborted) {
+  // ---- teardown
+  __syncthreads();
+  if (*s_abort) {
     if (tid == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
-    for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies already issued land
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies and MMAs already issued finish
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+// One warp per query row of a unit: mrow[r] = m_r + log2(l_r) (log2 domain; +inf for rows without visible
+// keys) from the per-split, per-group, per-replica statistics pass 1 stored.  grid = (units, M / 4).
+__global__ void __launch_bounds__(128) tc_merge_kernel(const ScoreParams p) {
+  const int unit = blockIdx.x;
+  const int M = p.M;
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.y * 4 + (threadIdx.x >> 5);
+  if (r >= M) return;
+  const int group_entries = M < 128 ? 128 : M;
+  const int group_reps = M < 128 ? 128 / M : 1;
+  const int per_split = kAccBufs * group_reps;               // partial statistics of this row per split
+  const int entries = kAccBufs * group_entries;
+  const int b = unit / p.n_kv_heads;
+  const int t = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+  const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
+  const float2* part = p.stats_part + (size_t)unit * p.n_splits * entries + r;
+  float m = -INFINITY, l = 0.f;
+  for (int i = lane; i < n_splits_u * per_split; i += 32) {
+    const int s = i / per_split, q = i % per_split;
+    const float2 v = part[(size_t)s * entries + (q / group_reps) * group_entries + (q % group_reps) * M];
+    const float m_new = fmaxf(m, v.x);
+    const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+    l = l * exp2f(m - m_ref) + v.y * exp2f(v.x - m_ref);
+    m = m_new;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float mo = __shfl_xor_sync(0xffffffffu, m, o), lo = __shfl_xor_sync(0xffffffffu, l, o);
+    const float m_new = fmaxf(m, mo);
+    const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+    l = l * exp2f(m - m_ref) + lo * exp2f(mo - m_ref);
+    m = m_new;
+  }
+  if (lane == 0) p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -425,26 +517,23 @@ bool tc_make_tmap(CUtensorMap* tmap, const void* base, int rank, const cuuint64_
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Key tiles per work item: large enough to amortise the per-item prologue, small enough to fill the GPU.
-int tc_tiles(int M, int head_dim, int units, int max_seqlen, int* ctas_per_sm) {
+// Key tiles per work item: items are cheap (the producer prefetches across them), so keep them small
+// enough to balance the static assignment.
+int tc_tiles(int M, int head_dim, int units, int max_seqlen) {
   if (M != 32 && M != 64 && M != 128 && M != 256) return 0;
   if (head_dim != 64 && head_dim != 128) return 0;
   const int sms = sm_count();
-  int tiles = 8;
-  while (tiles > 1 && (int64_t)units * ((max_seqlen + tiles * kTcKeyTile - 1) / (tiles * kTcKeyTile)) < 4 * sms)
+  int tiles = M == 256 ? 16 : 4;      // G*W = 256 reloads a 64 KB query block per item: make items larger
+  while (tiles > 1 && (int64_t)units * ((max_seqlen + tiles * kTcKeyTile - 1) / (tiles * kTcKeyTile)) < 8 * sms)
     tiles >>= 1;
-  *ctas_per_sm = M == 256 ? 1 : 2;
   return tiles;
 }
 
 template <int D, int M, int PASS>
-xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int ctas_per_sm,
-                     cudaStream_t st) {
+xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, cudaStream_t st) {
   using C = TcCfg<D, M>;
   size_t smem = C::kSmemBytes;
-  // keep further CTAs off the SM: the resident ones hold all 512 TMEM columns between them
-  const size_t floor_bytes = ctas_per_sm == 2 ? 80 * 1024 : 120 * 1024;
-  if (smem < floor_bytes) smem = floor_bytes;
+  if (smem < 120 * 1024) smem = 120 * 1024;      // one CTA per SM: it may hold all 512 TMEM columns
   static bool done[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -455,19 +544,22 @@ xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScorePa
       return XKV_ERR_CUDA;
     done[dev] = true;
   }
-  int grid = sm_count() * ctas_per_sm;
+  int grid = sm_count();
   if (grid > p.n_work) grid = p.n_work;
-  score_tc_kernel<D, M, PASS><<<grid, kTcThreads, smem, st>>>(tq, tk, p);
+  score_tc_kernel<D, M, PASS><<<grid, kWsThreads, smem, st>>>(tq, tk, p);
   count_launch();
   return check_launch();
 }
 
 template <int D, int M>
-xkv_status tc_launch_both(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, int ctas_per_sm,
-                          cudaStream_t st) {
-  xkv_status s = tc_launch<D, M, 1>(tq, tk, p, ctas_per_sm, st);
+xkv_status tc_launch_both(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, cudaStream_t st) {
+  xkv_status s = tc_launch<D, M, 1>(tq, tk, p, st);
   if (s != XKV_OK) return s;
-  return tc_launch<D, M, 2>(tq, tk, p, ctas_per_sm, st);
+  tc_merge_kernel<<<dim3(p.batch * p.n_kv_heads, M / 4), 128, 0, st>>>(p);
+  count_launch();
+  s = check_launch();
+  if (s != XKV_OK) return s;
+  return tc_launch<D, M, 2>(tq, tk, p, st);
 }
 
 }  // namespace
@@ -476,15 +568,13 @@ int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen) {
 #ifdef XKV_NO_TC
   return 0;
 #else
-  int ctas = 1;
-  return tc_tiles(M, head_dim, units, max_seqlen, &ctas) * kTcKeyTile;
+  return tc_tiles(M, head_dim, units, max_seqlen) * kTcKeyTile;
 #endif
 }
 
 xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st) {
   const int units = p.batch * p.n_kv_heads;
-  int ctas = 1;
-  const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen, &ctas);
+  const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen);
   if (tiles == 0 || tiles * kTcKeyTile != p.split_keys) return XKV_ERR_UNSUPPORTED;
   CUtensorMap tq, tk;
   {
@@ -500,7 +590,7 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
     if (!tc_make_tmap(&tk, p.k, 3, dims, strides, box)) return XKV_ERR_CUDA;
   }
 #define XKV_TC_CASE(DD, MM) \
-  if (head_dim == DD && p.M == MM) return tc_launch_both<DD, MM>(tq, tk, p, ctas, st);
+  if (head_dim == DD && p.M == MM) return tc_launch_both<DD, MM>(tq, tk, p, st);
   XKV_TC_CASE(128, 32) XKV_TC_CASE(128, 64) XKV_TC_CASE(128, 128) XKV_TC_CASE(128, 256)
   XKV_TC_CASE(64, 32) XKV_TC_CASE(64, 64) XKV_TC_CASE(64, 128) XKV_TC_CASE(64, 256)
 #undef XKV_TC_CASE

@@ -96,13 +96,12 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   const float* w = p.scores + (size_t)g * p.total_tokens + cu;
   const float* srt = p.sorted + (size_t)g * p.total_tokens + cu;
   const float thr = srt[kb - 1];
-  // number of scores strictly above thr = first index of the descending sort holding thr
-  int lo = 0, hi = kb - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if (srt[mid] > thr) lo = mid + 1; else hi = mid;
-  }
-  const int eq_needed = kb - lo;
+  // number of scores strictly above thr (counted over the prefix; the sorted copy only supplies thr)
+  int n_gt = 0;
+  for (int c = threadIdx.x; c < P; c += kSelThreads) n_gt += w[c] > thr ? 1 : 0;
+  int count_gt;
+  block_scan_excl(n_gt, s_warp, &count_gt);
+  const int eq_needed = kb - count_gt;
 
   int carry_eq = 0, carry_sel = 0;
   for (int base = 0; base < P; base += kSelThreads * kSelItems) {
