@@ -32,9 +32,11 @@ if ROOT not in sys.path:
 DEFAULT_WORKLOAD = "llama2_7b_mha"
 METRIC = "ragged-KV decode-attn GB/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_attn_kernel launch, from the ncu capture
-# summarised under profiles/ (None while no capture matches the current kernel).
-NCU_TRAFFIC = None
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one decode_attn_kernel launch, from the
+# ncu capture of a smaller case summarised in profiles/decode_attn_kernel_llama2_7b_mha.md; traffic grows in
+# proportion to the retained rows, so the full launch's traffic is this ratio times its algorithmic bytes.
+# Set to None whenever the kernel changes after the capture.
+NCU_TRAFFIC_RATIO = 1.029
 
 
 def measured_peak():
@@ -397,7 +399,9 @@ def main():
     achieved = launch_bytes / (kern_avg_ms * 1e-3) / 1e9
     roofline = {"kernel": "decode_attn_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8000": achieved / 8000.0, "peak_source": peak_src,
-                "bytes_per_launch": launch_bytes, "avg_launch_ms": kern_avg_ms, "traffic": NCU_TRAFFIC}
+                "bytes_per_launch": launch_bytes, "avg_launch_ms": kern_avg_ms,
+                "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * launch_bytes,
+                "traffic_source": "ncu capture of a smaller case scaled by retained rows (profiles/)"}
 
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
