@@ -107,6 +107,14 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const void* tmap, int x, 
       : "memory");
 }
 
+// Plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 __device__ __forceinline__ uint64_t tc_timer_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -143,6 +151,7 @@ constexpr int kWsThreads = 320;
 constexpr int kEpiThreads = 128;     // threads of one epilogue group
 constexpr int kWsStages = 4;       // shared-memory ring of key tiles
 constexpr int kAccBufs = 2;        // TMEM accumulator buffers
+constexpr int kMrowSlots = 4;      // pass 2: ring of row-normaliser vectors (one per item in flight)
 
 template <int D, int M>
 struct TcCfg {
@@ -160,7 +169,7 @@ struct TcCfg {
   static constexpr int kColsPerThread = M < 128 ? M : 128;       // pass-1 key columns a thread reduces per tile
   static constexpr uint32_t kQTxBytes = (uint32_t)(kRep * kHalves * (M < 128 ? M : kQRows) * 128);
   static constexpr size_t kSmemBytes = 1024 + (size_t)kQBufs * kQBytes + (size_t)kWsStages * kKTileBytes +
-                                       256 * 4 /*mrow*/ + 256 * 8 /*stats*/ + 256 /*barriers*/;
+                                       kMrowSlots * 256 * 4 /*row normalisers*/ + 256 /*barriers*/;
 };
 
 __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
@@ -228,9 +237,8 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
   uint8_t* k_s = q_s + (size_t)C::kQBufs * C::kQBytes;
-  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)kWsStages * C::kKTileBytes);   // [256]
-  float2* s_stat = reinterpret_cast<float2*>(s_mrow + 256);                              // [256]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_stat + 256);    // [kWsStages] tile landed
+  float* s_mrow = reinterpret_cast<float*>(k_s + (size_t)kWsStages * C::kKTileBytes);   // [kMrowSlots][256]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_mrow + kMrowSlots * 256);   // [kWsStages] tile landed
   uint64_t* empty_bar = full_bar + kWsStages;                        // [kWsStages] tile consumed by the MMAs
   uint64_t* qfull_bar = empty_bar + kWsStages;                       // [2] query rows landed
   uint64_t* qempty_bar = qfull_bar + 2;                              // [2] query rows no longer read
@@ -278,7 +286,9 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
         const uint32_t qb = it % C::kQBufs;
         ok = ws_wait(&qempty_bar[qb], ((it / C::kQBufs) & 1u) ^ 1u, s_abort);
         if (!ok) break;
-        mbar_arrive_expect_tx(&qfull_bar[qb], C::kQTxBytes);
+        mbar_arrive_expect_tx(&qfull_bar[qb], C::kQTxBytes + (PASS == 2 ? (uint32_t)(M * 4) : 0u));
+        if (PASS == 2)     // the item's row normalisers ride on the same barrier; slot reuse distance is four items
+          bulk_load_1d(s_mrow + (it % kMrowSlots) * 256, p.mrow + (size_t)sh.unit * M, M * 4, &qfull_bar[qb]);
         const int qrow0 = (sh.b * p.n_q_heads + sh.g * p.group) * p.window;
 #pragma unroll
         for (int rep = 0; rep < C::kRep; ++rep)
@@ -349,17 +359,21 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
     const int etid = tid & (kEpiThreads - 1);                               // thread within the group = TMEM lane
     const uint32_t tmem_lane = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);   // this warp's quarter of the lanes
     constexpr int kEntries = M < 128 ? 128 : M;                             // statistics entries per item
-    uint32_t gt = 0;
+    uint32_t gt = 0, it = 0;
     ItemShape sh;
     bool ok = true;
-    for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
-      if (sh.n_tiles == 0) continue;
+    for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n, ++it) {
+      if (sh.n_tiles == 0) {
+        --it;                                      // empty items are not counted (same rule in every role)
+        continue;
+      }
       float m0 = -INFINITY, l0 = 0.f, m1 = -INFINITY, l1 = 0.f;   // second pair: row tid+128 when M == 256
       const int limit0 = sh.t - p.window + ((etid % M) % p.window);
       const int limit1 = sh.t - p.window + ((etid + 128) % p.window);
       const int col_begin = M < 128 ? (etid / M) * C::kColsPerThread : 0;
       float* u = p.u + (size_t)sh.g * p.total_tokens + sh.cu;
-      const float4* mrow4 = reinterpret_cast<const float4*>(p.mrow + (size_t)sh.unit * M);
+      // landed before the MMA warp issued the item's first tile, whose completion this group waits for below
+      const float4* mrow4 = reinterpret_cast<const float4*>(s_mrow + (it % kMrowSlots) * 256);
       for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
         const uint32_t ab = gt % kAccBufs;
         if (ab != group) continue;               // the other group's tile
@@ -402,7 +416,7 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
           auto add_chunk = [&](const float (&v)[32], int cc) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-              const float4 mr = __ldg(&mrow4[(cc + i) >> 2]);      // same address in every thread: a broadcast
+              const float4 mr = mrow4[(cc + i) >> 2];              // same address in every thread: a broadcast
               acc += fast_exp2(fmaf(v[i + 0], p.scale_log2, -mr.x)) + fast_exp2(fmaf(v[i + 1], p.scale_log2, -mr.y)) +
                      fast_exp2(fmaf(v[i + 2], p.scale_log2, -mr.z)) + fast_exp2(fmaf(v[i + 3], p.scale_log2, -mr.w));
             }
