@@ -471,30 +471,65 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           p.part_ml[((size_t)item * G + gid) * 2 + 1] = l_row;
         }
       }
-      __threadfence();
-      __syncwarp();
+      __syncwarp();                 // the lanes' partial results are ordered before lane 0's fence (cumulative)
       int last = 0;
-      if (lane == 0) last = (atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1) == nc - 1) ? 1 : 0;
+      if (lane == 0) {
+        __threadfence();
+        last = (atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1) == nc - 1) ? 1 : 0;
+      }
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
         __threadfence();
         const int first = p.unit_info[e].x + h * nc;
-        for (int idx = lane; idx < G * D; idx += 32) {
-          const int g = idx / D, dc = idx % D;
+        // Merge the unit's chunks by log-sum-exp.  Per query head: lanes reduce the chunk maxima and the
+        // denominator, then every lane owns D/32 output columns and sweeps the chunks with independent,
+        // coalesced loads (four chunks in flight).
+        constexpr int kCols = D / 32;
+        for (int g = 0; g < G; ++g) {
+          const float* ml = p.part_ml + ((size_t)first * G + g) * 2;     // chunk c at ml[c * G * 2]
+          const float* po = p.part_o + ((size_t)first * G + g) * D + lane * kCols;
           float mmax = -INFINITY;
-          for (int c = 0; c < nc; ++c) mmax = fmaxf(mmax, __ldcg(&p.part_ml[((size_t)(first + c) * G + g) * 2]));
-          float num = 0.f, den = 0.f;
+          for (int c = lane; c < nc; c += 32) mmax = fmaxf(mmax, __ldcg(&ml[(size_t)c * G * 2]));
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
+          float den = 0.f;
+          float acc[kCols];
+#pragma unroll
+          for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
           if (mmax > -INFINITY) {
-            for (int c = 0; c < nc; ++c) {
-              const size_t pi = (size_t)(first + c) * G + g;
-              const float a = fast_exp2(__ldcg(&p.part_ml[pi * 2]) - mmax);
-              num += a * __ldcg(&p.part_o[pi * D + dc]);
-              den += a * __ldcg(&p.part_ml[pi * 2 + 1]);
+            for (int c = lane; c < nc; c += 32)
+              den += fast_exp2(__ldcg(&ml[(size_t)c * G * 2]) - mmax) * __ldcg(&ml[(size_t)c * G * 2 + 1]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+            int c = 0;
+            for (; c + 4 <= nc; c += 4) {
+              float a[4], v[4][kCols];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                a[k] = __ldcg(&ml[(size_t)(c + k) * G * 2]);
+#pragma unroll
+                for (int j = 0; j < kCols; ++j) v[k][j] = __ldcg(&po[(size_t)(c + k) * G * D + j]);
+              }
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float w = fast_exp2(a[k] - mmax);
+#pragma unroll
+                for (int j = 0; j < kCols; ++j) acc[j] += w * v[k][j];
+              }
+            }
+            for (; c < nc; ++c) {
+              const float w = fast_exp2(__ldcg(&ml[(size_t)c * G * 2]) - mmax);
+#pragma unroll
+              for (int j = 0; j < kCols; ++j) acc[j] += w * __ldcg(&po[(size_t)c * G * D + j]);
             }
           }
           const size_t row = q_row0 + g;
-          p.out[row * D + dc] = __float2bfloat16_rn(den > 0.f ? num / den : 0.f);
-          if (dc == 0 && p.lse != nullptr)
+          const float inv = den > 0.f ? 1.f / den : 0.f;
+#pragma unroll
+          for (int j = 0; j < kCols; j += 2)
+            *reinterpret_cast<uint32_t*>(p.out + row * D + lane * kCols + j) =
+                pack_bf16(acc[j] * inv, acc[j + 1] * inv);
+          if (lane == 0 && p.lse != nullptr)
             p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
         }
         if (lane == 0) p.tickets[e * p.n_kv_heads + h] = 0;
