@@ -285,17 +285,42 @@ def main():
         for l in range(L):
             sess.select_layer(l, int(budgets[l]), k[l], v[l])
         e[3].record()
-        for s in range(n_dec):
-            q, kn, vn = dec[s]
-            if host is not None:
-                q.copy_(host["dec"][s][0], non_blocking=True)
-                kn.copy_(host["dec"][s][1], non_blocking=True)
-                vn.copy_(host["dec"][s][2], non_blocking=True)
-            if kernel_events:
-                xkv.profile_events(k_start[s], k_stop[s])
-            sess.decode(q, kn, vn)
-            if host is not None:
-                host["out"].copy_(sess.out, non_blocking=True)
+        if host is None:
+            for s in range(n_dec):
+                q, kn, vn = dec[s]
+                if kernel_events:
+                    xkv.profile_events(k_start[s], k_stop[s])
+                sess.decode(q, kn, vn)
+        else:
+            # host leg: the step's inputs come from pinned host memory and its output goes back, every decode
+            # step; the copies run on a second stream so that step s+1's inputs travel while step s computes
+            main, cs = torch.cuda.current_stream(), host["stream"]
+            h2d = [ev() for _ in range(n_dec)]
+            done = [ev() for _ in range(n_dec)]
+            d2h = [ev() for _ in range(n_dec)]
+
+            def upload(s):
+                with torch.cuda.stream(cs):
+                    for dst, src in zip(dec[s], host["dec"][s]):
+                        dst.copy_(src, non_blocking=True)
+                    h2d[s].record(cs)
+
+            cs.wait_stream(main)
+            upload(0)
+            for s in range(n_dec):
+                if s + 1 < n_dec:
+                    upload(s + 1)
+                main.wait_event(h2d[s])
+                if s >= 2:
+                    main.wait_event(d2h[s - 2])          # the output buffer of step s-2 has been read back
+                out_buf = host["out_dev"][s & 1]
+                sess.decode(*dec[s], out=out_buf)
+                done[s].record(main)
+                with torch.cuda.stream(cs):
+                    cs.wait_event(done[s])
+                    host["out"].copy_(out_buf, non_blocking=True)
+                    d2h[s].record(cs)
+            main.wait_stream(cs)
         e[4].record()
         xkv.profile_events(None, None)
         return e, budgets
@@ -366,7 +391,8 @@ def main():
             host = {"q_win": [t.cpu().pin_memory() for t in q_win], "k": [t.cpu().pin_memory() for t in k],
                     "v": [t.cpu().pin_memory() for t in v],
                     "dec": [tuple(x.cpu().pin_memory() for x in dec[s]) for s in range(n_dec)],
-                    "out": torch.empty(sess.out.shape, dtype=sess.out.dtype, pin_memory=True)}
+                    "out": torch.empty(sess.out.shape, dtype=sess.out.dtype, pin_memory=True),
+                    "out_dev": [sess.out, torch.empty_like(sess.out)], "stream": torch.cuda.Stream()}
             h2d = sum(t.numel() * 2 for t in q_win + k + v) + sum(x.numel() * 2 for s in range(n_dec) for x in dec[s])
             d2h = sess.out.numel() * 2 * n_dec + sess.gains.numel() * 4
             step(host=host)
@@ -380,8 +406,9 @@ def main():
                    "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                    "ms_per_step": e_step_ms,
                    "note": "value: decode phase with q/k_new/v_new copied from pinned host memory and the output "
-                           "copied back every decode step; ms_per_step: the whole pass including the host-to-device "
-                           "copy of every layer's Q_win, K and V"}
+                           "copied back every decode step (copies on a second stream, overlapping the previous/next "
+                           "step's compute); ms_per_step: the whole pass including the host-to-device copy of every "
+                           "layer's Q_win, K and V"}
             del host
         except RuntimeError as err:                                  # e.g. pinned allocation refused
             e2e = {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,

@@ -481,57 +481,86 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       if (last) {
         __threadfence();
         const int first = p.unit_info[e].x + h * nc;
-        // Merge the unit's chunks by log-sum-exp.  Per query head: lanes reduce the chunk maxima and the
-        // denominator, then every lane owns D/32 output columns and sweeps the chunks with independent,
-        // coalesced loads (four chunks in flight).
+        // Merge the unit's chunks by log-sum-exp, 32 chunks at a time: lane c loads the (max, sum) of chunk c
+        // for every head at once, the weights exp2(m_c - max) stay in its registers and are handed out by
+        // shuffles, and every lane owns D/32 output columns of every head, so all loads of a step are
+        // independent of each other.
         constexpr int kCols = D / 32;
-        for (int g = 0; g < G; ++g) {
-          const float* ml = p.part_ml + ((size_t)first * G + g) * 2;     // chunk c at ml[c * G * 2]
-          const float* po = p.part_o + ((size_t)first * G + g) * D + lane * kCols;
-          float mmax = -INFINITY;
-          for (int c = lane; c < nc; c += 32) mmax = fmaxf(mmax, __ldcg(&ml[(size_t)c * G * 2]));
+        float mrun[kMaxGroup], den[kMaxGroup], acc[kMaxGroup][kCols];
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) mmax = fmaxf(mmax, __shfl_xor_sync(0xffffffffu, mmax, o));
-          float den = 0.f;
-          float acc[kCols];
+        for (int g = 0; g < kMaxGroup; ++g) {
+          mrun[g] = -INFINITY;
+          den[g] = 0.f;
 #pragma unroll
-          for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
-          if (mmax > -INFINITY) {
-            for (int c = lane; c < nc; c += 32)
-              den += fast_exp2(__ldcg(&ml[(size_t)c * G * 2]) - mmax) * __ldcg(&ml[(size_t)c * G * 2 + 1]);
+          for (int j = 0; j < kCols; ++j) acc[g][j] = 0.f;
+        }
+        for (int c0 = 0; c0 < nc; c0 += 32) {
+          const int c = c0 + lane;
+          float wgt[kMaxGroup];
+          float2 ml[kMaxGroup];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-            int c = 0;
-            for (; c + 4 <= nc; c += 4) {
-              float a[4], v[4][kCols];
+          for (int g = 0; g < kMaxGroup; ++g) {
+            ml[g] = make_float2(-INFINITY, 0.f);
+            if (g < G && c < nc)
+              ml[g] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(first + c) * G + g) * 2));
+          }
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                a[k] = __ldcg(&ml[(size_t)(c + k) * G * 2]);
+          for (int g = 0; g < kMaxGroup; ++g) {
+            if (g < G) {
+              float bm = ml[g].x;
 #pragma unroll
-                for (int j = 0; j < kCols; ++j) v[k][j] = __ldcg(&po[(size_t)(c + k) * G * D + j]);
-              }
+              for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+              const float m_new = fmaxf(mrun[g], bm);
+              const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+              const float rescale = fast_exp2(mrun[g] - m_ref);
+              wgt[g] = fast_exp2(ml[g].x - m_ref);
+              float ds = wgt[g] * ml[g].y;
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                const float w = fast_exp2(a[k] - mmax);
+              for (int o = 16; o > 0; o >>= 1) ds += __shfl_xor_sync(0xffffffffu, ds, o);
+              den[g] = den[g] * rescale + ds;
 #pragma unroll
-                for (int j = 0; j < kCols; ++j) acc[j] += w * v[k][j];
-              }
-            }
-            for (; c < nc; ++c) {
-              const float w = fast_exp2(__ldcg(&ml[(size_t)c * G * 2]) - mmax);
-#pragma unroll
-              for (int j = 0; j < kCols; ++j) acc[j] += w * __ldcg(&po[(size_t)c * G * D + j]);
+              for (int j = 0; j < kCols; ++j) acc[g][j] *= rescale;
+              mrun[g] = m_new;
             }
           }
-          const size_t row = q_row0 + g;
-          const float inv = den > 0.f ? 1.f / den : 0.f;
+          const int nb = min(32, nc - c0);
+          for (int cc = 0; cc < nb; cc += 2) {
+            float v[2][kMaxGroup][kCols];
 #pragma unroll
-          for (int j = 0; j < kCols; j += 2)
-            *reinterpret_cast<uint32_t*>(p.out + row * D + lane * kCols + j) =
-                pack_bf16(acc[j] * inv, acc[j + 1] * inv);
-          if (lane == 0 && p.lse != nullptr)
-            p.lse[row] = den > 0.f ? (mmax + log2f(den)) * 0.6931471805599453f : -INFINITY;
+            for (int k = 0; k < 2; ++k)
+#pragma unroll
+              for (int g = 0; g < kMaxGroup; ++g)
+#pragma unroll
+                for (int j = 0; j < kCols; ++j) {
+                  v[k][g][j] = 0.f;
+                  if (g < G && cc + k < nb)
+                    v[k][g][j] = __ldcg(&p.part_o[((size_t)(first + c0 + cc + k) * G + g) * D + lane * kCols + j]);
+                }
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+#pragma unroll
+              for (int g = 0; g < kMaxGroup; ++g)
+                if (g < G) {
+                  const float wk = __shfl_sync(0xffffffffu, wgt[g], (cc + k) & 31);
+                  if (cc + k < nb) {
+#pragma unroll
+                    for (int j = 0; j < kCols; ++j) acc[g][j] += wk * v[k][g][j];
+                  }
+                }
+          }
         }
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g)
+          if (g < G) {
+            const size_t row = q_row0 + g;
+            const float inv = den[g] > 0.f ? 1.f / den[g] : 0.f;
+#pragma unroll
+            for (int j = 0; j < kCols; j += 2)
+              *reinterpret_cast<uint32_t*>(p.out + row * D + lane * kCols + j) =
+                  pack_bf16(acc[g][j] * inv, acc[g][j + 1] * inv);
+            if (lane == 0 && p.lse != nullptr)
+              p.lse[row] = den[g] > 0.f ? (mrun[g] + log2f(den[g])) * 0.6931471805599453f : -INFINITY;
+          }
         if (lane == 0) p.tickets[e * p.n_kv_heads + h] = 0;
       }
     }

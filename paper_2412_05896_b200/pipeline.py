@@ -106,18 +106,17 @@ class XkvSession:
     def assign_pages(self, budgets) -> None:
         """Hand consecutive pool pages to every (layer, sequence) for its kept rows plus new tokens."""
         budgets = np.asarray(budgets)
+        k_lb = budgets.T if budgets.ndim == 2 else np.broadcast_to(budgets[:, None], (self.L, self.B))   # [L, B]
+        prefix = np.asarray(self.prefix)[None, :]
+        window = np.minimum(self.W, np.asarray(self.lengths))[None, :]
+        rows = np.minimum(k_lb, prefix) + window + self.max_new
+        n = np.minimum(-(-rows // self.page_size), self.max_pages_per_seq).astype(np.int64)               # pages
+        start = np.concatenate([[0], np.cumsum(n.ravel())[:-1]]).reshape(self.L, self.B)
+        if int(start.ravel()[-1] + n.ravel()[-1]) > self.n_pages:
+            raise RuntimeError("page pool too small for these budgets")
+        idx = np.arange(self.max_pages_per_seq, dtype=np.int64)[None, None, :]
         bt = self.block_table_host.numpy()
-        bt[:] = 0
-        nxt = 0
-        for l in range(self.L):
-            for b in range(self.B):
-                k_lb = int(budgets[b, l]) if budgets.ndim == 2 else int(budgets[l])
-                rows = min(k_lb, self.prefix[b]) + min(self.W, self.lengths[b]) + self.max_new
-                n = min(math.ceil(rows / self.page_size), self.max_pages_per_seq)
-                if nxt + n > self.n_pages:
-                    raise RuntimeError("page pool too small for these budgets")
-                bt[l, b, :n] = np.arange(nxt, nxt + n, dtype=np.int32)
-                nxt += n
+        bt[:] = np.where(idx < n[:, :, None], start[:, :, None] + idx, 0).astype(np.int32)
         self.block_table.copy_(self.block_table_host, non_blocking=True)
 
     def select_layer(self, layer: int, budget, k: torch.Tensor, v: torch.Tensor, sel: torch.Tensor | None = None,
