@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--chunk-rows", type=int, default=0, help="decode chunk size (0 = chosen on the device)")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -241,7 +242,7 @@ def main():
     N_total = None if w.budgets is not None else L * w.avg_budget
     sess = XkvSession(L, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
                       max_new_tokens=n_dec, max_budget=w.n_max or None, total_budget=N_total,
-                      curve_len=w.n_max or None, device=dev)
+                      curve_len=w.n_max or None, device=dev, decode_chunk_rows=args.chunk_rows)
     prefix = sess.prefix
 
     ev = lambda: torch.cuda.Event(enable_timing=True)

@@ -19,7 +19,9 @@ struct WorkspaceHeader {
   int32_t chunk_rows;  // decode: rows per chunk chosen by the plan
   int32_t work_counter;  // decode: next work item to hand to a warp
   int32_t prep_ticket;   // decode: CTAs of the prepare kernel that have finished
-  int32_t reserved[59];
+  int32_t n_multi;       // decode: (layer, sequence) units cut into more than one chunk
+  int32_t merge_counter; // decode: next split-K merge job to hand to a warp
+  int32_t reserved[57];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 
@@ -143,6 +145,13 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// Transposes an 8x8 matrix of 16-bit elements held one row pair per lane (lane = 4*row + column/2).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
 }
 
 // cp.async 16-byte copy global -> shared (zero-fills when src_bytes < 16).

@@ -11,11 +11,19 @@
 //                          ring of shared-memory stages: 16-row TMA tensor boxes (128-byte swizzle)
 //                          that complete on an mbarrier, issued by the warp itself a few tiles ahead
 //                          of where it computes, across item boundaries.  Per tile it runs online
-//                          softmax with mma.sync m16n8k16 for q.K^T and P.V (the G query heads of the
-//                          group sit on the M axis).  A unit with one chunk is normalised and stored by
-//                          its warp; otherwise partial (m, l, acc) go to the workspace and the last
-//                          warp to finish a chunk of the unit merges them by log-sum-exp (atomic
-//                          ticket, no waiting).
+//                          softmax with mma.sync m16n8k16, transposed: S^T = K.Q^T and O^T = V^T.P^T,
+//                          the 16 keys on the M axis and the G <= 8 query heads of the group on the N
+//                          axis, so no accumulator row is padding.  The softmax reference maximum is
+//                          raised lazily (only when a score exceeds it by 2^8), which keeps the
+//                          cross-lane reduction and the rescale out of the steady state; the scores of
+//                          the next tile are computed before the softmax of the current one.  A unit
+//                          with one chunk is normalised and stored by its warp; otherwise the chunk's
+//                          partial (m, l, acc) go to the workspace and a ticket counts the unit's
+//                          published chunks.  When the work items have run out, the warps share out
+//                          the split units one query head at a time (second counter) and merge the
+//                          chunks by log-sum-exp, all loads of a merge in flight together; by then
+//                          most of the streaming is over, so the merges neither queue behind it nor
+//                          run one after another in a single warp.
 // The path is HBM-bound: 4*d bytes per cached row per KV head per step; warps never wait for each
 // other, so item boundaries of one warp overlap with streaming in the others.
 #include <cuda.h>
@@ -57,6 +65,7 @@ struct DecodeParams {
   WorkspaceHeader* hdr;
   int32_t* tickets;   // [n_layers*batch*n_kv_heads]
   int2* unit_info;    // [n_layers*batch]: {first item of head 0, chunks per head}
+  int32_t* multi_list;  // [n_layers*batch]: the (layer, sequence) units that were cut into several chunks
   int4* items;        // [max_items]: {unit e, kv head, row_begin, row_end}
   float* part_o;      // [max_items][G][D]
   float* part_ml;     // [max_items][G][2]
@@ -82,6 +91,7 @@ __device__ void plan_items(const DecodeParams& p) {
   __shared__ int s_scan[32];
   __shared__ int s_carry;
   __shared__ int s_chunk;
+  __shared__ int s_multi;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n_warps = blockDim.x >> 5;
   const int n_units = p.n_layers * p.batch;
@@ -108,6 +118,7 @@ __device__ void plan_items(const DecodeParams& p) {
     }
     s_chunk = chunk;
     s_carry = 0;
+    s_multi = 0;
     p.hdr->chunk_rows = chunk;
   }
   __syncthreads();
@@ -139,6 +150,7 @@ __device__ void plan_items(const DecodeParams& p) {
     __syncthreads();
     const int carry = s_carry;
     const int excl = carry + s_scan[warp] + incl - nc;
+    if (e < n_units && nc > 1) p.multi_list[atomicAdd(&s_multi, 1)] = e;
     if (e < n_units) {
       const int first = excl * p.n_kv_heads;
       p.unit_info[e] = make_int2(first, nc);
@@ -160,8 +172,10 @@ __device__ void plan_items(const DecodeParams& p) {
     if (n_items > p.max_items) {
       record_status(p.hdr, XKV_ERR_WORKSPACE);
       p.hdr->n_items = 0;
+      p.hdr->n_multi = 0;
     } else {
       p.hdr->n_items = n_items;
+      p.hdr->n_multi = s_multi;
     }
   }
 }
@@ -219,6 +233,12 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* ptr) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
 // Bounded wait: two seconds of wall time at most.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
   for (int i = 0; i < 128; ++i)
@@ -253,6 +273,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   __syncthreads();
 
   const int n_items = p.hdr->n_items;
+  const int n_multi = p.hdr->n_multi;
   const int gid = lane >> 2, tig = lane & 3;
   const int mat = lane >> 3, mrow = lane & 7;
   const int G = p.group;
@@ -322,7 +343,28 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
   };
 
-  // ---- consumer side
+  // ---- consumer side.  Everything is computed transposed, keys on the M axis of the tensor-core tile and the
+  // (at most eight) query heads of the group on its N axis: S^T = K.Q^T is one m16n8 accumulator per 16-row
+  // tile, and O^T = V^T.P^T needs D/16 of them, so no accumulator row is padding.  In every fragment a lane
+  // then owns the two heads 2*tig, 2*tig+1.
+  const uint32_t k_lane_off = (uint32_t)(((mat & 1) * 8 + mrow) * 128 + ((((mat >> 1) & 1) ^ mrow) << 4));
+  const uint32_t v_lane_off = (uint32_t)(((mat >> 1) * 8 + mrow) * 128 + (((mat & 1) ^ mrow) << 4));
+  constexpr int kRegs = D / 4;        // accumulator registers per lane
+  constexpr float kLazy = 8.f;        // the reference maximum is raised only when a score exceeds it by 2^8
+
+  // waits for the tile with sequence number idx (bounded); flags the warp as aborted on failure
+  auto wait_tile = [&](uint32_t idx) {
+    if (aborted) return;
+    const int s = idx % C::kStages;
+    const uint32_t ph = (idx / C::kStages) & 1u;
+    const bool ok = ((int32_t)(issued - idx) > 0) && mbar_wait_bounded(&full_bar[s], ph);
+    if (!__all_sync(0xffffffffu, ok)) {
+      aborted = true;
+      no_more = true;
+      if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+    }
+  };
+
   while (true) {
     fill();
     if (fifo_count == 0) break;
@@ -335,40 +377,62 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int nc = p.unit_info[e].y;
     const size_t q_row0 = ((size_t)e * p.n_q_heads + (size_t)h * G);
 
-    uint32_t qa[D / 16][2];
+    // Q^T as the B operand: lane (gid, tig) holds head gid, columns 16*ks + 2*tig (+1) and + 8
+    uint32_t qb[D / 16][2];
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
-      qa[ks][0] = 0u;
-      qa[ks][1] = 0u;
+      qb[ks][0] = 0u;
+      qb[ks][1] = 0u;
       if (gid < G) {
         const __nv_bfloat16* qp = p.q + (q_row0 + gid) * D + 16 * ks + 2 * tig;
-        qa[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
-        qa[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
+        qb[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
+        qb[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
       }
     }
-    float o[D / 8][2];
+    float o[D / 16][4];               // O^T: [mt] = columns 16*mt + gid (regs 0,1) and + 8 (regs 2,3); heads 2*tig, +1
 #pragma unroll
-    for (int nt = 0; nt < D / 8; ++nt) o[nt][0] = o[nt][1] = 0.f;
-    float m_run = -INFINITY, l_part = 0.f;
+    for (int mt = 0; mt < D / 16; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    float m_ref[2] = {-3.0e38f, -3.0e38f};   // finite, so that (-inf) - m_ref stays -inf
+    float l_part[2] = {0.f, 0.f};
 
-    for (int r0 = I.z; r0 < I.w; r0 += kTileRows) {
-      if (issued == consumed) fill();
-      const int s = consumed % C::kStages;
-      const uint32_t ph = (consumed / C::kStages) & 1u;
-      if (!aborted) {
-        const bool ok = (issued != consumed) && mbar_wait_bounded(&full_bar[s], ph);
-        if (!__all_sync(0xffffffffu, ok)) {
-          aborted = true;
-          no_more = true;
-          if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
-        }
+    // S^T of one 16-row tile: rows gid (regs 0,1) and gid + 8 (regs 2,3), heads 2*tig, 2*tig + 1
+    auto qk_tile = [&](uint32_t idx, float (&acc)[4]) {
+      const uint32_t ks_base = smem_u32(ring + (size_t)(idx % C::kStages) * C::kStageBytes);
+      float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) {
+        uint32_t af[4];
+        ldmatrix_x4(af, ks_base + (ks >> 2) * C::kBoxBytes + (k_lane_off ^ (uint32_t)(((2 * ks) & 7) << 4)));
+        if (ks & 1) mma_bf16_16816(a1, af, qb[ks][0], qb[ks][1]);
+        else        mma_bf16_16816(a0, af, qb[ks][0], qb[ks][1]);
       }
-      const int wrows = min(kTileRows, I.w - r0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[i] = a0[i] + a1[i];
+    };
+
+    const int n_tiles = (I.w - I.z + kTileRows - 1) / kTileRows;
+    float s_next[4] = {0.f, 0.f, 0.f, 0.f};
+    if (n_tiles > 0) {
+      wait_tile(consumed);
+      if (!aborted) qk_tile(consumed, s_next);
+    }
+    for (int t = 0; t < n_tiles; ++t) {
+      float sv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) sv[i] = s_next[i] * p.scale_log2;
+      const int s = consumed % C::kStages;
+      const int wrows = min(kTileRows, I.w - (I.z + t * kTileRows));
+      if (t + 1 < n_tiles) {          // the next tile's scores do not depend on this tile's softmax
+        wait_tile(consumed + 1);
+        if (!aborted) qk_tile(consumed + 1, s_next);
+      }
       if (!aborted) {
-        const uint32_t ks_base = smem_u32(ring + (size_t)s * C::kStageBytes);
-        const uint32_t vs_base = ks_base + C::kTileBytes;
+        const uint32_t vs_base = smem_u32(ring + (size_t)s * C::kStageBytes) + C::kTileBytes;
         if (wrows < kTileRows) {
-          // rows past the end of the cache hold whatever the page held: clear V so 0 * x stays 0
+          // rows past the end of the cache hold whatever the page held: mask their scores and clear V so
+          // that 0 * x stays 0
+          if (gid >= wrows) sv[0] = sv[1] = -INFINITY;
+          if (gid + 8 >= wrows) sv[2] = sv[3] = -INFINITY;
           uint8_t* vs = ring + (size_t)s * C::kStageBytes + C::kTileBytes;
           const int n_bad = kTileRows - wrows;
           for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
@@ -380,65 +444,40 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           fence_proxy_async_smem();
           __syncwarp();
         }
-        // S[heads x 16 keys] = Q K^T
-        float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        float mx0 = fmaxf(sv[0], sv[2]), mx1 = fmaxf(sv[1], sv[3]);
+        const bool grow = (mx0 > m_ref[0] + kLazy) || (mx1 > m_ref[1] + kLazy);
+        if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const int key = (mat >> 1) * 8 + mrow;
-          const int c = 2 * ks + (mat & 1);
-          const uint32_t addr = ks_base + (c >> 3) * C::kBoxBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
-          uint32_t bfrag[4];
-          ldmatrix_x4(bfrag, addr);
-          const uint32_t a[4] = {qa[ks][0], 0u, qa[ks][1], 0u};
-          mma_bf16_16816(sacc[0], a, bfrag[0], bfrag[1]);
-          mma_bf16_16816(sacc[1], a, bfrag[2], bfrag[3]);
-        }
-        float s2[2][2];
-        float mt = -INFINITY;
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const bool in = (8 * nt + 2 * tig + j) < wrows;
-            s2[nt][j] = in ? sacc[nt][j] * p.scale_log2 : -INFINITY;
-            mt = fmaxf(mt, s2[nt][j]);
+          for (int x = 4; x < 32; x <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, x));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, x));
           }
-        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
-        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
-        const float m_new = fmaxf(m_run, mt);
-        const float alpha = fast_exp2(m_run - m_new);
-        float pr[2][2];
-        float psum = 0.f;
+          const float n0 = fmaxf(m_ref[0], mx0), n1 = fmaxf(m_ref[1], mx1);
+          const float al0 = fast_exp2(m_ref[0] - n0), al1 = fast_exp2(m_ref[1] - n1);
+          m_ref[0] = n0;
+          m_ref[1] = n1;
+          l_part[0] *= al0;
+          l_part[1] *= al1;
 #pragma unroll
-        for (int nt = 0; nt < 2; ++nt)
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            pr[nt][j] = fast_exp2(s2[nt][j] - m_new);
-            psum += pr[nt][j];
+          for (int mt = 0; mt < D / 16; ++mt) {
+            o[mt][0] *= al0;
+            o[mt][1] *= al1;
+            o[mt][2] *= al0;
+            o[mt][3] *= al1;
           }
-        l_part = l_part * alpha + psum;
-        m_run = m_new;
-#pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt) {
-          o[nt][0] *= alpha;
-          o[nt][1] *= alpha;
         }
-        const uint32_t pa[4] = {pack_bf16(pr[0][0], pr[0][1]), 0u, pack_bf16(pr[1][0], pr[1][1]), 0u};
+        const float p0 = fast_exp2(sv[0] - m_ref[0]), p1 = fast_exp2(sv[1] - m_ref[1]);
+        const float p2 = fast_exp2(sv[2] - m_ref[0]), p3 = fast_exp2(sv[3] - m_ref[1]);
+        l_part[0] += p0 + p2;
+        l_part[1] += p1 + p3;
+        // P^T as the B operand of O^T += V^T.P^T: transpose the two 8x8 blocks of the accumulator layout
+        const uint32_t b0 = movmatrix_trans(pack_bf16(p0, p1));
+        const uint32_t b1 = movmatrix_trans(pack_bf16(p2, p3));
 #pragma unroll
-        for (int dp = 0; dp < D / 16; ++dp) {
-          const int key = (mat & 1) * 8 + mrow;
-          const int c = 2 * dp + (mat >> 1);
-          const uint32_t addr = vs_base + (c >> 3) * C::kBoxBytes + key * 128 + (((c & 7) ^ (key & 7)) << 4);
-          uint32_t bfrag[4];
-          ldmatrix_x4_trans(bfrag, addr);
-          float c0[4] = {o[2 * dp][0], o[2 * dp][1], 0.f, 0.f};
-          float c1[4] = {o[2 * dp + 1][0], o[2 * dp + 1][1], 0.f, 0.f};
-          mma_bf16_16816(c0, pa, bfrag[0], bfrag[1]);
-          mma_bf16_16816(c1, pa, bfrag[2], bfrag[3]);
-          o[2 * dp][0] = c0[0];
-          o[2 * dp][1] = c0[1];
-          o[2 * dp + 1][0] = c1[0];
-          o[2 * dp + 1][1] = c1[1];
+        for (int mt = 0; mt < D / 16; ++mt) {
+          uint32_t af[4];
+          ldmatrix_x4_trans(af, vs_base + (mt >> 2) * C::kBoxBytes + (v_lane_off ^ (uint32_t)(((2 * mt) & 7) << 4)));
+          mma_bf16_16816(o[mt], af, b0, b1);
         }
       }
       __syncwarp();
@@ -446,124 +485,153 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       fill();                                   // the stage just released takes the next tile
     }
 
-    // ---- finish the work item
-    float l_row = l_part;
-    l_row += __shfl_xor_sync(0xffffffffu, l_row, 1);
-    l_row += __shfl_xor_sync(0xffffffffu, l_row, 2);
-    if (nc == 1) {
-      if (gid < G) {
-        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
-        __nv_bfloat16* orow = p.out + (q_row0 + gid) * D;
+    // ---- finish the work item: denominators of the lane's two heads over all rows
 #pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt)
-          *reinterpret_cast<uint32_t*>(orow + 8 * nt + 2 * tig) = pack_bf16(o[nt][0] * inv, o[nt][1] * inv);
-        if (tig == 0 && p.lse != nullptr)
-          p.lse[q_row0 + gid] = l_row > 0.f ? (m_run + log2f(l_row)) * 0.6931471805599453f : -INFINITY;
-      }
-    } else {
-      if (gid < G) {
-        float* po = p.part_o + ((size_t)item * G + gid) * D;
+    for (int x = 4; x < 32; x <<= 1) {
+      l_part[0] += __shfl_xor_sync(0xffffffffu, l_part[0], x);
+      l_part[1] += __shfl_xor_sync(0xffffffffu, l_part[1], x);
+    }
+    // normalises an accumulator in fragment layout and stores it as bf16 rows of the output
+    auto store_out = [&](float (&acc)[D / 16][4], const float (&den)[2], const float (&mx)[2]) {
+      const float inv0 = den[0] > 0.f ? 1.f / den[0] : 0.f;
+      const float inv1 = den[1] > 0.f ? 1.f / den[1] : 0.f;
+      __nv_bfloat16* orow = p.out + (q_row0 + gid) * D;
 #pragma unroll
-        for (int nt = 0; nt < D / 8; ++nt)
-          *reinterpret_cast<float2*>(po + 8 * nt + 2 * tig) = make_float2(o[nt][0], o[nt][1]);
-        if (tig == 0) {
-          p.part_ml[((size_t)item * G + gid) * 2 + 0] = m_run;
-          p.part_ml[((size_t)item * G + gid) * 2 + 1] = l_row;
+      for (int mt = 0; mt < D / 16; ++mt) {
+        // after the transpose the lane holds head gid, columns 16*mt + 2*tig (+1), then the same + 8
+        const uint32_t u0 = movmatrix_trans(pack_bf16(acc[mt][0] * inv0, acc[mt][1] * inv1));
+        const uint32_t u1 = movmatrix_trans(pack_bf16(acc[mt][2] * inv0, acc[mt][3] * inv1));
+        if (gid < G) {
+          *reinterpret_cast<uint32_t*>(orow + 16 * mt + 2 * tig) = u0;
+          *reinterpret_cast<uint32_t*>(orow + 16 * mt + 8 + 2 * tig) = u1;
         }
+      }
+      if (gid == 0 && p.lse != nullptr) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+          if (2 * tig + hh < G)
+            p.lse[q_row0 + 2 * tig + hh] =
+                den[hh] > 0.f ? (mx[hh] + log2f(den[hh])) * 0.6931471805599453f : -INFINITY;
+      }
+    };
+
+    if (nc == 1) {
+      store_out(o, l_part, m_ref);
+    } else {
+      // partial results of this chunk: [item][head][D] accumulators and [item][head] (max, sum)
+#pragma unroll
+      for (int mt = 0; mt < D / 16; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int head = 2 * tig + (i & 1);
+          if (head < G) p.part_o[((size_t)item * G + head) * D + 16 * mt + gid + 8 * (i >> 1)] = o[mt][i];
+        }
+      if (gid == 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+          if (2 * tig + hh < G)
+            *reinterpret_cast<float2*>(p.part_ml + ((size_t)item * G + 2 * tig + hh) * 2) =
+                make_float2(m_ref[hh], l_part[hh]);
       }
       __syncwarp();                 // the lanes' partial results are ordered before lane 0's fence (cumulative)
-      int last = 0;
       if (lane == 0) {
         __threadfence();
-        last = (atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1) == nc - 1) ? 1 : 0;
-      }
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        __threadfence();
-        const int first = p.unit_info[e].x + h * nc;
-        // Merge the unit's chunks by log-sum-exp, 32 chunks at a time: lane c loads the (max, sum) of chunk c
-        // for every head at once, the weights exp2(m_c - max) stay in its registers and are handed out by
-        // shuffles, and every lane owns D/32 output columns of every head, so all loads of a step are
-        // independent of each other.
-        constexpr int kCols = D / 32;
-        float mrun[kMaxGroup], den[kMaxGroup], acc[kMaxGroup][kCols];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-          mrun[g] = -INFINITY;
-          den[g] = 0.f;
-#pragma unroll
-          for (int j = 0; j < kCols; ++j) acc[g][j] = 0.f;
-        }
-        for (int c0 = 0; c0 < nc; c0 += 32) {
-          const int c = c0 + lane;
-          float wgt[kMaxGroup];
-          float2 ml[kMaxGroup];
-#pragma unroll
-          for (int g = 0; g < kMaxGroup; ++g) {
-            ml[g] = make_float2(-INFINITY, 0.f);
-            if (g < G && c < nc)
-              ml[g] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(first + c) * G + g) * 2));
-          }
-#pragma unroll
-          for (int g = 0; g < kMaxGroup; ++g) {
-            if (g < G) {
-              float bm = ml[g].x;
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
-              const float m_new = fmaxf(mrun[g], bm);
-              const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-              const float rescale = fast_exp2(mrun[g] - m_ref);
-              wgt[g] = fast_exp2(ml[g].x - m_ref);
-              float ds = wgt[g] * ml[g].y;
-#pragma unroll
-              for (int o = 16; o > 0; o >>= 1) ds += __shfl_xor_sync(0xffffffffu, ds, o);
-              den[g] = den[g] * rescale + ds;
-#pragma unroll
-              for (int j = 0; j < kCols; ++j) acc[g][j] *= rescale;
-              mrun[g] = m_new;
-            }
-          }
-          const int nb = min(32, nc - c0);
-          for (int cc = 0; cc < nb; cc += 2) {
-            float v[2][kMaxGroup][kCols];
-#pragma unroll
-            for (int k = 0; k < 2; ++k)
-#pragma unroll
-              for (int g = 0; g < kMaxGroup; ++g)
-#pragma unroll
-                for (int j = 0; j < kCols; ++j) {
-                  v[k][g][j] = 0.f;
-                  if (g < G && cc + k < nb)
-                    v[k][g][j] = __ldcg(&p.part_o[((size_t)(first + c0 + cc + k) * G + g) * D + lane * kCols + j]);
-                }
-#pragma unroll
-            for (int k = 0; k < 2; ++k)
-#pragma unroll
-              for (int g = 0; g < kMaxGroup; ++g)
-                if (g < G) {
-                  const float wk = __shfl_sync(0xffffffffu, wgt[g], (cc + k) & 31);
-                  if (cc + k < nb) {
-#pragma unroll
-                    for (int j = 0; j < kCols; ++j) acc[g][j] += wk * v[k][g][j];
-                  }
-                }
-          }
-        }
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g)
-          if (g < G) {
-            const size_t row = q_row0 + g;
-            const float inv = den[g] > 0.f ? 1.f / den[g] : 0.f;
-#pragma unroll
-            for (int j = 0; j < kCols; j += 2)
-              *reinterpret_cast<uint32_t*>(p.out + row * D + lane * kCols + j) =
-                  pack_bf16(acc[g][j] * inv, acc[g][j + 1] * inv);
-            if (lane == 0 && p.lse != nullptr)
-              p.lse[row] = den[g] > 0.f ? (mrun[g] + log2f(den[g])) * 0.6931471805599453f : -INFINITY;
-          }
-        if (lane == 0) p.tickets[e * p.n_kv_heads + h] = 0;
+        atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1);     // one more chunk of this unit is published
       }
     }
+  }
+
+  // ---- merge phase.  Once the work items have run out, the warps share out the units that were cut into several
+  // chunks, one query head at a time, and combine the chunks' partial results by log-sum-exp.  A job may find
+  // chunks of its unit still being computed: every such chunk is held by a warp that is still streaming (a warp
+  // comes here only after it has finished every item it took) and streaming warps wait for nothing but their own
+  // copies, so the bounded wait below ends.
+  constexpr int kCols = D / 32;
+  const int n_jobs = n_multi * p.n_kv_heads * G;
+  while (!aborted) {
+    int job = 0;
+    if (lane == 0) job = atomicAdd(&p.hdr->merge_counter, 1);
+    job = __shfl_sync(0xffffffffu, job, 0);
+    if (job >= n_jobs) break;
+    const int g = job % G, uh = job / G;
+    const int h = uh % p.n_kv_heads, e = p.multi_list[uh / p.n_kv_heads];
+    const int2 ui = p.unit_info[e];
+    const int nc = ui.y, first = ui.x + h * nc;
+    int ready = 1;
+    if (lane == 0) {
+      const int32_t* tk = &p.tickets[e * p.n_kv_heads + h];
+      if (ld_acquire_gpu(tk) < nc) {
+        const uint64_t t0 = global_timer_ns();
+        while (ld_acquire_gpu(tk) < nc) {
+          if (global_timer_ns() - t0 > 2000000000ull) {
+            ready = 0;
+            break;
+          }
+          __nanosleep(200);
+        }
+      }
+    }
+    ready = __shfl_sync(0xffffffffu, ready, 0);
+    if (!ready) {
+      if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+      break;
+    }
+    __threadfence();
+    float m_run = -3.0e38f, den = 0.f, acc[kCols];
+#pragma unroll
+    for (int j = 0; j < kCols; ++j) acc[j] = 0.f;
+    for (int c0 = 0; c0 < nc; c0 += 32) {
+      // lane c holds the weight of chunk c0 + c; the chunks' rows are then read sixteen at a time
+      const int c = c0 + lane;
+      float2 ml = make_float2(-3.0e38f, 0.f);
+      if (c < nc) ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(first + c) * G + g) * 2));
+      float bm = ml.x;
+#pragma unroll
+      for (int x = 16; x > 0; x >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, x));
+      const float m_new = fmaxf(m_run, bm);
+      const float rescale = fast_exp2(m_run - m_new);
+      const float wgt = c < nc ? fast_exp2(ml.x - m_new) : 0.f;
+      float ds = wgt * ml.y;
+#pragma unroll
+      for (int x = 16; x > 0; x >>= 1) ds += __shfl_xor_sync(0xffffffffu, ds, x);
+      den = den * rescale + ds;
+      m_run = m_new;
+#pragma unroll
+      for (int j = 0; j < kCols; ++j) acc[j] *= rescale;
+      const int nb = min(32, nc - c0);
+      for (int cc = 0; cc < nb; cc += 16) {
+        float v[16][kCols];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const float* src = p.part_o + ((size_t)(first + c0 + cc + k) * G + g) * D + lane * kCols;
+          if (cc + k < nb) {
+            if constexpr (kCols == 4) {
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(src));
+              v[k][0] = t.x; v[k][1] = t.y; v[k][2] = t.z; v[k][3] = t.w;
+            } else {
+              const float2 t = __ldcg(reinterpret_cast<const float2*>(src));
+              v[k][0] = t.x; v[k][1] = t.y;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < kCols; ++j) v[k][j] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          const float wk = __shfl_sync(0xffffffffu, wgt, (cc + k) & 31);
+#pragma unroll
+          for (int j = 0; j < kCols; ++j) acc[j] += wk * v[k][j];
+        }
+      }
+    }
+    const size_t row = (size_t)e * p.n_q_heads + (size_t)h * G + g;
+    const float inv = den > 0.f ? 1.f / den : 0.f;
+#pragma unroll
+    for (int j = 0; j < kCols; j += 2)
+      *reinterpret_cast<uint32_t*>(p.out + row * D + lane * kCols + j) = pack_bf16(acc[j] * inv, acc[j + 1] * inv);
+    if (lane == 0 && p.lse != nullptr)
+      p.lse[row] = den > 0.f ? (m_run + log2f(den)) * 0.6931471805599453f : -INFINITY;
   }
   if (aborted) {
     // let copies already issued land before this CTA's shared memory can be handed on
@@ -604,7 +672,7 @@ bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows) {
 }
 
 struct DecodeLayout {
-  size_t tickets, unit_info, items, part_o, part_ml, total;
+  size_t tickets, unit_info, multi, items, part_o, part_ml, total;
   int64_t max_items;
 };
 
@@ -626,6 +694,7 @@ bool decode_layout(const xkv_dims* d, int n_layers, int max_cache_len, int chunk
   size_t off = kHeaderBytes;
   L->tickets = off;   off = align_up(off + (size_t)units * 4, 256);
   L->unit_info = off; off = align_up(off + (size_t)lb * 8, 256);
+  L->multi = off;     off = align_up(off + (size_t)lb * 4, 256);
   L->items = off;     off = align_up(off + (size_t)max_items * 16, 256);
   L->part_o = off;    off = align_up(off + (size_t)max_items * G * d->head_dim * 4, 256);
   L->part_ml = off;   off = align_up(off + (size_t)max_items * G * 2 * 4, 256);
@@ -716,6 +785,7 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   p.tickets = reinterpret_cast<int32_t*>(ws + L.tickets);
   p.unit_info = reinterpret_cast<int2*>(ws + L.unit_info);
+  p.multi_list = reinterpret_cast<int32_t*>(ws + L.multi);
   p.items = reinterpret_cast<int4*>(ws + L.items);
   p.part_o = reinterpret_cast<float*>(ws + L.part_o);
   p.part_ml = reinterpret_cast<float*>(ws + L.part_ml);
