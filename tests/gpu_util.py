@@ -30,7 +30,7 @@ class DirectCache:
     """A ragged paged cache filled by torch indexing (not by the library): K/V rows of every
     (layer, sequence) are scattered into randomly ordered pages."""
 
-    def __init__(self, L, B, Hkv, d, lens, page_size, extra_rows, device, seed=0, v_shift=0.0):
+    def __init__(self, L, B, Hkv, d, lens, page_size, extra_rows, device, seed=0, v_shift=0.0, k_rows=None):
         g = torch.Generator(device="cpu").manual_seed(seed)
         self.L, self.B, self.Hkv, self.d, self.page_size = L, B, Hkv, d, page_size
         self.lens = np.asarray(lens, dtype=np.int64).reshape(L, B)
@@ -47,6 +47,8 @@ class DirectCache:
             for b in range(B):
                 n = int(self.lens[l, b])
                 k = torch.randn(n, Hkv, d, generator=g).to(torch.bfloat16)
+                if k_rows is not None:                      # caller-made keys: k_rows(l, b, n) -> [n, Hkv, d]
+                    k = k_rows(l, b, n).to(torch.bfloat16)
                 v = (torch.randn(n, Hkv, d, generator=g) + v_shift).to(torch.bfloat16)
                 self.K[(l, b)], self.V[(l, b)] = k, v
                 if n == 0:

@@ -74,6 +74,53 @@ def test_decode_peaked_attention_and_shifted_values():
     _run_case(2, 2, 4, 4, 64, lens, 32, 256, True, seed=6, stress=True)
 
 
+@pytest.mark.parametrize("profile", ["ramp", "jumps", "falling", "late_peak"])
+def test_decode_score_profiles_along_the_cache(profile):
+    """Scores that rise slowly, jump, fall or peak at the very end along the cache: the running softmax
+    maximum is then raised often, rarely, never after the first tile, or once at the last row."""
+    require_lib()
+    L, B, Hq, Hkv, d, ps = 1, 3, 8, 2, 128, 16
+    lens = [[700, 333, 2049]]
+    gen = torch.Generator(device="cpu").manual_seed(77)
+    u = (torch.randint(0, 2, (Hkv, d), generator=gen) * 2 - 1).to(torch.float32)      # +-1: q.k = c * d exactly
+    unit = np.sqrt(d) * 1.4426950408889634                                            # log2-domain score per unit c
+
+    def k_rows(l, b, n):
+        j = torch.arange(n, dtype=torch.float32)
+        if profile == "ramp":
+            c = 60.0 / unit * j / max(n - 1, 1)                       # about +0.03 .. +0.2 per row, +60 overall
+        elif profile == "jumps":
+            c = 20.0 / unit * torch.floor(j / 97.0)                   # +20 every 97 rows
+        elif profile == "falling":
+            c = -40.0 / unit * j / max(n - 1, 1)
+        else:
+            c = torch.zeros(n)
+            c[-1] = 30.0 / unit                                        # one dominant row at the end
+        noise = 0.05 * torch.randn(n, Hkv, d, generator=gen)
+        return c[:, None, None] * u[None] + noise
+
+    cache = DirectCache(L, B, Hkv, d, lens, ps, extra_rows=1, device=DEV, seed=8, k_rows=k_rows)
+    dims = xkv.Dims(B, Hq, Hkv, d, 16, 1, 0, 0.0, Hkv * d, d)
+    G = Hq // Hkv
+    q = torch.stack([u[h // G] for h in range(Hq)])[None, None].repeat(L, B, 1, 1).to(torch.bfloat16)
+    for chunk_rows in (0, 128):
+        ws = torch.empty(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=cache.max_pages * ps,
+                                             chunk_rows=chunk_rows), dtype=torch.uint8, device=DEV)
+        out = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
+        lse = torch.empty(L, B, Hq, dtype=torch.float32, device=DEV)
+        xkv.decode_attn(dims, cache.handle(), 0, L, q.to(DEV), None, None, out, lse, chunk_rows, ws)
+        torch.cuda.synchronize()
+        assert xkv.read_device_status(ws) == xkv.OK
+        ref = np.zeros((L, B, Hq, d))
+        ref_lse = np.zeros((L, B, Hq))
+        for b in range(B):
+            K, V = f64(cache.K[(0, b)]), f64(cache.V[(0, b)])
+            for h in range(Hq):
+                ref[0, b, h], ref_lse[0, b, h] = O.decode_attention(f64(q[0, b, h]), K[:, h // G], V[:, h // G])
+        check_attention(out, ref, f"{profile} chunk {chunk_rows}", rel_l2=True)
+        assert np.allclose(lse.cpu().numpy().astype(np.float64), ref_lse, atol=2e-3, rtol=1e-4)
+
+
 def test_decode_many_units_long_chunks():
     rng = np.random.default_rng(3)
     lens = rng.integers(1, 900, size=(6, 16)).tolist()
