@@ -276,6 +276,7 @@ def main():
                 v[l].copy_(host["v"][l], non_blocking=True)
         for l in range(L):
             sess.score_layer(l, q_win[l], k[l])
+        sess.join()
         e[1].record()
         if w.budgets is not None:
             budgets = np.asarray(w.budgets, dtype=np.int32)
@@ -285,6 +286,7 @@ def main():
         e[2].record()
         for l in range(L):
             sess.select_layer(l, int(budgets[l]), k[l], v[l])
+        sess.join()
         e[3].record()
         if host is None:
             for s in range(n_dec):

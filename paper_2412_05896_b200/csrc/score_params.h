@@ -34,4 +34,9 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
 // Key split the tcgen05 variant uses (0 if it does not cover the shape).
 int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen);
 
+// Single-launch variant (xkv_score_fused.cu): both passes by thread-block clusters, the second one fed from L2.
+// Covers G*W in {32, 64, 128} while the keys of the units in flight fit in L2.
+bool score_fused_covers(int M, int head_dim, int units, int max_seqlen);
+xkv_status score_fused_pass(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st);
+
 }  // namespace xkv

@@ -349,7 +349,6 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   // then owns the two heads 2*tig, 2*tig+1.
   const uint32_t k_lane_off = (uint32_t)(((mat & 1) * 8 + mrow) * 128 + ((((mat >> 1) & 1) ^ mrow) << 4));
   const uint32_t v_lane_off = (uint32_t)(((mat >> 1) * 8 + mrow) * 128 + (((mat & 1) ^ mrow) << 4));
-  constexpr int kRegs = D / 4;        // accumulator registers per lane
   constexpr float kLazy = 8.f;        // the reference maximum is raised only when a score exceeds it by 2^8
 
   // waits for the tile with sequence number idx (bounded); flags the warp as aborted on failure

@@ -789,7 +789,9 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
 
   if (cudaMemsetAsync(ws, 0, L.u, st) != cudaSuccess) return XKV_ERR_CUDA;   // header, tickets, ready flags
   xkv_status s;
-  if (L.use_tc) {
+  if (L.use_tc && score_fused_covers(p.M, d->head_dim, units, max_seqlen)) {
+    s = score_fused_pass(p, d->head_dim, max_seqlen, st);      // both passes in one cluster kernel, keys read once
+  } else if (L.use_tc) {
     s = score_tc_passes(p, d->head_dim, max_seqlen, st);
   } else {
     s = d->head_dim == 128 ? launch_passes<128>(p, L, st) : launch_passes<64>(p, L, st);

@@ -14,127 +14,12 @@
 //           exp2(s*c - normaliser[row]) over the query rows straight out of TMEM -> column score u[key].
 //           Items are walked in reverse so that the keys pass 1 streamed last are re-read from L2.
 // No CTA ever waits for another one; every mbarrier wait is bounded.
-#include <cuda.h>
-
-#include <cmath>
-#include <mutex>
-
-#include "common.cuh"
-#include "score_params.h"
+#include "tc_common.cuh"
 
 namespace xkv {
 namespace {
 
-constexpr int kTcThreads = 128;
-constexpr int kTcKeyTile = 128;                 // keys per MMA tile
-
-// ---------------------------------------------------------------------------------------------
-// tcgen05 / TMEM wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(cols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before_sync() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after_sync() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, bf16 inputs, fp32 accumulate; issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
-      "}\n" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
-      : "memory");
-}
-// mbarrier arrives once all MMAs issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-// 32 consecutive fp32 columns of this thread's TMEM lane; the values may be used after tmem_wait_ld().
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor of a K-major operand stored as rows of 128 bytes (64 bf16) with the
-// 128-byte swizzle, eight-row groups 1024 bytes apart (what a TMA box {64, rows} with SWIZZLE_128B writes).
-__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);   // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                         // leading byte offset (unused with swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset: next eight-row group
-  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
-  return d;
-}
-
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t umma_idesc(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const void* tmap, int x, int y, int z, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-
-// Plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
-__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
-__device__ __forceinline__ uint64_t tc_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded mbarrier wait: two seconds at most.
-__device__ __forceinline__ bool tc_mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = tc_timer_ns();
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (tc_timer_ns() - t0 > 2000000000ull) return false;
-  }
-}
-__device__ __forceinline__ int tc_ld_acquire(const int* ptr) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
-  return v;
-}
+using namespace tc;
 
 // ---------------------------------------------------------------------------------------------
 // Kernel: warp-specialised pipeline
@@ -147,49 +32,6 @@ __device__ __forceinline__ int tc_ld_acquire(const int* ptr) {
 // Work items are assigned statically (item = CTA + n * grid), so each role walks the same sequence on its
 // own and the producer runs ahead across item boundaries.
 // ---------------------------------------------------------------------------------------------
-constexpr int kWsThreads = 320;
-constexpr int kEpiThreads = 128;     // threads of one epilogue group
-constexpr int kWsStages = 4;       // shared-memory ring of key tiles
-constexpr int kAccBufs = 2;        // TMEM accumulator buffers
-constexpr int kMrowSlots = 4;      // pass 2: ring of row-normaliser vectors (one per item in flight)
-
-template <int D, int M>
-struct TcCfg {
-  static constexpr int kHalves = D / 64;                         // 128-byte swizzled K segments per row
-  static constexpr int kSteps = D / 16;                          // MMA k-steps per tile
-  static constexpr int kQRows = M < 128 ? 128 : M;               // rows of the query operand buffer
-  static constexpr int kRep = M < 128 ? 128 / M : 1;             // replicas of the query rows across lanes
-  static constexpr int kQHalfBytes = kQRows * 128;
-  static constexpr int kQBytes = kHalves * kQHalfBytes;
-  static constexpr int kQBufs = M == 256 ? 1 : 2;
-  static constexpr int kKHalfBytes = kTcKeyTile * 128;
-  static constexpr int kKTileBytes = kHalves * kKHalfBytes;
-  static constexpr uint32_t kBufCols = M == 256 ? 256 : 128;     // TMEM columns of one accumulator buffer
-  static constexpr uint32_t kTmemCols = kAccBufs * kBufCols;
-  static constexpr int kColsPerThread = M < 128 ? M : 128;       // pass-1 key columns a thread reduces per tile
-  static constexpr uint32_t kQTxBytes = (uint32_t)(kRep * kHalves * (M < 128 ? M : kQRows) * 128);
-  static constexpr size_t kSmemBytes = 1024 + (size_t)kQBufs * kQBytes + (size_t)kWsStages * kKTileBytes +
-                                       kMrowSlots * 256 * 4 /*row normalisers*/ + 256 /*barriers*/;
-};
-
-__device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
-                                          float& m, float& l) {
-  float x[32];
-  float vmax = -INFINITY;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    x[i] = (masked && c0 + i > limit) ? -INFINITY : v[i];
-    vmax = fmaxf(vmax, x[i]);
-  }
-  const float m_new = fmaxf(m, vmax * scale);
-  const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-  float sum = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) sum += fast_exp2(fmaf(x[i], scale, -m_ref));
-  l = l * fast_exp2(m - m_ref) + sum;
-  m = m_new;
-}
-
 struct ItemShape {
   int unit, split, b, g, cu, t, P, key_begin, key_end, n_tiles;
 };
@@ -211,21 +53,6 @@ __device__ __forceinline__ bool item_shape(const ScoreParams& p, int n, ItemShap
   it->key_end = min(it->key_begin + p.split_keys, PASS == 1 ? it->t : it->P);
   it->n_tiles = it->key_end > it->key_begin ? (it->key_end - it->key_begin + kTcKeyTile - 1) / kTcKeyTile : 0;
   return true;
-}
-
-// Bounded mbarrier wait (two seconds) that also gives up when another role has raised the abort flag.
-__device__ __forceinline__ bool ws_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = tc_timer_ns();
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (tc_timer_ns() - t0 > 2000000000ull) {
-      *abort_flag = 1;
-      return false;
-    }
-  }
 }
 
 template <int D, int M, int PASS>
@@ -504,33 +331,6 @@ __global__ void __launch_bounds__(128) tc_merge_kernel(const ScoreParams p) {
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn tc_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  });
-  return fn;
-}
-
-bool tc_make_tmap(CUtensorMap* tmap, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides,
-                  const cuuint32_t* box) {
-  EncodeTiledFn enc = tc_encode_fn();
-  if (enc == nullptr) return false;
-  const cuuint32_t estr[3] = {1u, 1u, 1u};
-  return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides, box,
-             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Key tiles per work item: items are cheap (the producer prefetches across them), so keep them small
 // enough to balance the static assignment.
 int tc_tiles(int M, int head_dim, int units, int max_seqlen) {
@@ -591,18 +391,7 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
   const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen);
   if (tiles == 0 || tiles * kTcKeyTile != p.split_keys) return XKV_ERR_UNSUPPORTED;
   CUtensorMap tq, tk;
-  {
-    const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)p.batch * p.n_q_heads * p.window};
-    const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
-    const cuuint32_t box[2] = {64u, (cuuint32_t)p.M};
-    if (!tc_make_tmap(&tq, p.q_win, 2, dims, strides, box)) return XKV_ERR_CUDA;
-  }
-  {
-    const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)p.n_kv_heads, (cuuint64_t)p.total_tokens};
-    const cuuint64_t strides[2] = {(cuuint64_t)p.stride_head * 2, (cuuint64_t)p.stride_token * 2};
-    const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)kTcKeyTile};
-    if (!tc_make_tmap(&tk, p.k, 3, dims, strides, box)) return XKV_ERR_CUDA;
-  }
+  if (!tc_make_score_tmaps(p, head_dim, &tq, &tk)) return XKV_ERR_CUDA;
 #define XKV_TC_CASE(DD, MM) \
   if (head_dim == DD && p.M == MM) return tc_launch_both<DD, MM>(tq, tk, p, st);
   XKV_TC_CASE(128, 32) XKV_TC_CASE(128, 64) XKV_TC_CASE(128, 128) XKV_TC_CASE(128, 256)

@@ -20,7 +20,7 @@ class XkvSession:
                  pool_kernel: int, lengths: list[int], pool_mode: int = xkv.POOL_MAX, page_size: int = 16,
                  max_new_tokens: int = 0, max_budget: int | None = None, total_budget: int | None = None,
                  curve_len: int | None = None, device="cuda:0", scale: float = 0.0,
-                 decode_chunk_rows: int = 0):
+                 decode_chunk_rows: int = 0, n_lanes: int = 2):
         self.L, self.Hq, self.Hkv, self.d, self.W = n_layers, n_q_heads, n_kv_heads, head_dim, window
         self.B = len(lengths)
         self.lengths = list(lengths)
@@ -47,8 +47,17 @@ class XkvSession:
         self.sorted = torch.empty(n_layers, n_kv_heads, self.T, **f32)
         self.gains = torch.empty(n_layers, self.B, self.curve_len, **f32)
         self.gains_host = torch.empty(n_layers, self.B, self.curve_len, dtype=torch.float32, pin_memory=True)
-        self.ws_score = self._ws(xkv.workspace_bytes(xkv.OP_SCORE, self.dims, self.max_seqlen, self.T))
-        self.ws_select = self._ws(xkv.workspace_bytes(xkv.OP_SELECT_COMPACT, self.dims, self.max_seqlen, self.T))
+        # Layers are independent in the scoring and in the eviction phase, so consecutive layers go to
+        # n_lanes side streams, each with its own workspace: the short latency-bound kernels of one layer
+        # (sort, curves, selection) then run under the HBM-bound ones of the next.
+        self.n_lanes = max(1, n_lanes)
+        self.lanes = [torch.cuda.Stream(device=self.device) for _ in range(self.n_lanes)] if self.n_lanes > 1 else []
+        n_ws = max(1, self.n_lanes)
+        self.ws_score = [self._ws(xkv.workspace_bytes(xkv.OP_SCORE, self.dims, self.max_seqlen, self.T))
+                         for _ in range(n_ws)]
+        self.ws_select = [self._ws(xkv.workspace_bytes(xkv.OP_SELECT_COMPACT, self.dims, self.max_seqlen, self.T))
+                          for _ in range(n_ws)]
+        self._lanes_busy = False
 
         # ragged paged cache: a pool large enough for any split of the global budget
         per_layer_cap = min(max_budget if max_budget else self.max_prefix, self.max_prefix)
@@ -83,18 +92,41 @@ class XkvSession:
         self.r_avg: float | None = None
 
     def _ws(self, nbytes: int) -> torch.Tensor:
-        return torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        return torch.zeros(nbytes, dtype=torch.uint8, device=self.device)   # status word reads OK before first use
 
     # ------------------------------------------------------------------ prefill
+    def _lane(self, layer: int, *tensors):
+        """(stream, workspace index) of a layer; the side stream first waits for what the caller's stream holds,
+        and the caller's tensors are marked as in use on it (they may be temporaries)."""
+        if not self.lanes:
+            return torch.cuda.current_stream(), 0
+        i = layer % self.n_lanes
+        self.lanes[i].wait_stream(torch.cuda.current_stream())
+        for t in tensors:
+            if isinstance(t, torch.Tensor) and t.is_cuda:
+                t.record_stream(self.lanes[i])
+        self._lanes_busy = True
+        return self.lanes[i], i
+
+    def join(self) -> None:
+        """The caller's stream waits for the layers queued on the side streams."""
+        if self._lanes_busy:
+            cur = torch.cuda.current_stream()
+            for s in self.lanes:
+                cur.wait_stream(s)
+            self._lanes_busy = False
+
     def score_layer(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, want_curves: bool = True,
                     mass: torch.Tensor | None = None) -> None:
+        stream, i = self._lane(layer, q_win, k, mass)
         xkv.score(self.dims, q_win, k, self.cu, self.T, self.max_seqlen, self.scores[layer],
                   self.sorted[layer] if want_curves else None, self.gains[layer] if want_curves else None,
-                  mass, self.curve_len, self.ws_score)
+                  mass, self.curve_len, self.ws_score[i], stream=stream)
 
     def solve_budgets(self, total: int | None = None, r_target: float = 0.0, n_min: int = 0, n_max: int = 0,
                       per_sequence: bool = False):
         """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host."""
+        self.join()
         self.gains_host.copy_(self.gains, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         budgets, r_avg = xkv.alloc_budgets(self.gains_host.numpy(), np.asarray(self.prefix, dtype=np.int32),
@@ -121,9 +153,10 @@ class XkvSession:
 
     def select_layer(self, layer: int, budget, k: torch.Tensor, v: torch.Tensor, sel: torch.Tensor | None = None,
                      per_sequence: bool = False) -> None:
+        stream, i = self._lane(layer, k, v, sel)
         xkv.select_compact(self.dims, layer, budget, per_sequence, self.scores[layer], self.sorted[layer], k, v,
                            self.cu, self.T, self.max_seqlen, self.cache, sel,
-                           0 if sel is None else sel.shape[-1], self.ws_select)
+                           0 if sel is None else sel.shape[-1], self.ws_select[i], stream=stream)
 
     def prefill(self, q_win: list[torch.Tensor], k: list[torch.Tensor], v: list[torch.Tensor],
                 budgets=None, total: int | None = None, n_min: int = 0, n_max: int = 0):
@@ -137,12 +170,14 @@ class XkvSession:
         self.assign_pages(budgets)
         for l in range(self.L):
             self.select_layer(l, int(budgets[l]), k[l], v[l])
+        self.join()
         return budgets
 
     # ------------------------------------------------------------------ generation
     def decode(self, q: torch.Tensor, k_new: torch.Tensor | None, v_new: torch.Tensor | None,
                out: torch.Tensor | None = None, lse: torch.Tensor | None = None, layer_begin: int = 0,
                layer_end: int | None = None, chunk_rows: int | None = None) -> torch.Tensor:
+        self.join()
         out = self.out if out is None else out
         layer_end = self.L if layer_end is None else layer_end
         xkv.decode_attn(self.dims, self.cache, layer_begin, layer_end, q, k_new, v_new, out,
@@ -151,5 +186,10 @@ class XkvSession:
         return out
 
     def device_status(self, which: str = "decode") -> int:
-        ws = {"decode": self.ws_decode, "score": self.ws_score, "select": self.ws_select}[which]
-        return xkv.read_device_status(ws)
+        self.join()
+        ws = {"decode": [self.ws_decode], "score": self.ws_score, "select": self.ws_select}[which]
+        for w in ws:
+            st = xkv.read_device_status(w)
+            if st != xkv.OK:
+                return st
+        return xkv.OK
