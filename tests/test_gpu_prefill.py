@@ -65,6 +65,8 @@ CASES = [
     ([1500], 16, 4, 128, 64, 3, 0),              # G*W = 256 query rows
     ([9000, 4097], 2, 2, 128, 16, 7, 0),         # several sort chunks and merge passes
     ([33, 17, 16, 1], 2, 1, 64, 16, 1, 0),       # at and below the window length
+    ([8192, 4500, 130], 2, 2, 128, 32, 7, 0),    # G*W = 32, single-read kernel with clusters of eight
+    ([4096, 31, 32, 33, 160], 3, 3, 64, 32, 5, 1),   # G*W = 32, clusters of four, lengths around the window
 ]
 
 
@@ -87,6 +89,38 @@ def test_score_sort_and_curves(lengths, Hq, Hkv, d, W, ps, mode):
     for b, t in enumerate(lengths):
         if t > W:
             assert abs(got_mass[b, min(t - W, sess.curve_len) - 1] - 1.0) < 2e-5 or t - W > sess.curve_len
+
+
+@pytest.mark.parametrize("Hq,Hkv,W", [(2, 2, 32), (8, 2, 32), (4, 2, 8)])
+@pytest.mark.parametrize("profile", ["ramp", "jumps", "falling"])
+def test_scores_with_logit_profiles_along_the_keys_and_across_rows(profile, Hq, Hkv, W):
+    """Logits that rise, jump or fall along the key axis, with query rows of very different scale: the running
+    softmax reference of a row is then raised often, rarely or never, and the rows of one tile sit hundreds of
+    units apart (log2 domain)."""
+    require_lib()
+    d, ps, lengths = 128, 5, [3000, 777]
+    T = sum(lengths)
+    gen = torch.Generator(device="cpu").manual_seed(4242)
+    u = (torch.randint(0, 2, (Hkv, d), generator=gen) * 2 - 1).to(torch.float32)           # q.k = a * c * d exactly
+    unit = np.sqrt(d) * 1.4426950408889634                                                 # log2 units per a*c
+    pos = torch.cat([torch.arange(t, dtype=torch.float32) / max(t - 1, 1) for t in lengths])
+    if profile == "ramp":
+        c = 60.0 / unit * pos
+    elif profile == "jumps":
+        c = 15.0 / unit * torch.floor(pos * 7.0)
+    else:
+        c = -60.0 / unit * pos
+    k = c[:, None, None] * u[None] + 0.05 * torch.randn(T, Hkv, d, generator=gen)
+    a = 0.25 * (1.0 + torch.arange(W, dtype=torch.float32))                                # row scale 0.25 .. W/4
+    q = a[None, None, :, None] * u.repeat_interleave(Hq // Hkv, 0)[None, :, None, :] + \
+        0.05 * torch.randn(len(lengths), Hq, W, d, generator=gen)
+    q, k = q.to(torch.bfloat16), k.to(torch.bfloat16)
+    sess = XkvSession(1, Hq, Hkv, d, W, ps, lengths, device=DEV)
+    sess.score_layer(0, q.to(DEV), k.to(DEV))
+    torch.cuda.synchronize()
+    assert sess.device_status("score") == xkv.OK
+    w_ref = _oracle_scores(q, k, sess.cu_host, W, ps, 0)
+    _check_scores(sess, 0, w_ref, lengths, Hkv, W)
 
 
 def _cache_rows(sess, layer, b, g, n):
