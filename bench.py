@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--no-full-cache", action="store_true", help="skip the uncompressed-cache decode comparison")
     ap.add_argument("--chunk-rows", type=int, default=0, help="decode chunk size (0 = chosen on the device)")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
     args = ap.parse_args()
@@ -417,6 +418,44 @@ def main():
             e2e = {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                    "note": f"host leg failed: {str(err)[:120]}"}
 
+    # ---------------------------------------------------------------- full-cache decode, for comparison only
+    full_cache = None
+    if world == 1 and not args.no_full_cache:
+        per_layer = sum(-(-(t + n_dec + sess.page_size) // sess.page_size) * sess.page_size for t in lengths) \
+            * Hkv * d * 2 * 2                                            # K and V pages of one uncompressed layer
+        free_b, _ = torch.cuda.mem_get_info(dev)
+        n_full = int(min(L, (free_b - (4 << 30)) // max(per_layer, 1)))
+        if n_full >= 1:
+            full = XkvSession(n_full, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
+                              max_new_tokens=n_dec, device=dev)
+            keep_all = np.full(n_full, max(full.prefix), dtype=np.int32)
+            full.assign_pages(keep_all)
+            for l in range(n_full):
+                full.select_layer(l, int(keep_all[l]), k[l], v[l])      # budget = prefix length: nothing is evicted
+            full.join()
+            f0, f1 = ev(), ev()
+            n_warm, n_timed = 2, min(6, n_dec - 2)
+            for s in range(n_warm + n_timed):
+                if s == n_warm:
+                    f0.record()
+                q, kn, vn = dec[s]
+                full.decode(q[:n_full], kn[:n_full], vn[:n_full])
+            f1.record()
+            torch.cuda.synchronize()
+            if full.device_status("decode") != xkv.OK:
+                raise SystemExit("full-cache decode reported a device error")
+            f_ms = f0.elapsed_time(f1) / n_timed
+            f_bytes = sum(t + n_warm + (n_timed + 1) / 2 for t in lengths) * n_full * Hkv * 2 * d * 2
+            comp_ms = float(phase[:, 3].mean()) / n_dec
+            full_cache = {"layers_measured": n_full, "ms_per_decode_step_all_layers": f_ms * L / n_full,
+                          "GBps": f_bytes / (f_ms * 1e-3) / 1e9, "compressed_ms_per_decode_step": comp_ms,
+                          "ratio_full_over_compressed": f_ms * L / n_full / comp_ms,
+                          "note": "same decode kernel over the uncompressed cache (budget = prefix length)" +
+                                  ("" if n_full == L else f"; {n_full} of {L} layers fit beside the inputs, time "
+                                                          f"scaled by {L}/{n_full}")}
+            del full
+            torch.cuda.empty_cache()
+
     if rank != 0:
         if world > 1:
             dist.barrier()
@@ -466,6 +505,7 @@ def main():
         "phases_ms": {"score": float(phase[:, 0].mean()), "solver_and_page_table": float(phase[:, 1].mean()),
                       "select_compact": float(phase[:, 2].mean()), "decode": float(phase[:, 3].mean())},
         "timed_region_ms": region_ms_max,
+        "full_cache_decode": full_cache,
         "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
         "clocks": clocks,
         "paper_context": "paper reports end-to-end only (RTX A6000): 61.6% KV memory reduction, 2.1x compute "
