@@ -42,7 +42,7 @@ constexpr int kTileRows = 16;        // cache rows per pipeline stage = one TMA 
 constexpr int kChunkAlign = 64;      // chunk_rows granularity
 constexpr int kAttnWarps = 8;
 constexpr int kAttnThreads = kAttnWarps * 32;
-constexpr int kTargetItems = 4 * 148 * kAttnWarps;  // auto chunking aims at about this many extra work items
+constexpr int kTargetItems = 12 * 148 * kAttnWarps;  // auto chunking aims at about this many extra work items (a dozen per warp keeps the tail short)
 constexpr int kMinChunkRows = 256;
 constexpr int kMaxGroup = 8;
 constexpr int kFifo = 4;             // work items a warp may have fetched but not yet finished
