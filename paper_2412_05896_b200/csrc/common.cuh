@@ -21,7 +21,8 @@ struct WorkspaceHeader {
   int32_t prep_ticket;   // decode: CTAs of the prepare kernel that have finished
   int32_t n_multi;       // decode: (layer, sequence) units cut into more than one chunk
   int32_t merge_counter; // decode: next split-K merge job to hand to a warp
-  int32_t reserved[57];
+  int32_t grid_arrivals; // decode: CTAs of the self-planning launch that have finished appending
+  int32_t reserved[56];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
 

@@ -47,6 +47,7 @@ constexpr int kMinChunkRows = 256;
 constexpr int kMaxGroup = 8;
 constexpr int kFifo = 4;             // work items a warp may have fetched but not yet finished
 constexpr int kPrepThreads = 256;
+constexpr int kMaxPlanUnits = 2048;  // (layer, sequence) units up to which the attention kernel plans for itself
 
 struct DecodeParams {
   const __nv_bfloat16* q;
@@ -61,6 +62,7 @@ struct DecodeParams {
   int32_t layer_begin, n_layers, batch, n_q_heads, n_kv_heads, group;
   int32_t page_size, max_pages_per_seq, n_pages;
   int32_t chunk_rows_forced, max_items;
+  int32_t fused_plan, do_append;   // fused_plan: the attention kernel appends and plans in its own prologue
   float scale_log2;
   WorkspaceHeader* hdr;
   int32_t* tickets;   // [n_layers*batch*n_kv_heads]
@@ -80,12 +82,54 @@ struct Cfg {
   static constexpr int kStages = (D == 128) ? 3 : 6;
   static constexpr int kRingBytes = kStages * kStageBytes;     // per warp
   static constexpr int kSmemBytes = 1024 + kAttnWarps * kRingBytes + kAttnWarps * kStages * 8 +
-                                    kAttnWarps * kFifo * 16 + 64;
+                                    kAttnWarps * kFifo * 20 + (kMaxPlanUnits + 1) * 4 + kMaxPlanUnits * 2 + 64;
 };
 
 // ---------------------------------------------------------------------------------------------
 // Append (optional) and plan.  grid = n_layers*batch CTAs when appending, else 1.
 // ---------------------------------------------------------------------------------------------
+// Rows per chunk for a launch whose caches hold `total` rows over all (layer, sequence, KV head) units.
+__device__ __forceinline__ int choose_chunk(long long total, int forced) {
+  if (forced > 0) return forced;
+  long long c = (total + kTargetItems - 1) / kTargetItems;
+  c = (c + kChunkAlign - 1) / kChunkAlign * kChunkAlign;
+  if (c < kMinChunkRows) c = kMinChunkRows;
+  if (c > (1 << 30)) c = 1 << 30;
+  return (int)c;
+}
+
+// Stores the new K/V row of every KV head of unit e = (layer, sequence) in slot seq_lens and advances seq_lens.
+__device__ __forceinline__ void append_unit(const DecodeParams& p, int D, int e, int* s_page) {
+  const int tid = threadIdx.x;
+  const int l_rel = e / p.batch, b = e % p.batch;
+  const int le = (p.layer_begin + l_rel) * p.batch + b;
+  const int n = p.seq_lens[le];
+  __syncthreads();                 // s_page may still be read for the previous unit
+  if (tid == 0) {
+    int page = -1;
+    if (n >= 0 && n < p.max_pages_per_seq * p.page_size)
+      page = p.block_table[(size_t)le * p.max_pages_per_seq + n / p.page_size];
+    if (page < 0 || page >= p.n_pages) {
+      page = -1;
+      record_status(p.hdr, XKV_ERR_CAPACITY);
+    }
+    *s_page = page;
+  }
+  __syncthreads();
+  const int page = *s_page;
+  if (page >= 0) {
+    const int chunks = D / 8;
+    for (int idx = tid; idx < p.n_kv_heads * chunks; idx += blockDim.x) {
+      const int h = idx / chunks, c = idx % chunks;
+      const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
+      const size_t src = ((size_t)e * p.n_kv_heads + h) * D + c * 8;
+      *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
+      *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
+    }
+    if (tid == 0) p.seq_lens[le] = n + 1;
+  }
+}
+
 __device__ void plan_items(const DecodeParams& p) {
   __shared__ long long s_red[32];
   __shared__ int s_scan[32];
@@ -108,14 +152,7 @@ __device__ void plan_items(const DecodeParams& p) {
     long long total = 0;
     for (int w = 0; w < n_warps; ++w) total += s_red[w];
     total *= p.n_kv_heads;
-    int chunk = p.chunk_rows_forced;
-    if (chunk <= 0) {
-      long long c = (total + kTargetItems - 1) / kTargetItems;
-      c = (c + kChunkAlign - 1) / kChunkAlign * kChunkAlign;
-      if (c < kMinChunkRows) c = kMinChunkRows;
-      if (c > (1 << 30)) c = 1 << 30;
-      chunk = (int)c;
-    }
+    const int chunk = choose_chunk(total, p.chunk_rows_forced);
     s_chunk = chunk;
     s_carry = 0;
     s_multi = 0;
@@ -184,35 +221,7 @@ __global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodePara
   __shared__ int s_page;
   __shared__ int s_last;
   const int tid = threadIdx.x;
-  if (do_append) {
-    const int e = blockIdx.x;
-    const int l_rel = e / p.batch, b = e % p.batch;
-    const int le = (p.layer_begin + l_rel) * p.batch + b;
-    const int n = p.seq_lens[le];
-    if (tid == 0) {
-      int page = -1;
-      if (n >= 0 && n < p.max_pages_per_seq * p.page_size)
-        page = p.block_table[(size_t)le * p.max_pages_per_seq + n / p.page_size];
-      if (page < 0 || page >= p.n_pages) {
-        page = -1;
-        record_status(p.hdr, XKV_ERR_CAPACITY);
-      }
-      s_page = page;
-    }
-    __syncthreads();
-    const int page = s_page;
-    if (page >= 0) {
-      const int chunks = D / 8;
-      for (int idx = tid; idx < p.n_kv_heads * chunks; idx += blockDim.x) {
-        const int h = idx / chunks, c = idx % chunks;
-        const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
-        const size_t src = ((size_t)e * p.n_kv_heads + h) * D + c * 8;
-        *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
-        *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
-      }
-      if (tid == 0) p.seq_lens[le] = n + 1;
-    }
-  }
+  if (do_append) append_unit(p, D, blockIdx.x, &s_page);
   // the last CTA to get here sees every sequence length already advanced and writes the plan
   __threadfence();
   __syncthreads();
@@ -260,8 +269,14 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint8_t* ring = smem + (size_t)warp * C::kRingBytes;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes) + warp * C::kStages;
-  int4* fifo = reinterpret_cast<int4*>(smem + (size_t)kAttnWarps * C::kRingBytes + kAttnWarps * C::kStages * 8) +
-               warp * kFifo;
+  uint8_t* fifo_base = smem + (size_t)kAttnWarps * C::kRingBytes + kAttnWarps * C::kStages * 8;
+  int4* fifo = reinterpret_cast<int4*>(fifo_base) + warp * kFifo;                        // item descriptors
+  int* fifo_idx = reinterpret_cast<int*>(fifo_base + kAttnWarps * kFifo * 16) + warp * kFifo;   // and their indices
+  int* s_excl = reinterpret_cast<int*>(fifo_base + kAttnWarps * kFifo * 20);   // [units + 1] chunks before each unit
+  uint16_t* s_multi = reinterpret_cast<uint16_t*>(s_excl + kMaxPlanUnits + 1);  // units cut into several chunks
+  __shared__ int s_plan[4];                                                     // chunk rows, split units, page scratch
+  __shared__ int s_scan[2 * kAttnWarps];
+  __shared__ long long s_rows[kAttnWarps];
 
   if (tid == 0) {
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes);
@@ -272,8 +287,135 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   }
   __syncthreads();
 
-  const int n_items = p.hdr->n_items;
-  const int n_multi = p.hdr->n_multi;
+  const bool fused = p.fused_plan != 0;
+  const int n_units = p.n_layers * p.batch;
+  if (fused) {
+    // ---- prologue of the self-planning launch: append, meet, plan
+    for (int e = blockIdx.x; e < n_units; e += gridDim.x) {
+      if (p.do_append) append_unit(p, D, e, &s_plan[3]);
+      for (int h = tid; h < p.n_kv_heads; h += kAttnThreads) p.tickets[e * p.n_kv_heads + h] = 0;
+    }
+    // every CTA of the grid is resident (cooperative launch): wait until all have appended
+    __threadfence();
+    __syncthreads();
+    int met = 1;
+    if (tid == 0) {
+      atomicAdd(&p.hdr->grid_arrivals, 1);
+      const uint64_t t0 = global_timer_ns();
+      while (ld_acquire_gpu(&p.hdr->grid_arrivals) < (int)gridDim.x) {
+        if (global_timer_ns() - t0 > 2000000000ull) {
+          met = 0;
+          record_status(p.hdr, XKV_ERR_TIMEOUT);
+          break;
+        }
+        __nanosleep(64);
+      }
+      __threadfence();
+    }
+    if (!__syncthreads_and(met)) return;
+    // the plan, computed by every CTA for itself: chunk size from the total length, then the number of chunks
+    // before each unit (and the list of units with more than one)
+    constexpr int kPer = kMaxPlanUnits / kAttnThreads;
+    int nloc[kPer];
+    long long rows = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int e = tid * kPer + i;
+      int n = 0;
+      if (e < n_units) n = __ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]);
+      nloc[i] = n > 0 ? n : 0;
+      rows += nloc[i];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rows += __shfl_xor_sync(0xffffffffu, rows, o);
+    if (lane == 0) s_rows[warp] = rows;
+    __syncthreads();
+    long long total = 0;
+#pragma unroll
+    for (int w8 = 0; w8 < kAttnWarps; ++w8) total += s_rows[w8];
+    const int chunk = choose_chunk(total * p.n_kv_heads, p.chunk_rows_forced);
+    int cnt = 0, mcnt = 0;
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int e = tid * kPer + i;
+      const int nc = e < n_units ? (nloc[i] == 0 ? 1 : (nloc[i] + chunk - 1) / chunk) : 0;
+      nloc[i] = nc;
+      cnt += nc;
+      mcnt += nc > 1 ? 1 : 0;
+    }
+    int icnt = cnt, imcnt = mcnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, icnt, o), b = __shfl_up_sync(0xffffffffu, imcnt, o);
+      if (lane >= o) {
+        icnt += a;
+        imcnt += b;
+      }
+    }
+    if (lane == 31) {
+      s_scan[warp] = icnt;
+      s_scan[kAttnWarps + warp] = imcnt;
+    }
+    __syncthreads();
+    int base = icnt - cnt, mbase = imcnt - mcnt, all = 0, mall = 0;
+#pragma unroll
+    for (int w8 = 0; w8 < kAttnWarps; ++w8) {
+      if (w8 < warp) {
+        base += s_scan[w8];
+        mbase += s_scan[kAttnWarps + w8];
+      }
+      all += s_scan[w8];
+      mall += s_scan[kAttnWarps + w8];
+    }
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+      const int e = tid * kPer + i;
+      if (e < n_units) {
+        s_excl[e] = base;
+        if (nloc[i] > 1) s_multi[mbase++] = (uint16_t)e;
+        base += nloc[i];
+      }
+    }
+    if (tid == 0) {
+      s_excl[n_units] = all;
+      s_plan[0] = chunk;
+      s_plan[1] = mall;
+      s_plan[2] = ((long long)all * p.n_kv_heads <= (long long)p.max_items) ? all * p.n_kv_heads : -1;
+      if (blockIdx.x == 0) {
+        p.hdr->chunk_rows = chunk;
+        p.hdr->n_items = s_plan[2] < 0 ? 0 : s_plan[2];
+        p.hdr->n_multi = mall;
+        if (s_plan[2] < 0) record_status(p.hdr, XKV_ERR_WORKSPACE);
+      }
+    }
+    __syncthreads();
+  }
+  const int n_items = fused ? max(s_plan[2], 0) : p.hdr->n_items;
+  const int n_multi = fused ? (s_plan[2] < 0 ? 0 : s_plan[1]) : p.hdr->n_multi;
+  const int plan_chunk = fused ? s_plan[0] : 0;
+  // work item idx -> {unit e, KV head, first row, end row}
+  auto item_desc = [&](int idx) -> int4 {
+    if (!fused) return p.items[idx];
+    const int q = idx / p.n_kv_heads;
+    int lo = 0, hi = n_units;                      // s_excl[lo] <= q < s_excl[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_excl[mid] <= q) lo = mid;
+      else hi = mid;
+    }
+    const int first_chunk = s_excl[lo], nc = s_excl[lo + 1] - first_chunk;
+    const int local = idx - first_chunk * p.n_kv_heads;
+    const int h = local / nc, c = local % nc;
+    int n = __ldcg(&p.seq_lens[(p.layer_begin + lo / p.batch) * p.batch + lo % p.batch]);
+    n = n > 0 ? n : 0;
+    const int rb = c * plan_chunk;
+    return make_int4(lo, h, rb, min(n, rb + plan_chunk));
+  };
+  // {first work item of the unit's KV head 0, chunks per KV head}
+  auto unit_info = [&](int e) -> int2 {
+    if (!fused) return p.unit_info[e];
+    return make_int2(s_excl[e] * p.n_kv_heads, s_excl[e + 1] - s_excl[e]);
+  };
   const int gid = lane >> 2, tig = lane & 3;
   const int mat = lane >> 3, mrow = lane & 7;
   const int G = p.group;
@@ -299,10 +441,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
           return false;
         }
         if (lane == 0) next_idx = atomicAdd(&p.hdr->work_counter, 1);   // fetched early, used at the next item
-        p_desc = p.items[idx];
+        p_desc = item_desc(idx);
         p_item = idx;
         const int slot = (fifo_head + fifo_count) % kFifo;
-        if (lane == 0) fifo[slot] = make_int4(idx, 0, 0, 0);
+        if (lane == 0) {
+          fifo[slot] = p_desc;
+          fifo_idx[slot] = idx;
+        }
         ++fifo_count;
         p_row = p_desc.z;
         if (p_row >= p_desc.w) continue;          // empty cache: the consumer side writes zeros
@@ -368,12 +513,12 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     fill();
     if (fifo_count == 0) break;
     __syncwarp();
-    const int item = fifo[fifo_head].x;
+    const int item = fifo_idx[fifo_head];
+    const int4 I = fifo[fifo_head];
     fifo_head = (fifo_head + 1) % kFifo;
     --fifo_count;
-    const int4 I = p.items[item];
     const int e = I.x, h = I.y;
-    const int nc = p.unit_info[e].y;
+    const int nc = unit_info(e).y;
     const size_t q_row0 = ((size_t)e * p.n_q_heads + (size_t)h * G);
 
     // Q^T as the B operand: lane (gid, tig) holds head gid, columns 16*ks + 2*tig (+1) and + 8
@@ -553,8 +698,9 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     job = __shfl_sync(0xffffffffu, job, 0);
     if (job >= n_jobs) break;
     const int g = job % G, uh = job / G;
-    const int h = uh % p.n_kv_heads, e = p.multi_list[uh / p.n_kv_heads];
-    const int2 ui = p.unit_info[e];
+    const int h = uh % p.n_kv_heads;
+    const int e = fused ? (int)s_multi[uh / p.n_kv_heads] : p.multi_list[uh / p.n_kv_heads];
+    const int2 ui = unit_info(e);
     const int nc = ui.y, first = ui.x + h * nc;
     int ready = 1;
     if (lane == 0) {
@@ -719,7 +865,25 @@ xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const Decod
     done[dev] = true;
   }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_start, st);
-  decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
+  if (p.fused_plan) {
+    // the prologue's grid-wide meeting needs every CTA resident: a cooperative launch guarantees it
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)sm_count());
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = Cfg<D>::kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_attn_kernel<D>, tk, tv, p) != cudaSuccess) {
+      cudaGetLastError();
+      return XKV_ERR_CUDA;
+    }
+  } else {
+    decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
+  }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_stop, st);
   count_launch();
   return check_launch();
@@ -789,13 +953,21 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   p.part_o = reinterpret_cast<float*>(ws + L.part_o);
   p.part_ml = reinterpret_cast<float*>(ws + L.part_ml);
 
-  if (cudaMemsetAsync(ws, 0, L.unit_info, st) != cudaSuccess) return XKV_ERR_CUDA;   // header + tickets
   const int n_units = Lr * d->batch;
   const int do_append = k_new != nullptr ? 1 : 0;
-  decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append);
-  count_launch();
-  xkv_status s = check_launch();
-  if (s != XKV_OK) return s;
+  // Up to kMaxPlanUnits units the attention kernel appends and plans in its own prologue (one launch);
+  // beyond that a separate kernel appends and writes the work-item table.
+  p.fused_plan = n_units <= kMaxPlanUnits ? 1 : 0;
+  p.do_append = do_append;
+  if (p.fused_plan) {
+    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;   // status, counters
+  } else {
+    if (cudaMemsetAsync(ws, 0, L.unit_info, st) != cudaSuccess) return XKV_ERR_CUDA;    // header + tickets
+    decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append);
+    count_launch();
+    xkv_status s = check_launch();
+    if (s != XKV_OK) return s;
+  }
   if (d->head_dim == 128) return launch_attn<128>(tk, tv, p, st);
   return launch_attn<64>(tk, tv, p, st);
 }

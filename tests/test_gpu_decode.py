@@ -127,6 +127,14 @@ def test_decode_many_units_long_chunks():
     _run_case(6, 16, 8, 8, 128, lens, 16, 0, True, seed=9)
 
 
+def test_decode_more_units_than_the_attention_kernel_plans_for_itself():
+    """Above 2048 (layer, sequence) units a separate kernel appends and writes the work-item table."""
+    rng = np.random.default_rng(11)
+    lens = rng.integers(0, 70, size=(8, 300)).tolist()
+    _run_case(8, 300, 2, 1, 64, lens, 16, 0, True, seed=21, steps=2)
+    _run_case(8, 300, 2, 1, 64, lens, 16, 64, False, seed=22)
+
+
 def test_decode_capacity_overflow_is_reported_not_faulted():
     require_lib()
     L, B, Hq, Hkv, d, ps = 1, 2, 4, 4, 64, 16
