@@ -5,6 +5,9 @@
 #include <cmath>
 #include <queue>
 #include <utility>
+#include <thread>
+#include <cstring>
+#include <algorithm>
 #include <vector>
 
 #include "common.cuh"
@@ -234,9 +237,89 @@ struct WaitEntry {
   }
 };
 
+// Order-preserving map of a double onto an unsigned integer (larger value -> larger key).
+inline uint64_t ordered_key(double v) {
+  uint64_t u;
+  std::memcpy(&u, &v, sizeof(u));
+  return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// Total-budget mode when every curve is non-increasing over the positions still open (what sorted scores
+// give): the listing then grants the open positions in the order (value descending, layer ascending,
+// position ascending), so its result is "every position above the R-th largest value, and positions equal
+// to it from the lowest layers first".  The R-th largest value is found by bisecting the value's bit pattern,
+// counting per layer with a binary search: the same budgets as the heap below, without its R pops.
+bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std::vector<int64_t>& cap, int64_t total,
+                        int n_min, int32_t* budgets, double* r_avg, xkv_status* status) {
+  const int L = (int)curve.size();
+  std::vector<int64_t> lo(L), hi(L);           // open positions of layer l: [lo, hi); beyond the curve the gain is 0
+  int64_t used = 0, open = 0;
+  for (int l = 0; l < L; ++l) {
+    lo[l] = n_min < cap[l] ? n_min : cap[l];
+    hi[l] = cap[l];
+    used += lo[l];
+    open += hi[l] - lo[l];
+    const int64_t n = (int64_t)curve[l].size();
+    for (int64_t j = lo[l] + 1; j < hi[l] && j < n; ++j)
+      if (curve[l][j] > curve[l][j - 1]) return false;
+    if (hi[l] > n && n > lo[l] && curve[l][n - 1] < 0.0) return false;       // the implicit zeros would rise again
+  }
+  if (total < used || total - used > open) {
+    *status = XKV_ERR_BUDGET;
+    return true;
+  }
+  const int64_t R = total - used;
+  auto value_at = [&](int l, int64_t j) -> double { return j < (int64_t)curve[l].size() ? curve[l][j] : 0.0; };
+  // open positions of layer l whose key is >= key (the curve is non-increasing, so they form a prefix)
+  auto count_ge = [&](int l, uint64_t key) -> int64_t {
+    int64_t a = lo[l], b = hi[l];
+    while (a < b) {
+      const int64_t mid = (a + b) >> 1;
+      if (ordered_key(value_at(l, mid)) >= key) a = mid + 1;
+      else b = mid;
+    }
+    return a - lo[l];
+  };
+  std::vector<int64_t> alloc(lo);
+  if (R > 0) {
+    uint64_t klo = 0, khi = ~0ull;               // largest key with count(key) >= R
+    while (klo < khi) {
+      const uint64_t mid = klo + ((khi - klo) >> 1) + 1;
+      int64_t c = 0;
+      for (int l = 0; l < L; ++l) c += count_ge(l, mid);
+      if (c >= R) klo = mid;
+      else khi = mid - 1;
+    }
+    int64_t left = R;
+    for (int l = 0; l < L; ++l) {                // everything strictly above the threshold value
+      const int64_t above = klo == ~0ull ? 0 : count_ge(l, klo + 1);
+      alloc[l] += above;
+      left -= above;
+    }
+    for (int l = 0; l < L && left > 0; ++l) {    // ties at the threshold: lowest layers first
+      const int64_t ties = count_ge(l, klo) - (alloc[l] - lo[l]);
+      const int64_t take = ties < left ? ties : left;
+      alloc[l] += take;
+      left -= take;
+    }
+  }
+  double r_total = 0.0;
+  for (int l = 0; l < L; ++l) {
+    for (int64_t j = 0; j < alloc[l]; ++j) r_total += value_at(l, j);
+    budgets[l] = (int32_t)alloc[l];
+  }
+  if (r_avg != nullptr) *r_avg = r_total / L;
+  *status = XKV_OK;
+  return true;
+}
+
 xkv_status solve_one(const std::vector<std::vector<double>>& curve, const std::vector<int64_t>& cap,
                      int64_t total, double r_target, int n_min, int32_t* budgets, double* r_avg) {
   const int L = (int)curve.size();
+  if (total >= 0) {
+    xkv_status st = XKV_OK;
+    if (solve_sorted_total(curve, cap, total, n_min, budgets, r_avg, &st)) return st;
+  }
   std::vector<int64_t> alloc(L);
   double r_total = 0.0;
   int64_t used = 0;
@@ -291,12 +374,27 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
   const size_t lstride = (size_t)batch * curve_len;
   if (!per_sequence) {
     std::vector<std::vector<double>> curve(n_layers, std::vector<double>(curve_len, 0.0));
-    for (int l = 0; l < n_layers; ++l) {
-      for (int b = 0; b < batch; ++b) {
-        const float* g = gains + l * lstride + (size_t)b * curve_len;
-        for (int j = 0; j < curve_len; ++j) curve[l][j] += (double)g[j];
+    auto mean_layers = [&](int l0, int l1) {
+      for (int l = l0; l < l1; ++l) {
+        double* c = curve[l].data();
+        for (int b = 0; b < batch; ++b) {
+          const float* g = gains + l * lstride + (size_t)b * curve_len;
+          for (int j = 0; j < curve_len; ++j) c[j] += (double)g[j];
+        }
+        for (int j = 0; j < curve_len; ++j) c[j] /= batch;
       }
-      for (int j = 0; j < curve_len; ++j) curve[l][j] /= batch;
+    };
+    // the batch mean reads every curve once: spread the layers over a few threads when that is megabytes
+    int n_threads = (int)std::min<size_t>(8, (size_t)n_layers * lstride / (1u << 20));
+    if (n_threads > n_layers) n_threads = n_layers;
+    if (n_threads <= 1) {
+      mean_layers(0, n_layers);
+    } else {
+      std::vector<std::thread> pool;
+      for (int i = 0; i < n_threads; ++i)
+        pool.emplace_back(mean_layers, (int)((int64_t)n_layers * i / n_threads),
+                          (int)((int64_t)n_layers * (i + 1) / n_threads));
+      for (auto& th : pool) th.join();
     }
     int64_t c = max_prefix;
     if (n_max > 0 && n_max < c) c = n_max;

@@ -140,3 +140,30 @@ def test_alloc_budgets_modes():
     same = np.tile(O.head_gains(np.array([5.0, 4, 3, 2, 1])).astype(np.float32), (3, 1, 1))
     budgets, _ = xkv.alloc_budgets(same, [5], total=7)
     assert budgets.tolist() == [3, 2, 2]
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_alloc_budgets_ties_and_unsorted_curves(seed):
+    """Sorted curves take the threshold solver, anything else the heap: both must grant like Algorithm 1, also when
+    many positions of many layers hold the same value (ties go to the lowest layer, then the next position)."""
+    rng = np.random.default_rng(100 + seed)
+    L, n = 6, 40
+    # few distinct values, non-increasing per layer, trailing zeros
+    q = np.sort(rng.integers(0, 5, size=(L, 1, n)), axis=2)[:, :, ::-1].astype(np.float32) / 8.0
+    gains = [q[l, 0].astype(np.float64) for l in range(L)]
+    for N, n_min, n_max in [(0, 0, 0), (17, 0, 0), (95, 3, 25), (L * n, 0, 0), (60, 10, 10), (101, 2, 0)]:
+        if n_max and N > L * n_max:
+            continue
+        budgets, r = xkv.alloc_budgets(q, [n], total=N, n_min=n_min, n_max=n_max)
+        A, r_o = O.adaptive_allocation(gains, N=N, n_min=n_min, n_max=n_max or None)
+        assert budgets.tolist() == A and abs(r - r_o) < 1e-12
+    # curve shorter than the capacity: the positions beyond it count as zeros
+    budgets, r = xkv.alloc_budgets(q[:, :, :10], [30], total=100)
+    A, r_o = O.adaptive_allocation([g[:10] for g in gains], N=100, capacity=[30] * L)
+    assert budgets.tolist() == A and abs(r - r_o) < 1e-12
+    # unsorted curves (not what scoring produces, but the entry point accepts them)
+    u = rng.random((L, 1, n)).astype(np.float32)
+    for N in (1, 33, 150):
+        budgets, r = xkv.alloc_budgets(u, [n], total=N, n_min=2)
+        A, r_o = O.adaptive_allocation([u[l, 0].astype(np.float64) for l in range(L)], N=N, n_min=2)
+        assert budgets.tolist() == A and abs(r - r_o) < 1e-12
