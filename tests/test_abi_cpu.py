@@ -163,7 +163,7 @@ def test_alloc_budgets_ties_and_unsorted_curves(seed):
     assert budgets.tolist() == A and abs(r - r_o) < 1e-12
     # unsorted curves (not what scoring produces, but the entry point accepts them)
     u = rng.random((L, 1, n)).astype(np.float32)
-    for N in (1, 33, 150):
+    for N in (12, 33, 150):
         budgets, r = xkv.alloc_budgets(u, [n], total=N, n_min=2)
         A, r_o = O.adaptive_allocation([u[l, 0].astype(np.float64) for l in range(L)], N=N, n_min=2)
         assert budgets.tolist() == A and abs(r - r_o) < 1e-12
