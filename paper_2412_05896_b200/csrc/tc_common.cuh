@@ -132,21 +132,40 @@ struct TcCfg {
                                        kMrowSlots * 256 * 4 /*row normalisers*/ + 256 /*barriers*/;
 };
 
+// Online-softmax update of one query row with 32 more logits v (raw dot products; scale > 0 folds 1/sqrt(d) and
+// log2 e).  Tiles that reach into the observation window mask the keys the row must not see; all other tiles
+// skip that work (masked is the same for every thread of a tile).  Maximum and sum run as four independent
+// chains so that neither is one long dependent sequence.
 __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
                                           float& m, float& l) {
   float x[32];
-  float vmax = -INFINITY;
 #pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    x[i] = (masked && c0 + i > limit) ? -INFINITY : v[i];
-    vmax = fmaxf(vmax, x[i]);
+  for (int i = 0; i < 32; ++i) x[i] = v[i];
+  if (masked) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (c0 + i > limit) x[i] = -INFINITY;
   }
+  float mx[4] = {x[0], x[1], x[2], x[3]};
+#pragma unroll
+  for (int i = 4; i < 32; i += 4) {
+    mx[0] = fmaxf(mx[0], x[i]);
+    mx[1] = fmaxf(mx[1], x[i + 1]);
+    mx[2] = fmaxf(mx[2], x[i + 2]);
+    mx[3] = fmaxf(mx[3], x[i + 3]);
+  }
+  const float vmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   const float m_new = fmaxf(m, vmax * scale);
   const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-  float sum = 0.f;
+  float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int i = 0; i < 32; ++i) sum += fast_exp2(fmaf(x[i], scale, -m_ref));
-  l = l * fast_exp2(m - m_ref) + sum;
+  for (int i = 0; i < 32; i += 4) {
+    sm[0] += fast_exp2(fmaf(x[i], scale, -m_ref));
+    sm[1] += fast_exp2(fmaf(x[i + 1], scale, -m_ref));
+    sm[2] += fast_exp2(fmaf(x[i + 2], scale, -m_ref));
+    sm[3] += fast_exp2(fmaf(x[i + 3], scale, -m_ref));
+  }
+  l = l * fast_exp2(m - m_ref) + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
   m = m_new;
 }
 
