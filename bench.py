@@ -275,9 +275,7 @@ def main():
                 q_win[l].copy_(host["q_win"][l], non_blocking=True)
                 k[l].copy_(host["k"][l], non_blocking=True)
                 v[l].copy_(host["v"][l], non_blocking=True)
-        for l in range(L):
-            sess.score_layer(l, q_win[l], k[l])
-        sess.join()
+        sess.score_layers(q_win, k)
         e[1].record()
         if w.budgets is not None:
             budgets = np.asarray(w.budgets, dtype=np.int32)
@@ -285,9 +283,7 @@ def main():
             budgets, _ = sess.solve_budgets(total=N_total, n_min=w.n_min, n_max=w.n_max)
         sess.assign_pages(budgets)
         e[2].record()
-        for l in range(L):
-            sess.select_layer(l, int(budgets[l]), k[l], v[l])
-        sess.join()
+        sess.select_layers(budgets, k, v)
         e[3].record()
         if host is None:
             for s in range(n_dec):

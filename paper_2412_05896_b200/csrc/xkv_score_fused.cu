@@ -412,7 +412,7 @@ xkv_status fused_launch(const CUtensorMap& tq, const CUtensorMap& tk, const Scor
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (max_clusters[dev] == 0) {
-    if (cudaFuncSetAttribute(score_fused_kernel<D, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+    if (cudaFuncSetAttribute(score_fused_kernel<D, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return XKV_ERR_CUDA;
     // clusters that can be resident together: units are dealt to exactly that many, so none waits for an SM

@@ -36,14 +36,17 @@ struct ItemShape {
   int unit, split, b, g, cu, t, P, key_begin, key_end, n_tiles;
 };
 
-// Item n of this CTA; returns false when the sequence is exhausted.  Empty items have n_tiles == 0.
+// Item n of this CTA; returns false when the sequence is exhausted.  Empty items have n_tiles == 0.  Items are
+// numbered split-major (all units' split 0, then all units' split 1, ...): with ragged lengths the empty items
+// are the high splits of short sequences, and this order gives every CTA the same share of every split level.
 template <int PASS>
 __device__ __forceinline__ bool item_shape(const ScoreParams& p, int n, ItemShape* it) {
   int idx = blockIdx.x + n * gridDim.x;
   if (idx >= p.n_work) return false;
   if (PASS == 2) idx = p.n_work - 1 - idx;       // reverse: the keys pass 1 read last are still in L2
-  it->unit = idx / p.n_splits;
-  it->split = idx % p.n_splits;
+  const int units = p.batch * p.n_kv_heads;
+  it->unit = idx % units;
+  it->split = idx / units;
   it->b = it->unit / p.n_kv_heads;
   it->g = it->unit % p.n_kv_heads;
   it->cu = p.cu_seqlens[it->b];
@@ -292,14 +295,16 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
   if (warp == 0) tmem_dealloc(tmem_base, C::kTmemCols);
 }
 
-// One warp per query row of a unit: mrow[r] = m_r + log2(l_r) (log2 domain; +inf for rows without visible
-// keys) from the per-split, per-group, per-replica statistics pass 1 stored.  grid = (units, M / 4).
-__global__ void __launch_bounds__(128) tc_merge_kernel(const ScoreParams p) {
+// grid = (units, M / 32), blockDim = (32 query rows, up to 32 slices): mrow[r] = m_r + log2(l_r) (log2 domain; +inf for
+// rows without visible keys) from the per-split, per-group, per-replica statistics pass 1 stored.  Consecutive
+// rows are consecutive in every partial vector, so a warp's load is one 256-byte segment; a slice takes every
+// blockDim.y-th partial, and the slices are combined through shared memory.
+__global__ void __launch_bounds__(1024) tc_merge_kernel(const ScoreParams p) {
+  __shared__ float2 s_part[32][33];
   const int unit = blockIdx.x;
   const int M = p.M;
-  const int lane = threadIdx.x & 31;
-  const int r = blockIdx.y * 4 + (threadIdx.x >> 5);
-  if (r >= M) return;
+  const int rl = threadIdx.x, sl = threadIdx.y, n_sl = blockDim.y;
+  const int r = blockIdx.y * 32 + rl;
   const int group_entries = M < 128 ? 128 : M;
   const int group_reps = M < 128 ? 128 / M : 1;
   const int per_split = kAccBufs * group_reps;               // partial statistics of this row per split
@@ -308,24 +313,34 @@ __global__ void __launch_bounds__(128) tc_merge_kernel(const ScoreParams p) {
   const int t = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
   const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
   const float2* part = p.stats_part + (size_t)unit * p.n_splits * entries + r;
+  const int n = n_splits_u * per_split;
   float m = -INFINITY, l = 0.f;
-  for (int i = lane; i < n_splits_u * per_split; i += 32) {
-    const int s = i / per_split, q = i % per_split;
-    const float2 v = part[(size_t)s * entries + (q / group_reps) * group_entries + (q % group_reps) * M];
+  auto fold = [&](float2 v) {
     const float m_new = fmaxf(m, v.x);
     const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
     l = l * exp2f(m - m_ref) + v.y * exp2f(v.x - m_ref);
     m = m_new;
+  };
+  auto at = [&](int i) -> const float2* {
+    const int s = i / per_split, q = i % per_split;
+    return part + (size_t)s * entries + (q / group_reps) * group_entries + (q % group_reps) * M;
+  };
+  int i = sl;
+  for (; i + 3 * n_sl < n; i += 4 * n_sl) {
+    const float2 v0 = __ldcg(at(i)), v1 = __ldcg(at(i + n_sl)), v2 = __ldcg(at(i + 2 * n_sl)),
+                 v3 = __ldcg(at(i + 3 * n_sl));
+    fold(v0);
+    fold(v1);
+    fold(v2);
+    fold(v3);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float mo = __shfl_xor_sync(0xffffffffu, m, o), lo = __shfl_xor_sync(0xffffffffu, l, o);
-    const float m_new = fmaxf(m, mo);
-    const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-    l = l * exp2f(m - m_ref) + lo * exp2f(mo - m_ref);
-    m = m_new;
+  for (; i < n; i += n_sl) fold(__ldcg(at(i)));
+  s_part[sl][rl] = make_float2(m, l);
+  __syncthreads();
+  if (sl == 0) {
+    for (int k = 1; k < n_sl; ++k) fold(s_part[k][rl]);
+    p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
   }
-  if (lane == 0) p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -354,7 +369,7 @@ xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScorePa
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
   if (!done[dev]) {
     if (cudaFuncSetAttribute(score_tc_kernel<D, M, PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             227 * 1024) != cudaSuccess)
+                             (int)smem) != cudaSuccess)      // the kernel also has a few KB of static shared memory
       return XKV_ERR_CUDA;
     done[dev] = true;
   }
@@ -369,7 +384,11 @@ template <int D, int M>
 xkv_status tc_launch_both(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, cudaStream_t st) {
   xkv_status s = tc_launch<D, M, 1>(tq, tk, p, st);
   if (s != XKV_OK) return s;
-  tc_merge_kernel<<<dim3(p.batch * p.n_kv_heads, M / 4), 128, 0, st>>>(p);
+  // about four partials per slice: short sequences get small CTAs, long ones many loads in flight
+  const int n_part = p.n_splits * kAccBufs * (M < 128 ? 128 / M : 1);
+  int slices = 1;
+  while (slices < 32 && slices * 4 < n_part) slices <<= 1;
+  tc_merge_kernel<<<dim3(p.batch * p.n_kv_heads, M / 32), dim3(32, slices), 0, st>>>(p);
   count_launch();
   s = check_launch();
   if (s != XKV_OK) return s;

@@ -5,6 +5,11 @@
 //                  keeps every position above it and the lowest positions equal to it until k are
 //                  kept (ties go to the lower position), which yields the kept positions already in
 //                  ascending order.  The window positions follow.
+//   select_count_kernel, select_chunk_kernel
+//                  the same selection for prefixes longer than one sweep step (4096 positions): one CTA per
+//                  (unit, 4096-position chunk) first counts the scores above and equal to the threshold, then
+//                  every chunk finds its place from the counts of the chunks before it and writes its kept
+//                  positions, so a long sequence is swept by many CTAs at once instead of one.
 //   gather_kernel  16-byte vectorised copy of the kept K and V rows (256-byte rows for d = 128) into
 //                  the layer's cache pages; pure data movement, HBM-bound.
 #include "common.cuh"
@@ -34,6 +39,8 @@ struct SelectParams {
   __nv_bfloat16* v_pages;
   int64_t total_tokens, stride_token, stride_head;
   int32_t batch, n_kv_heads, head_dim, window, page_size, max_pages_per_seq, n_pages;
+  int2* counts;                // [units][n_chunks] scores above / equal to the threshold per chunk (chunked path)
+  int32_t n_chunks;
   WorkspaceHeader* hdr;
 };
 
@@ -134,6 +141,113 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   }
 }
 
+constexpr int kSelChunk = kSelThreads * kSelItems;     // positions one CTA sweeps in the chunked path
+
+// grid = (units, n_chunks): scores of the chunk above and equal to the unit's threshold.
+__global__ void __launch_bounds__(kSelThreads) select_count_kernel(SelectParams p) {
+  __shared__ int s_warp[33];
+  const int unit = blockIdx.x, chunk = blockIdx.y;
+  const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
+  int cu, t, P, kb;
+  unit_shape(p, b, &cu, &t, &P, &kb);
+  if (kb == 0 || kb == P || chunk * kSelChunk >= P) return;      // nothing to count: no selection by score
+  const float* w = p.scores + (size_t)g * p.total_tokens + cu;
+  const float thr = p.sorted[(size_t)g * p.total_tokens + cu + kb - 1];
+  const int c0 = chunk * kSelChunk + threadIdx.x * kSelItems;
+  int n_gt = 0, n_eq = 0;
+#pragma unroll
+  for (int i = 0; i < kSelItems; ++i) {
+    const float x = (c0 + i < P) ? w[c0 + i] : -1.f;
+    n_gt += x > thr ? 1 : 0;
+    n_eq += x == thr ? 1 : 0;
+  }
+  int tot;
+  block_scan_excl(n_gt | (n_eq << 16), s_warp, &tot);           // at most 4096 of either: 16 bits each
+  if (threadIdx.x == 0) p.counts[(size_t)unit * p.n_chunks + chunk] = make_int2(tot & 0xffff, tot >> 16);
+}
+
+// grid = (units, n_chunks): the kept positions of the chunk, placed after those of the chunks before it.
+__global__ void __launch_bounds__(kSelThreads) select_chunk_kernel(SelectParams p) {
+  __shared__ int s_warp[33];
+  __shared__ int s_base[3];
+  const int unit = blockIdx.x, chunk = blockIdx.y;
+  const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
+  int cu, t, P, kb;
+  unit_shape(p, b, &cu, &t, &P, &kb);
+  const int n_keep = kb + (t - P);
+  const bool fits = n_keep <= p.max_pages_per_seq * p.page_size;
+  if (chunk == 0 && threadIdx.x == 0 && g == 0) {
+    p.seq_lens_layer[b] = fits ? n_keep : 0;
+    if (!fits) record_status(p.hdr, XKV_ERR_CAPACITY);
+  }
+  if (!fits) return;
+  int32_t* sel = p.sel + (size_t)unit * p.sel_stride;
+  if (chunk == 0)
+    for (int i = threadIdx.x; i < t - P; i += kSelThreads) sel[kb + i] = P + i;   // window positions
+  const int begin = chunk * kSelChunk;
+  if (kb == 0 || begin >= P) return;
+  const int c0 = begin + threadIdx.x * kSelItems;
+  if (kb == P) {
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i)
+      if (c0 + i < P) sel[c0 + i] = c0 + i;
+    return;
+  }
+  // totals over the unit and over the chunks before this one
+  if (threadIdx.x < 32) {
+    int gt_all = 0, gt_before = 0, eq_before = 0;
+    const int n_ch = (P + kSelChunk - 1) / kSelChunk;
+    for (int c = threadIdx.x; c < n_ch; c += 32) {
+      const int2 v = __ldcg(&p.counts[(size_t)unit * p.n_chunks + c]);
+      gt_all += v.x;
+      if (c < chunk) {
+        gt_before += v.x;
+        eq_before += v.y;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      gt_all += __shfl_xor_sync(0xffffffffu, gt_all, o);
+      gt_before += __shfl_xor_sync(0xffffffffu, gt_before, o);
+      eq_before += __shfl_xor_sync(0xffffffffu, eq_before, o);
+    }
+    if (threadIdx.x == 0) {
+      s_base[0] = kb - gt_all;        // positions equal to the threshold that are kept (the lowest ones)
+      s_base[1] = gt_before;
+      s_base[2] = eq_before;
+    }
+  }
+  __syncthreads();
+  const int eq_needed = s_base[0];
+  const int eq_start = s_base[2];
+  const int dst_start = s_base[1] + min(eq_start, eq_needed);
+  const float* w = p.scores + (size_t)g * p.total_tokens + cu;
+  const float thr = p.sorted[(size_t)g * p.total_tokens + cu + kb - 1];
+  float x[kSelItems];
+  int n_eq = 0;
+#pragma unroll
+  for (int i = 0; i < kSelItems; ++i) {
+    x[i] = (c0 + i < P) ? w[c0 + i] : -1.f;
+    n_eq += (x[i] == thr) ? 1 : 0;
+  }
+  int tot_eq;
+  int eq_before = eq_start + block_scan_excl(n_eq, s_warp, &tot_eq);
+  bool keep[kSelItems];
+  int n_sel = 0;
+#pragma unroll
+  for (int i = 0; i < kSelItems; ++i) {
+    const bool is_eq = x[i] == thr;
+    keep[i] = (c0 + i < P) && (x[i] > thr || (is_eq && eq_before < eq_needed));
+    eq_before += is_eq ? 1 : 0;
+    n_sel += keep[i] ? 1 : 0;
+  }
+  int tot_sel;
+  int dst = dst_start + block_scan_excl(n_sel, s_warp, &tot_sel);
+#pragma unroll
+  for (int i = 0; i < kSelItems; ++i)
+    if (keep[i] && dst < kb) sel[dst++] = c0 + i;
+}
+
 __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) {
   const int unit = blockIdx.x;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
@@ -165,8 +279,8 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
 }
 
 struct SelectLayout {
-  size_t budget, sel, total;
-  int sel_stride;
+  size_t budget, sel, counts, total;
+  int sel_stride, n_chunks;
 };
 
 void select_layout(const xkv_dims* d, int max_seqlen, SelectLayout* L) {
@@ -174,6 +288,8 @@ void select_layout(const xkv_dims* d, int max_seqlen, SelectLayout* L) {
   L->budget = off; off = align_up(off + (size_t)d->batch * 4, 256);
   L->sel_stride = (max_seqlen + 3) / 4 * 4;
   L->sel = off;    off = align_up(off + (size_t)d->batch * d->n_kv_heads * L->sel_stride * 4, 256);
+  L->n_chunks = (max_seqlen + kSelChunk - 1) / kSelChunk;
+  L->counts = off; off = align_up(off + (size_t)d->batch * d->n_kv_heads * L->n_chunks * 8, 256);
   L->total = off;
 }
 
@@ -226,6 +342,8 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
   p.max_pages_per_seq = c->max_pages_per_seq;
   p.n_pages = c->n_pages;
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+  p.counts = reinterpret_cast<int2*>(ws + L.counts);
+  p.n_chunks = L.n_chunks;
 
   if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;
   if (per_sequence) {
@@ -234,9 +352,20 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
     p.budget_dev = reinterpret_cast<const int32_t*>(ws + L.budget);
   }
   const int n_units = d->batch * d->n_kv_heads;
-  select_kernel<<<n_units, kSelThreads, 0, st>>>(p);
-  count_launch();
-  xkv_status s = check_launch();
+  xkv_status s;
+  if (L.n_chunks <= 1) {
+    select_kernel<<<n_units, kSelThreads, 0, st>>>(p);
+    count_launch();
+    s = check_launch();
+  } else {
+    select_count_kernel<<<dim3(n_units, L.n_chunks), kSelThreads, 0, st>>>(p);
+    count_launch();
+    s = check_launch();
+    if (s != XKV_OK) return s;
+    select_chunk_kernel<<<dim3(n_units, L.n_chunks), kSelThreads, 0, st>>>(p);
+    count_launch();
+    s = check_launch();
+  }
   if (s != XKV_OK) return s;
   if (max_keep > 0) {
     dim3 grid(n_units, (max_keep + kGatherRows - 1) / kGatherRows);

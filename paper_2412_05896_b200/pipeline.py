@@ -7,6 +7,7 @@ Every computation happens inside libxkv.so; this file allocates, copies and call
 """
 from __future__ import annotations
 
+import ctypes
 import math
 
 import numpy as np
@@ -123,6 +124,49 @@ class XkvSession:
                   self.sorted[layer] if want_curves else None, self.gains[layer] if want_curves else None,
                   mass, self.curve_len, self.ws_score[i], stream=stream)
 
+    def score_layers(self, q_win: list[torch.Tensor], k: list[torch.Tensor]) -> None:
+        """score_layer for every layer, with one fork and one join of the side streams for the whole phase (the
+        inputs of all layers must be ready on the caller's stream at the call)."""
+        cur = torch.cuda.current_stream()
+        streams = self.lanes if self.lanes else [cur]
+        for s in self.lanes:
+            s.wait_stream(cur)
+        lib, dims, cu = xkv.lib(), ctypes.byref(self.dims), self.cu.data_ptr()
+        esz = self.scores[0].numel() * 4
+        gsz = self.gains[0].numel() * 4
+        for l in range(self.L):
+            i = l % len(streams)
+            ws = self.ws_score[i]
+            st = lib.xkv_score(dims, q_win[l].data_ptr(), k[l].data_ptr(), cu, self.T, self.max_seqlen,
+                               self.scores.data_ptr() + l * esz, self.sorted.data_ptr() + l * esz,
+                               self.gains.data_ptr() + l * gsz, None, self.curve_len, ws.data_ptr(), ws.numel(),
+                               streams[i].cuda_stream)
+            if st < 0:
+                raise xkv.XkvError(st, "xkv_score")
+        self._lanes_busy = bool(self.lanes)
+        self.join()
+
+    def select_layers(self, budgets, k: list[torch.Tensor], v: list[torch.Tensor]) -> None:
+        """select_layer for every layer under one budget per layer, forked and joined once like score_layers."""
+        cur = torch.cuda.current_stream()
+        streams = self.lanes if self.lanes else [cur]
+        for s in self.lanes:
+            s.wait_stream(cur)
+        lib, dims, cu, cache = xkv.lib(), ctypes.byref(self.dims), self.cu.data_ptr(), ctypes.byref(self.cache)
+        esz = self.scores[0].numel() * 4
+        b32 = np.ascontiguousarray(budgets, dtype=np.int32)
+        for l in range(self.L):
+            i = l % len(streams)
+            ws = self.ws_select[i]
+            st = lib.xkv_select_compact(dims, l, b32.ctypes.data + 4 * l, 0, self.scores.data_ptr() + l * esz,
+                                        self.sorted.data_ptr() + l * esz, k[l].data_ptr(), v[l].data_ptr(), cu,
+                                        self.T, self.max_seqlen, cache, None, 0, ws.data_ptr(), ws.numel(),
+                                        streams[i].cuda_stream)
+            if st < 0:
+                raise xkv.XkvError(st, "xkv_select_compact")
+        self._lanes_busy = bool(self.lanes)
+        self.join()
+
     def solve_budgets(self, total: int | None = None, r_target: float = 0.0, n_min: int = 0, n_max: int = 0,
                       per_sequence: bool = False):
         """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host."""
@@ -161,16 +205,13 @@ class XkvSession:
     def prefill(self, q_win: list[torch.Tensor], k: list[torch.Tensor], v: list[torch.Tensor],
                 budgets=None, total: int | None = None, n_min: int = 0, n_max: int = 0):
         """Score every layer, split the budget (unless given), evict and compact every layer."""
-        for l in range(self.L):
-            self.score_layer(l, q_win[l], k[l])
+        self.score_layers(q_win, k)
         if budgets is None:
             budgets, _ = self.solve_budgets(total=total, n_min=n_min, n_max=n_max)
         else:
             self.budgets = np.asarray(budgets, dtype=np.int32)
         self.assign_pages(budgets)
-        for l in range(self.L):
-            self.select_layer(l, int(budgets[l]), k[l], v[l])
-        self.join()
+        self.select_layers(budgets, k, v)
         return budgets
 
     # ------------------------------------------------------------------ generation

@@ -132,12 +132,13 @@ def _cache_rows(sess, layer, b, g, n):
 
 
 @pytest.mark.parametrize("quantised", [True, False])
-@pytest.mark.parametrize("d,page_size", [(128, 16), (64, 64)])
-def test_select_compact_is_bit_exact_on_given_scores(quantised, d, page_size):
+@pytest.mark.parametrize("d,page_size,lengths", [(128, 16, [1000, 4000, 40, 12, 3100]),       # one sweep step per unit
+                                                 (64, 64, [1000, 13000, 40, 12, 4200])])      # chunked selection
+def test_select_compact_is_bit_exact_on_given_scores(quantised, d, page_size, lengths):
     """Selection and compaction alone: scores are inputs, so the kept sets must equal the oracle's
     exactly (ties to the lower position) and the cache must hold the oracle's rows bit for bit."""
     require_lib()
-    lengths, Hkv, W = [1000, 5000, 40, 12, 4200], 2, 16
+    Hkv, W = 2, 16
     B, T = len(lengths), sum(lengths)
     g = torch.Generator(device="cpu").manual_seed(11 + d)
     scores = torch.rand(Hkv, T, generator=g) ** 4
@@ -154,7 +155,7 @@ def test_select_compact_is_bit_exact_on_given_scores(quantised, d, page_size):
     v = torch.randn(T, Hkv, d, generator=g).to(torch.bfloat16)
     sess.scores[0].copy_(scores)
     sess.sorted[0].copy_(srt)
-    for budget in (0, 1, 7, 300, 984, 985, 4999, 10 ** 6):
+    for budget in (0, 1, 7, 300, 984, 985, 3999, 4183, 4184, 4185, 8200, 12983, 12984, 10 ** 6):
         sess.assign_pages([budget])
         sess.k_pages.fill_(float("nan"))
         sel = torch.full((B, Hkv, sess.max_seqlen), -1, dtype=torch.int32, device=DEV)
