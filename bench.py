@@ -207,23 +207,20 @@ def main():
     import torch.distributed as dist
 
     from paper_2412_05896_b200 import build as _build
+    from paper_2412_05896_b200 import replicas
     from paper_2412_05896_b200 import workloads as WL
     from paper_2412_05896_b200 import xkv
     from paper_2412_05896_b200.pipeline import XkvSession
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.env_ranks()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the XKV path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    replicas.init("nccl", torch.device(dev))
     if rank == 0:
         _build.build()
-    if world > 1:
-        dist.barrier()
+    replicas.barrier()
     xkv.lib()
 
     w0 = WL.CONFIGS[args.workload]
@@ -231,7 +228,7 @@ def main():
         w0 = replace(w0, decode_steps=args.decode_steps)
     if args.layers:
         w0 = replace(w0, n_layers=args.layers)
-    w = replace(w0, seed=w0.seed + 7919 * rank)          # every rank draws its own batch
+    w = replicas.replica_workload(w0, rank)              # every rank draws its own batch
     L, B, Hkv, d, W = w.n_layers, w.batch, w.n_kv_heads, w.head_dim, w.window
     lengths = WL.prompt_lengths(w)
     n_dec = w.decode_steps
@@ -365,23 +362,14 @@ def main():
     kern_ms = np.array([r[2] for r in recs])                       # [steps, n_dec]
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, dev)
 
     def sum_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return replicas.sum_over_ranks(x, dev)
 
-    dec_ms_max = max_over_ranks(dec_ms_total)
+    rate, dec_ms_max, _ = replicas.whole_job_rate(float(sum(dbytes)) * args.steps, dec_ms_total, dev)
     region_ms_max = max_over_ranks(region_ms)
-    all_bytes = sum_over_ranks(float(sum(dbytes)) * args.steps)
-    value = all_bytes / (dec_ms_max * 1e-3) / 1e9
+    value = rate / 1e9
     tokens_per_s = world * B * n_dec * args.steps / (dec_ms_max * 1e-3)
 
     # ---------------------------------------------------------------- end-to-end leg (host buffers)

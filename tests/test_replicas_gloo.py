@@ -1,0 +1,69 @@
+"""The multi-GPU mode is N independent replicas; its host-side plumbing (per-rank batches, barrier, max/sum of the
+timing, whole-job rate, rank-0-only reference arm) is exercised here with two gloo ranks on the CPU."""
+import os
+import socket
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2412_05896_b200 import replicas
+from paper_2412_05896_b200 import workloads as WL
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank: int, world: int, port: int, out):
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    r, w, local = replicas.init("gloo")
+    assert (r, w, local) == (rank, world, rank)
+    wl = replicas.replica_workload(WL.CONFIGS["llama3_8b_ragged"], rank)
+    lengths = WL.prompt_lengths(wl)
+    gathered = [None] * world
+    dist.all_gather_object(gathered, lengths)
+    # this rank processed (rank + 1) * 1000 units in 10 ms (rank 0) or 40 ms (rank 1)
+    rate, ms_max, total = replicas.whole_job_rate(1000.0 * (rank + 1), 10.0 + 30.0 * rank)
+    replicas.barrier()
+    out.put((rank, gathered, replicas.max_over_ranks(float(rank)), replicas.sum_over_ranks(float(rank + 1)), rate,
+             ms_max, total))
+    dist.destroy_process_group()
+
+
+def test_two_replicas_draw_their_own_batches_and_report_the_whole_job():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, gathered, mx, sm, rate, ms_max, total in results:
+        assert gathered[0] != gathered[1], "the ranks must not share a batch"
+        assert len(gathered[0]) == len(gathered[1]) == WL.CONFIGS["llama3_8b_ragged"].batch
+        assert mx == 1.0 and sm == 3.0
+        assert total == 3000.0 and ms_max == 40.0
+        assert abs(rate - 3000.0 / 0.040) < 1e-6       # all ranks' units over the slowest rank's time
+    # a lone process is rank 0 of 1 and the reductions are the identity
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+        os.environ.pop(k, None)
+    assert replicas.env_ranks() == (0, 1, 0)
+    assert replicas.whole_job_rate(500.0, 250.0) == (2000.0, 250.0, 500.0)
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=env, timeout=120)
+    assert res.returncode == 0 and res.stdout.strip() == ""
