@@ -8,8 +8,9 @@
 // next unit in the other half of the 512 columns.  Per unit a CTA
 //   A. streams its tiles by TMA, one tcgen05.mma chain per tile into the tile's TMEM slot; an epilogue
 //      thread owns one key, so the softmax statistics of a query row run across the lanes of a warp: the
-//      warp exchanges its 32 x 32 block by a halving butterfly (31 shuffles) and lane r keeps the running
-//      (reference, sum of exponentials) of row r.  The reference is the row maximum at the warp's first
+//      thread sums its key slot's exponentials per row over the warp's tiles, and once per unit the warp
+//      exchanges the 32 x 32 block by a halving butterfly (31 shuffles) so that lane r holds the (reference,
+//      sum of exponentials) of row r.  The reference is the row maximum at the warp's first
 //      tile and is raised only when a logit exceeds it by 2^8; it reaches the other lanes through a
 //      32-float strip of shared memory;
 //   X. sends its per-warp statistics to every CTA of the cluster with st.async into their shared memory
@@ -18,8 +19,9 @@
 //   B. reads the logits again, from TMEM, and sums exp2(s*c - normaliser[row]) over the query rows: the
 //      column score u[key] (Eq. 2 summed over the window, before pooling).  The slot is then free for the
 //      unit after next.
-// The producer and the MMA issuer run up to a whole unit ahead of the epilogue, so the keys keep streaming
-// while a cluster exchanges.  The only waits on other CTAs are those of step X, within a cluster, whose
+// The producer and the MMA issuer run up to a whole unit ahead of the epilogue, and the epilogue runs steps X
+// (the wait) and B of a unit after step A of the next one, so neither the keys nor the epilogue wait for the
+// exchange; the statistics of up to four units can sit in a CTA's shared memory.  The only waits on other CTAs are those of step X, within a cluster, whose
 // CTAs the hardware schedules together; they are bounded like every other wait here, and a CTA leaves only
 // after a cluster-wide barrier, so no store can reach the shared memory of a CTA that has gone.
 #include "tc_common.cuh"
@@ -34,6 +36,7 @@ constexpr int kSlotsPerUnit = 8;             // 128-key tiles of one unit a CTA 
 constexpr int kSlots = 2 * kSlotsPerUnit;    // x 32 columns = all 512 columns
 constexpr int kEpiAll = 2 * kEpiThreads;     // epilogue threads of a CTA
 constexpr int kClusterMax = 8;
+constexpr int kStatSlots = 4;                // units whose exchanged statistics may be in a CTA's shared memory
 constexpr float kLazyRaise = 8.f;
 
 template <int D, int CS>
@@ -44,10 +47,10 @@ struct FusedCfg {
   static constexpr int kQBytes = kHalves * kQHalfBytes;
   static constexpr int kKHalfBytes = kTcKeyTile * 128;
   static constexpr int kKTileBytes = kHalves * kKHalfBytes;
-  static constexpr int kStages = D == 128 ? 5 : 8;
-  static constexpr size_t kStatsBytes = 2 * (size_t)CS * kEpiAll * 8;      // [parity][source CTA][thread]
+  static constexpr int kStages = D == 128 ? (CS <= 4 ? 5 : 4) : 8;
+  static constexpr size_t kStatsBytes = kStatSlots * (size_t)CS * kEpiAll * 8;   // [slot][source CTA][thread]
   static constexpr size_t kSmemBytes = 1024 + (size_t)2 * kQBytes + (size_t)kStages * kKTileBytes + kStatsBytes +
-                                       2 * kRows * 4 /*row normalisers*/ + 8 * kRows * 4 /*reference strips*/ +
+                                       2 * kRows * 4 /*row normalisers*/ + 16 * kRows * 4 /*reference and rescale strips*/ +
                                        512 /*barriers*/;
 };
 
@@ -135,17 +138,18 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
   uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   uint8_t* q_s = smem;
   uint8_t* k_s = q_s + (size_t)2 * C::kQBytes;
-  float2* s_stats = reinterpret_cast<float2*>(k_s + (size_t)C::kStages * C::kKTileBytes);   // [2][CS][256]
-  float* s_mrow = reinterpret_cast<float*>(s_stats + 2 * CS * kEpiAll);                     // [2][32]
+  float2* s_stats = reinterpret_cast<float2*>(k_s + (size_t)C::kStages * C::kKTileBytes);   // [4][CS][256]
+  float* s_mrow = reinterpret_cast<float*>(s_stats + kStatSlots * CS * kEpiAll);            // [2][32]
   float* s_ref = s_mrow + 2 * kRows;                                                        // [8 warps][32]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_ref + 8 * kRows);
+  float* s_fac = s_ref + 8 * kRows;                                                         // [8 warps][32]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_fac + 8 * kRows);
   uint64_t* empty_bar = full_bar + C::kStages;
   uint64_t* qfull_bar = empty_bar + C::kStages;
   uint64_t* qempty_bar = qfull_bar + 2;
   uint64_t* resfull_bar = qempty_bar + 2;            // [kSlots] the tile's logits are complete in TMEM
   uint64_t* resempty_bar = resfull_bar + kSlots;     // [kSlots] both readings of the slot are over
-  uint64_t* stats_bar = resempty_bar + kSlots;       // [2] statistics of the whole cluster have landed here
-  uint64_t* mrow_bar = stats_bar + 2;                // [2] this CTA's row normalisers are written
+  uint64_t* stats_bar = resempty_bar + kSlots;       // [4] statistics of the whole cluster have landed here
+  uint64_t* mrow_bar = stats_bar + kStatSlots;       // [2] this CTA's row normalisers are written
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(mrow_bar + 2);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
@@ -159,9 +163,9 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
     for (int i = 0; i < 2; ++i) {
       mbar_init(&qfull_bar[i], 1);
       mbar_init(&qempty_bar[i], 1);
-      mbar_init(&stats_bar[i], 1);             // one arrival (with the expected byte count) per unit
       mbar_init(&mrow_bar[i], 8);              // one arrival per epilogue warp
     }
+    for (int i = 0; i < kStatSlots; ++i) mbar_init(&stats_bar[i], 1);   // one arrival (with the byte count) per unit
     for (int i = 0; i < kSlots; ++i) {
       mbar_init(&resfull_bar[i], 1);
       mbar_init(&resempty_bar[i], 4);          // one arrival per warp of the group that reads the slot
@@ -256,16 +260,76 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
     const uint32_t stats_base = smem_u32(s_stats), stats_bar_base = smem_u32(stats_bar);
     float* ref = s_ref + warp * kRows;
     const float4* ref4 = reinterpret_cast<const float4*>(ref);
+    float* fac = s_fac + warp * kRows;
+    const float4* fac4 = reinterpret_cast<const float4*>(fac);
     uint32_t it = 0, useq = 0, slot_uses = 0;
     UnitShape sh;
     bool ok = true;
+    // The unit whose statistics have been sent but whose column sums are still to be formed: its steps X (wait)
+    // and B run after step A of the next unit, so the exchange has a whole unit's worth of work to land behind.
+    bool have_pend = false;
+    UnitShape pend;
+    uint32_t pend_useq = 0, pend_slot0 = 0;
+    auto finish = [&](const UnitShape& u, uint32_t q, uint32_t slot0) {
+      const uint32_t st = q % kStatSlots, st_phase = (q / kStatSlots) & 1u;
+      const uint32_t par = q & 1u, phase = (q >> 1) & 1u;
+      ok = __all_sync(0xffffffffu, ws_wait(&stats_bar[st], st_phase, s_abort));
+      if (!ok) return;
+      // row normalisers: thread r < 32 merges every entry of query row r (entries r, r + 32, ... of each CTA)
+      if (eall < kRows) {
+        float m = -INFINITY, l = 0.f;
+        for (int src = 0; src < CS; ++src)
+          for (int k = eall; k < kEpiAll; k += kRows) {
+            const float2 v = s_stats[(st * CS + src) * kEpiAll + k];
+            const float m_new = fmaxf(m, v.x);
+            const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+            l = l * exp2f(m - m_ref) + v.y * exp2f(v.x - m_ref);
+            m = m_new;
+          }
+        s_mrow[par * kRows + eall] = (l > 0.f) ? m + log2f(l) : INFINITY;
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&mrow_bar[par]);
+      if (u.n1 == 0) return;
+      ok = __all_sync(0xffffffffu, ws_wait(&mrow_bar[par], phase, s_abort));
+      if (!ok) return;
+      // ---- B: column sums out of TMEM; a thread owns one key
+      float* uo = p.u + (size_t)u.g * p.total_tokens + u.cu;
+      const float4* mrow4 = reinterpret_cast<const float4*>(s_mrow + par * kRows);
+      for (int ti = (int)group; ti < u.n1; ti += 2) {
+        const uint32_t slot = slot0 + (uint32_t)ti;
+        slot_uses ^= 1u << slot;
+        if (ti < u.n2) {
+          float v[32];
+          tmem_ld32(tmem_lane + slot * kRows, v);
+          tmem_wait_ld();
+          float sum = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            const float4 mr = mrow4[i >> 2];
+            sum += fast_exp2(fmaf(v[i + 0], p.scale_log2, -mr.x)) + fast_exp2(fmaf(v[i + 1], p.scale_log2, -mr.y)) +
+                   fast_exp2(fmaf(v[i + 2], p.scale_log2, -mr.z)) + fast_exp2(fmaf(v[i + 3], p.scale_log2, -mr.w));
+          }
+          const int key = (u.tile_begin + ti) * kTcKeyTile + etid;
+          if (key < u.P) uo[key] = sum;
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&resempty_bar[slot]);
+      }
+    };
     for (int n = 0; ok && unit_shape<CS>(p, n, cluster, n_clusters, rank, &sh); ++n) {
       if (sh.t == 0) continue;                       // nothing to exchange: every CTA of the cluster skips it
-      const uint32_t par = useq & 1u, phase = (useq >> 1) & 1u;
-      ++useq;
+      const uint32_t my_useq = useq++;
+      const uint32_t st = my_useq % kStatSlots;
       const uint32_t slot0 = (it & 1u) * kSlotsPerUnit;
-      // ---- A: statistics of row `lane` over the keys of this warp
-      float r_run = -INFINITY, l_run = 0.f;          // reference (log2 domain) and sum of exponentials of row `lane`
+      if (sh.n1 > 0) ++it;
+      // ---- A: statistics of row `lane` over the keys of this warp.  The exponentials are summed per thread
+      // (one key slot, 32 rows) over the warp's tiles of the unit and exchanged across the lanes once at the end.
+      float r_run = -INFINITY;                       // reference (log2 domain) of row `lane`
+      float acc[32];                                 // this key slot's sum of exp2(x - reference[row]) per row
+#pragma unroll
+      for (int i = 0; i < 32; ++i) acc[i] = 0.f;
       bool first = true;
       for (int ti = (int)group; ti < sh.n1; ti += 2) {
         const uint32_t slot = slot0 + (uint32_t)ti;
@@ -296,17 +360,20 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
           dmax = fmaxf(fmaxf(dmax, fmaxf(y[i], y[i + 1])), fmaxf(y[i + 2], y[i + 3]));
         }
         if (__any_sync(0xffffffffu, first || dmax > kLazyRaise || r_run == -INFINITY)) {
-          // exact maximum of every row over this warp's 32 keys; lane r raises (or first sets) its reference
+          // exact maximum of every row over this warp's 32 keys; lane r raises (or first sets) its reference and
+          // tells the other lanes by how much the sums gathered so far shrink
           float tcopy[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) tcopy[i] = x[i];
           const float tmax = warp_transpose_reduce(tcopy, lane, [](float a, float b) { return fmaxf(a, b); });
+          float shrink = 1.f;
           if (tmax > r_run) {
-            l_run = (r_run == -INFINITY) ? 0.f : l_run * fast_exp2(r_run - tmax);
+            shrink = (r_run == -INFINITY) ? 1.f : fast_exp2(r_run - tmax);   // nothing was gathered under -inf
             r_run = tmax;
           }
           __syncwarp();
           ref[lane] = (r_run == -INFINITY) ? 0.f : r_run;
+          fac[lane] = shrink;
           __syncwarp();
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
@@ -316,68 +383,42 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
             y[i + 2] = x[i + 2] - r4.z;
             y[i + 3] = x[i + 3] - r4.w;
           }
+          if (!first) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              const float4 f4 = fac4[i >> 2];
+              acc[i] *= f4.x;
+              acc[i + 1] *= f4.y;
+              acc[i + 2] *= f4.z;
+              acc[i + 3] *= f4.w;
+            }
+          }
           first = false;
         }
 #pragma unroll
-        for (int i = 0; i < 32; ++i) y[i] = fast_exp2(y[i]);
-        l_run += warp_transpose_reduce(y, lane, [](float a, float b) { return a + b; });
+        for (int i = 0; i < 32; ++i) acc[i] += fast_exp2(y[i]);
       }
+      const float l_run = warp_transpose_reduce(acc, lane, [](float a, float b) { return a + b; });
       if (!ok) break;
-      // ---- X: the statistics of row `lane` from this warp go to slot [par][rank][eall] of every CTA of the cluster
-      if (eall == 0) mbar_arrive_expect_tx(&stats_bar[par], (uint32_t)(CS * kEpiAll * 8));
+      // ---- X: the statistics of row `lane` from this warp go to slot [st][rank][eall] of every CTA of the cluster
+      if (eall == 0) mbar_arrive_expect_tx(&stats_bar[st], (uint32_t)(CS * kEpiAll * 8));
       {
-        const uint32_t slot = stats_base + (uint32_t)(((par * CS + rank) * kEpiAll + eall) * 8);
-        const uint32_t bar = stats_bar_base + par * 8u;
+        const uint32_t slot = stats_base + (uint32_t)(((st * CS + rank) * kEpiAll + eall) * 8);
+        const uint32_t bar = stats_bar_base + st * 8u;
 #pragma unroll
         for (uint32_t dst = 0; dst < (uint32_t)CS; ++dst)
           st_async_f2(map_to_rank(slot, dst), r_run, l_run, map_to_rank(bar, dst));
       }
-      ok = __all_sync(0xffffffffu, ws_wait(&stats_bar[par], phase, s_abort));
-      if (!ok) break;
-      // row normalisers: thread r < 32 merges every entry of query row r (entries r, r + 32, ... of each CTA)
-      if (eall < kRows) {
-        float m = -INFINITY, l = 0.f;
-        for (int src = 0; src < CS; ++src)
-          for (int k = eall; k < kEpiAll; k += kRows) {
-            const float2 v = s_stats[(par * CS + src) * kEpiAll + k];
-            const float m_new = fmaxf(m, v.x);
-            const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-            l = l * exp2f(m - m_ref) + v.y * exp2f(v.x - m_ref);
-            m = m_new;
-          }
-        s_mrow[par * kRows + eall] = (l > 0.f) ? m + log2f(l) : INFINITY;
+      if (have_pend) {
+        finish(pend, pend_useq, pend_slot0);
+        if (!ok) break;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&mrow_bar[par]);
-      if (sh.n1 == 0) continue;
-      ok = __all_sync(0xffffffffu, ws_wait(&mrow_bar[par], phase, s_abort));
-      if (!ok) break;
-      // ---- B: column sums out of TMEM; a thread owns one key
-      float* u = p.u + (size_t)sh.g * p.total_tokens + sh.cu;
-      const float4* mrow4 = reinterpret_cast<const float4*>(s_mrow + par * kRows);
-      for (int ti = (int)group; ti < sh.n1; ti += 2) {
-        const uint32_t slot = slot0 + (uint32_t)ti;
-        slot_uses ^= 1u << slot;
-        if (ti < sh.n2) {
-          float v[32];
-          tmem_ld32(tmem_lane + slot * kRows, v);
-          tmem_wait_ld();
-          float acc = 0.f;
-#pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            const float4 mr = mrow4[i >> 2];
-            acc += fast_exp2(fmaf(v[i + 0], p.scale_log2, -mr.x)) + fast_exp2(fmaf(v[i + 1], p.scale_log2, -mr.y)) +
-                   fast_exp2(fmaf(v[i + 2], p.scale_log2, -mr.z)) + fast_exp2(fmaf(v[i + 3], p.scale_log2, -mr.w));
-          }
-          const int key = (sh.tile_begin + ti) * kTcKeyTile + etid;
-          if (key < sh.P) u[key] = acc;
-        }
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&resempty_bar[slot]);
-      }
-      ++it;
+      pend = sh;
+      pend_useq = my_useq;
+      pend_slot0 = slot0;
+      have_pend = true;
     }
+    if (ok && have_pend) finish(pend, pend_useq, pend_slot0);
   }
 
   // ---- teardown
