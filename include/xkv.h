@@ -7,6 +7,7 @@
  *                         scores per KV head, their descending sort, and the layer's
  *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
  *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
+ *      xkv_average_budgets  host: the averaged list of the online scenario           (Sec. IV-D)
  *   3. xkv_select_compact per layer: top-k per (sequence, KV head) and gather of the kept K/V
  *                         rows into a ragged paged cache                             (Alg. 2 steps 5-7)
  *   4. xkv_decode_attn    per generation step: attention over the ragged compacted caches,
@@ -149,6 +150,23 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
                              int32_t curve_len, const int32_t* prefix_len, int32_t per_sequence,
                              int64_t total, double r_target, int32_t n_min, int32_t n_max,
                              int32_t* budgets, double* r_avg);
+
+/*
+ * xkv_average_budgets -- the averaged allocation list of the online scenario (Sec. IV-D), host only.
+ *
+ * The lists that xkv_alloc_budgets produced for a sample of tasks of one type are averaged layer by
+ * layer; later tasks of that type skip the allocation and are evicted under the averaged list.
+ *
+ * lists      host int32 [n_tasks][n_layers], every entry >= 0
+ * out        host out int32 [n_layers]
+ *
+ * The paper leaves the rounding open. Here every layer gets the floor of its mean, and the slots that
+ * leaves over -- up to the mean of the recorded totals rounded half up -- go one each to the layers with
+ * the largest fractional parts, the lower layer first among equals; lists that all add up to N therefore
+ * give a list that adds up to N. Errors: XKV_ERR_INVALID_ARG for null pointers, non-positive counts or a
+ * negative entry.
+ */
+xkv_status xkv_average_budgets(const int32_t* lists, int32_t n_tasks, int32_t n_layers, int32_t* out);
 
 /*
  * xkv_select_compact -- top-k and eviction of one layer (Alg. 2 steps 5-7).

@@ -237,6 +237,30 @@ def allocation_objective(gains: list[np.ndarray], List_A: list[int]) -> float:
     return sum(float(np.sum(np.asarray(g[:n], dtype=np.float64))) for g, n in zip(gains, List_A)) / len(gains)
 
 
+def averaged_allocation(lists: list[list[int]]) -> list[int]:
+    """Online scenario (Sec. IV-D): the allocation lists recorded for the sampled tasks are averaged layer by
+    layer and the averaged list is applied to later tasks of the same type.
+
+    The paper does not say how the averages become integers.  Reading taken here: every layer gets the floor of
+    its mean, and the slots this leaves over (so that the list adds up to the rounded mean of the recorded
+    totals) go one each to the layers with the largest fractional parts, lower layer first among equals.
+    Exact integer arithmetic throughout.
+    """
+    n = len(lists)
+    L = len(lists[0])
+    sums = [sum(int(lst[i]) for lst in lists) for i in range(L)]
+    base = [s // n for s in sums]
+    rem = [s % n for s in sums]                       # fractional part of layer i's mean is rem[i] / n
+    total = sum(sums)
+    target = (2 * total + n) // (2 * n)               # mean of the recorded totals, rounded half up
+    left = target - sum(base)
+    order = sorted(range(L), key=lambda i: (-rem[i], i))
+    out = list(base)
+    for i in order[:left]:
+        out[i] += 1
+    return out
+
+
 def bruteforce_allocation(gains: list[np.ndarray], N: int, n_min: int = 0,
                           n_max: int | None = None) -> tuple[list[int], float]:
     """Enumerate every split of N over the layers (tiny inputs only) and return the best of Eq. 17."""

@@ -417,4 +417,30 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
   return XKV_OK;
 }
 
+xkv_status xkv_average_budgets(const int32_t* lists, int32_t n_tasks, int32_t n_layers, int32_t* out) {
+  if (lists == nullptr || out == nullptr || n_tasks <= 0 || n_layers <= 0) return XKV_ERR_INVALID_ARG;
+  std::vector<int64_t> sums(n_layers, 0);
+  int64_t total = 0;
+  for (int t = 0; t < n_tasks; ++t)
+    for (int l = 0; l < n_layers; ++l) {
+      const int32_t v = lists[(size_t)t * n_layers + l];
+      if (v < 0) return XKV_ERR_INVALID_ARG;
+      sums[l] += v;
+      total += v;
+    }
+  const int64_t n = n_tasks;
+  const int64_t target = (2 * total + n) / (2 * n);          // mean of the recorded totals, rounded half up
+  int64_t given = 0;
+  std::vector<std::pair<int64_t, int>> frac(n_layers);        // (remainder of the division by n, layer)
+  for (int l = 0; l < n_layers; ++l) {
+    out[l] = (int32_t)(sums[l] / n);
+    given += out[l];
+    frac[l] = {sums[l] % n, l};
+  }
+  std::stable_sort(frac.begin(), frac.end(),
+                   [](const std::pair<int64_t, int>& a, const std::pair<int64_t, int>& b) { return a.first > b.first; });
+  for (int64_t i = 0; i < target - given && i < n_layers; ++i) out[frac[(size_t)i].second] += 1;
+  return XKV_OK;
+}
+
 }  // extern "C"

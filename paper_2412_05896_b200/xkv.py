@@ -22,7 +22,7 @@ OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
+EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
            "xkv_workspace_bytes",
            "xkv_read_device_status", "xkv_profile_events", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
     L.xkv_score.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, vp, vp, vp, i32, vp, sz, vp]
     L.xkv_alloc_budgets.restype = i32
     L.xkv_alloc_budgets.argtypes = [vp, i32, i32, i32, vp, i32, i64, ctypes.c_double, i32, i32, vp, vp]
+    L.xkv_average_budgets.restype = i32
+    L.xkv_average_budgets.argtypes = [vp, i32, i32, vp]
     L.xkv_select_compact.restype = i32
     L.xkv_select_compact.argtypes = [ctypes.POINTER(Dims), i32, vp, i32, vp, vp, vp, vp, vp, i64, i32,
                                      ctypes.POINTER(Cache), vp, i32, vp, sz, vp]
@@ -162,6 +164,15 @@ def alloc_budgets(gains: np.ndarray, prefix_len, per_sequence: bool = False, tot
                                    int(total), float(r_target), n_min, n_max, budgets.ctypes.data,
                                    r_avg.ctypes.data), "xkv_alloc_budgets")
     return budgets, (r_avg if per_sequence else float(r_avg[0]))
+
+
+def average_budgets(lists) -> np.ndarray:
+    """lists: int [n_tasks, n_layers] recorded by alloc_budgets for sampled tasks -> the averaged list [n_layers]."""
+    lists = np.ascontiguousarray(lists, dtype=np.int32)
+    n_tasks, L = lists.shape
+    out = np.zeros(L, dtype=np.int32)
+    _check(lib().xkv_average_budgets(lists.ctypes.data, n_tasks, L, out.ctypes.data), "xkv_average_budgets")
+    return out
 
 
 def select_compact(dims: Dims, layer: int, budget, per_sequence: bool, scores, sorted_scores, k, v, cu_seqlens,

@@ -167,3 +167,23 @@ def test_alloc_budgets_ties_and_unsorted_curves(seed):
         budgets, r = xkv.alloc_budgets(u, [n], total=N, n_min=2)
         A, r_o = O.adaptive_allocation([u[l, 0].astype(np.float64) for l in range(L)], N=N, n_min=2)
         assert budgets.tolist() == A and abs(r - r_o) < 1e-12
+
+
+def test_average_budgets_matches_oracle_and_keeps_the_total():
+    """Online scenario (Sec. IV-D): layer-wise average of the recorded lists."""
+    # by hand: means 4, 14/3, 22/3; recorded totals 16 each -> floors 4, 4, 7 and one slot to the larger fraction 2/3
+    assert O.averaged_allocation([[3, 5, 8], [4, 4, 8], [5, 5, 6]]) == [4, 5, 7]
+    assert xkv.average_budgets([[3, 5, 8], [4, 4, 8], [5, 5, 6]]).tolist() == [4, 5, 7]
+    assert xkv.average_budgets([[1, 1], [2, 2]]).tolist() == [2, 1]            # equal fractions: the lower layer
+    rng = np.random.default_rng(5)
+    for n_tasks, L, N in [(1, 8, 100), (3, 32, 16384), (7, 5, 33), (10, 32, 65536)]:
+        lists = rng.multinomial(N, rng.dirichlet(np.ones(L)), size=n_tasks)
+        got = xkv.average_budgets(lists)
+        assert got.tolist() == O.averaged_allocation(lists.tolist())
+        assert got.sum() == N                                                   # every recorded list adds up to N
+        mean = lists.mean(axis=0)
+        assert np.all(got >= np.floor(mean)) and np.all(got <= np.floor(mean) + 1)
+        if n_tasks == 1:
+            assert got.tolist() == lists[0].tolist()
+    with pytest.raises(xkv.XkvError):
+        xkv.average_budgets([[1, -1]])

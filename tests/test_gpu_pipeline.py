@@ -146,6 +146,32 @@ def test_full_budget_reproduces_full_attention():
     assert sess.seq_lens.cpu().numpy().tolist() == [[lengths[0] + 1]] * w.n_layers
 
 
+def test_online_scenario_averaged_list_applied_to_a_new_task():
+    """Sec. IV-D: allocation lists recorded on a few sampled tasks are averaged, and a later task of the same type
+    is evicted under the averaged list without running the allocation.  Uses the paper's own defaults (observation
+    window 8, average pooling of size 7)."""
+    require_lib()
+    base = replace(WL.CONFIGS["mistral_7b_gqa"], n_layers=4, n_q_heads=8, n_kv_heads=2, batch=1, prompt=1500,
+                   window=8, pool_kernel=7, pool_mode=1, avg_budget=160, n_min=16, n_max=600, decode_steps=2)
+    N = base.n_layers * base.avg_budget
+    recorded = []
+    for task in range(3):
+        w = replace(base, seed=base.seed + 31 * (task + 1))
+        lengths = WL.prompt_lengths(w)
+        sess = XkvSession(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.window, w.pool_kernel, lengths,
+                          pool_mode=w.pool_mode, max_budget=w.n_max, total_budget=N, curve_len=w.n_max, device=DEV)
+        tens = [WL.layer_tensors(w, l, DEV, lengths) for l in range(w.n_layers)]
+        sess.score_layers([t[0] for t in tens], [t[1] for t in tens])
+        budgets, _ = sess.solve_budgets(total=N, n_min=w.n_min, n_max=w.n_max)
+        assert sess.device_status("score") == xkv.OK and budgets.sum() == N
+        recorded.append(budgets.tolist())
+    averaged = xkv.average_budgets(recorded)
+    assert averaged.tolist() == O.averaged_allocation(recorded) and averaged.sum() == N
+    assert len({tuple(r) for r in recorded}) > 1, "the sampled tasks should not all give the same list"
+    # a new task of the same type: no allocation, eviction under the averaged list, then generation
+    run_path(replace(base, seed=base.seed + 1000, budgets=tuple(int(x) for x in averaged)), stress=True)
+
+
 def test_deterministic_across_runs():
     w = SCALED["ragged"]
     a, _, _ = run_path(w, False)
