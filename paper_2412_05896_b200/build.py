@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every CUDA source into paper_2412_05896_b200/libxkv.so; returns its path."""
     if not force and not is_stale():
         return LIB
-    cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+    cmd = [_nvcc(), "--threads", "0", "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
