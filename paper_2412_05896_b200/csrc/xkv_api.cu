@@ -385,7 +385,9 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
       }
     };
     // the batch mean reads every curve once: spread the layers over a few threads when that is megabytes
-    int n_threads = (int)std::min<size_t>(8, (size_t)n_layers * lstride / (1u << 20));
+    int n_threads = (int)std::min<size_t>(8, (size_t)n_layers * lstride / (4u << 20));
+    const int hw = (int)std::thread::hardware_concurrency();
+    if (hw > 0 && n_threads > hw) n_threads = hw;
     if (n_threads > n_layers) n_threads = n_layers;
     if (n_threads <= 1) {
       mean_layers(0, n_layers);
