@@ -42,7 +42,7 @@ extern "C" {
 typedef int32_t xkv_status;
 #define XKV_OK               0
 #define XKV_ERR_INVALID_ARG (-1) /* null/misaligned pointer, non-positive size, inconsistent dims    */
-#define XKV_ERR_UNSUPPORTED (-2) /* head_dim not in {64,128}, G*W not a multiple of 16 or > 256, ... */
+#define XKV_ERR_UNSUPPORTED (-2) /* head_dim not in {64,128}, G*W > 256, ... */
 #define XKV_ERR_WORKSPACE   (-3) /* workspace_bytes smaller than xkv_workspace_bytes() reports        */
 #define XKV_ERR_BUDGET      (-4) /* negative budget, total beyond capacity, unreachable R target      */
 #define XKV_ERR_CUDA        (-5) /* a CUDA runtime/driver call or a launch failed                     */
@@ -62,7 +62,7 @@ typedef struct xkv_dims {
   int32_t n_q_heads;     /* Hq                                                                 */
   int32_t n_kv_heads;    /* Hkv, divides Hq                                                    */
   int32_t head_dim;      /* d, 64 or 128                                                       */
-  int32_t window;        /* W = ows, observation-window size (Eq. 3); G*W multiple of 16, <=256 */
+  int32_t window;        /* W = ows, observation-window size (Eq. 3); G*W <= 256 */
   int32_t pool_kernel;   /* ps, odd, 1..63 (Alg. 2 step 4); 1 = no pooling                     */
   int32_t pool_mode;     /* XKV_POOL_MAX or XKV_POOL_AVG                                       */
   float   scale;         /* logit scale; 0 selects 1/sqrt(d) (Eq. 2)                           */

@@ -24,6 +24,7 @@ struct ScoreParams {
   int32_t slice_tiles, n_work;
   int64_t total_tokens, stride_token, stride_head;
   int32_t batch, n_q_heads, n_kv_heads, group, window, M, pool_kernel, pool_mode;
+  int32_t M_real;      // G*W; M is M_real rounded up to a multiple of 16 (the padding rows never contribute)
   int32_t split_keys, n_splits, n_chunks, curve_len;
   float scale_log2;
 };

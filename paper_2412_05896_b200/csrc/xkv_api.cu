@@ -51,7 +51,7 @@ xkv_status check_prefill_dims(const xkv_dims* d) {
   if (d->pool_kernel < 1 || d->pool_kernel > 63 || d->pool_kernel % 2 == 0) return XKV_ERR_INVALID_ARG;
   if (d->pool_mode != XKV_POOL_MAX && d->pool_mode != XKV_POOL_AVG) return XKV_ERR_INVALID_ARG;
   const int64_t rows = (int64_t)(d->n_q_heads / d->n_kv_heads) * d->window;
-  if (rows % 16 != 0 || rows > 256) return XKV_ERR_UNSUPPORTED;
+  if (rows < 1 || rows > 256) return XKV_ERR_UNSUPPORTED;
   if (d->kv_stride_head < d->head_dim || d->kv_stride_head % 8 != 0) return XKV_ERR_INVALID_ARG;
   if (d->kv_stride_token < (int64_t)d->n_kv_heads * d->head_dim || d->kv_stride_token % 8 != 0)
     return XKV_ERR_INVALID_ARG;

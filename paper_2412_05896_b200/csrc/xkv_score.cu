@@ -90,7 +90,8 @@ __device__ __forceinline__ void load_q(const ScoreParams& p, const UnitShape& us
   const __nv_bfloat16* qg = p.q_win + ((size_t)us.b * p.n_q_heads + (size_t)us.g * p.group) * p.window * D;
   for (int idx = threadIdx.x; idx < p.M * kChunks; idx += kPassThreads) {
     const int r = idx / kChunks, c = idx % kChunks;
-    cp_async_16(smem_u32(q_s) + swz(r, c, D * 2), qg + (size_t)r * D + c * 8, 16);
+    const bool real = r < p.M_real;               // rows that only pad G*W to a multiple of 16 are zero-filled
+    cp_async_16(smem_u32(q_s) + swz(r, c, D * 2), qg + (size_t)(real ? r : 0) * D + c * 8, real ? 16 : 0);
   }
 }
 
@@ -259,7 +260,8 @@ __device__ __forceinline__ void publish_stats(const ScoreParams& p, const UnitSh
           const float2 v = __ldcg(&part[(size_t)s * M]);
           l += v.y * exp2f(v.x - m);
         }
-      p.mrow[(size_t)unit * M + r] = (l > 0.f) ? m + log2f(l) : INFINITY;
+      // a normaliser of +inf makes a row contribute exp2(-inf) = 0: rows without visible keys, padding rows
+      p.mrow[(size_t)unit * M + r] = (l > 0.f && r < p.M_real) ? m + log2f(l) : INFINITY;
     }
     __threadfence();
     __syncthreads();
@@ -661,7 +663,8 @@ struct ScoreLayout {
 
 void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) {
   const int units = d->batch * d->n_kv_heads;
-  const int M = (d->n_q_heads / d->n_kv_heads) * d->window;
+  const int M_real = (d->n_q_heads / d->n_kv_heads) * d->window;
+  const int M = (M_real + 15) / 16 * 16;
   const int sms = sm_count();
   // Resident variant: key tiles per split chosen so that two CTAs fit on an SM (one for G*W = 256).
   int tiles = M <= 64 ? 3 : (M <= 128 ? 2 : 4);
@@ -688,7 +691,7 @@ void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) 
     L->ctas_per_sm = ctas_for(fixed + kPassStages * tile_bytes);
   }
   // the tcgen05 kernel takes the passes over when it covers the shape (it is a resident variant too)
-  const int tc_split = score_tc_split_keys(M, d->head_dim, units, max_seqlen);
+  const int tc_split = M_real == M ? score_tc_split_keys(M, d->head_dim, units, max_seqlen) : 0;
   L->use_tc = tc_split > 0;
   if (L->use_tc) {
     L->resident = true;            // one work item per (unit, split); the kernel runs as two launches
@@ -772,7 +775,8 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
   p.n_kv_heads = d->n_kv_heads;
   p.group = d->n_q_heads / d->n_kv_heads;
   p.window = d->window;
-  p.M = p.group * d->window;
+  p.M_real = p.group * d->window;
+  p.M = (p.M_real + 15) / 16 * 16;
   p.pool_kernel = d->pool_kernel;
   p.pool_mode = d->pool_mode;
   p.split_keys = L.split_keys;

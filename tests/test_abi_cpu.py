@@ -45,7 +45,8 @@ def test_workspace_sizes_and_rejections():
     forced = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, d, n_layers=4, max_cache_len=4096, chunk_rows=64)
     assert auto > 0 and forced > 0
     lib = xkv.lib()
-    for bad in (_dims(head_dim=96), _dims(window=3), _dims(n_kv_heads=3), _dims(pool_kernel=4),
+    assert xkv.workspace_bytes(xkv.OP_SCORE, _dims(window=3), max_seqlen=1000, total_tokens=1500) > 0   # rows are padded
+    for bad in (_dims(head_dim=96), _dims(window=0), _dims(n_kv_heads=3), _dims(pool_kernel=4),
                 _dims(window=128)):
         assert lib.xkv_workspace_bytes(xkv.OP_SCORE, ctypes.byref(bad), 100, 100, 0, 0, 0) == 0
     assert lib.xkv_workspace_bytes(99, ctypes.byref(d), 100, 100, 1, 1, 0) == 0

@@ -67,6 +67,8 @@ CASES = [
     ([33, 17, 16, 1], 2, 1, 64, 16, 1, 0),       # at and below the window length
     ([8192, 4500, 130], 2, 2, 128, 32, 7, 0),    # G*W = 32, single-read kernel with clusters of eight
     ([4096, 31, 32, 33, 160], 3, 3, 64, 32, 5, 1),   # G*W = 32, clusters of four, lengths around the window
+    ([300, 1000, 5], 4, 4, 64, 8, 7, 1),         # G*W = 8 (MHA with the paper's window of 8): padded to 16 rows
+    ([700, 129], 6, 2, 128, 8, 7, 0),            # G*W = 24: padded to 32 rows
 ]
 
 
