@@ -195,6 +195,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the uncompressed-cache decode comparison")
+    ap.add_argument("--lanes", type=int, default=None, help="side streams of the scoring and eviction phases")
     ap.add_argument("--chunk-rows", type=int, default=0, help="decode chunk size (0 = chosen on the device)")
     ap.add_argument("--layers", type=int, default=None, help="override the number of layers (small profiling cases)")
     args = ap.parse_args()
@@ -240,7 +241,8 @@ def main():
     N_total = None if w.budgets is not None else L * w.avg_budget
     sess = XkvSession(L, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
                       max_new_tokens=n_dec, max_budget=w.n_max or None, total_budget=N_total,
-                      curve_len=w.n_max or None, device=dev, decode_chunk_rows=args.chunk_rows)
+                      curve_len=w.n_max or None, device=dev, decode_chunk_rows=args.chunk_rows,
+                      **({} if args.lanes is None else {"n_lanes": args.lanes}))
     prefix = sess.prefix
 
     ev = lambda: torch.cuda.Event(enable_timing=True)

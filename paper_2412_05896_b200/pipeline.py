@@ -21,7 +21,7 @@ class XkvSession:
                  pool_kernel: int, lengths: list[int], pool_mode: int = xkv.POOL_MAX, page_size: int = 16,
                  max_new_tokens: int = 0, max_budget: int | None = None, total_budget: int | None = None,
                  curve_len: int | None = None, device="cuda:0", scale: float = 0.0,
-                 decode_chunk_rows: int = 0, n_lanes: int = 2):
+                 decode_chunk_rows: int = 0, n_lanes: int = 3):
         self.L, self.Hq, self.Hkv, self.d, self.W = n_layers, n_q_heads, n_kv_heads, head_dim, window
         self.B = len(lengths)
         self.lengths = list(lengths)
