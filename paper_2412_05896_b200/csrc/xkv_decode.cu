@@ -313,6 +313,8 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       __threadfence();
     }
     if (!__syncthreads_and(met)) return;
+    // the rows other CTAs stored with ordinary writes are read below by TMA (the asynchronous proxy)
+    asm volatile("fence.proxy.async.global;" ::: "memory");
     // the plan, computed by every CTA for itself: chunk size from the total length, then the number of chunks
     // before each unit (and the list of units with more than one)
     constexpr int kPer = kMaxPlanUnits / kAttnThreads;
