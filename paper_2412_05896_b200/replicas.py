@@ -63,3 +63,20 @@ def whole_job_rate(units_local: float, ms_local: float, device="cpu") -> tuple[f
     ms_max = max_over_ranks(ms_local, device)
     total = sum_over_ranks(units_local, device)
     return total / (ms_max * 1e-3), ms_max, total
+
+
+def batch_mean_curves_over_ranks(gains, device="cpu"):
+    """One budget list for the sequences of all ranks (instead of one list per replica): the curves the solver
+    averages over a batch are averaged over every rank's batch.  gains: float [L, B_local, curve_len] as written by
+    xkv_score (torch tensor or array; every rank must use the same L and curve_len).  Returns a torch float64
+    tensor [L, 1, curve_len] that xkv.alloc_budgets takes as a batch of one: the mean over all sequences of the
+    job.  This is the only exchange a sharded run of the path needs -- L x curve_len numbers, before the host
+    solver; K, V and the scores never leave their GPU.
+    """
+    g = torch.as_tensor(gains).to(device=device, dtype=torch.float64)
+    total = g.sum(dim=1, keepdim=True)
+    count = torch.tensor([float(g.shape[1])], device=device, dtype=torch.float64)
+    if dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(total, op=dist.ReduceOp.SUM)
+        dist.all_reduce(count, op=dist.ReduceOp.SUM)
+    return total / count

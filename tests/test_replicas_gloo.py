@@ -62,6 +62,43 @@ def test_two_replicas_draw_their_own_batches_and_report_the_whole_job():
     assert replicas.whole_job_rate(500.0, 250.0) == (2000.0, 250.0, 500.0)
 
 
+def _curve_worker(rank: int, world: int, port: int, out):
+    import numpy as np
+    from oracle import xkv_oracle as O
+    from paper_2412_05896_b200 import xkv
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    replicas.init("gloo")
+    L, n = 5, 40
+    b_local = 2 + rank                                    # the ranks hold batches of different size
+    rng = np.random.default_rng(77)
+    all_curves = np.stack([[O.head_gains(rng.random(n) ** (2 + l)) for _ in range(5)] for l in range(L)])   # [L, 5, n]
+    mine = all_curves[:, :2] if rank == 0 else all_curves[:, 2:]
+    assert mine.shape[1] == b_local
+    shared = replicas.batch_mean_curves_over_ranks(mine.astype(np.float32)).numpy()
+    budgets, r = xkv.alloc_budgets(shared.astype(np.float32), [n], total=60, n_min=2)
+    whole, r_whole = xkv.alloc_budgets(all_curves.astype(np.float32), [n] * 5, total=60, n_min=2)
+    out.put((rank, budgets.tolist(), whole.tolist(), float(np.abs(shared[:, 0] - all_curves.astype(np.float32).mean(1)).max())))
+    dist.destroy_process_group()
+
+
+def test_budget_list_shared_by_all_ranks_equals_the_list_of_the_whole_batch():
+    """The one exchange of a sharded run: curves averaged over every rank's sequences before the solver."""
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_curve_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert results[0][1] == results[1][1], "every rank must derive the same list"
+    for rank, budgets, whole, err in results:
+        assert budgets == whole and sum(budgets) == 60 and err < 1e-6
+
+
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
