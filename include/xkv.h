@@ -211,6 +211,10 @@ xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t
  * chunk_rows 0 = chosen on the device from the cache lengths; otherwise a multiple of 64
  * workspace  dev, at least xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...) bytes
  * Device status XKV_ERR_CAPACITY if an append does not fit its page table (that row is skipped).
+ * Launches: up to 2048 (layer, sequence) units the call is one small memset and one kernel, launched
+ * cooperatively with one block per SM (the blocks append, meet once and plan their work themselves),
+ * so the device must be able to hold that grid at once -- other work on the GPU delays the launch, it
+ * does not break it. Larger problems run a separate append-and-plan kernel first.
  */
 xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin,
                            int32_t layer_end, const void* q, const void* k_new, const void* v_new,
