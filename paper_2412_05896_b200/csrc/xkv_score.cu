@@ -554,6 +554,26 @@ __device__ __forceinline__ int merge_path(const float* A, int la, const float* B
   return lo;
 }
 
+// The same split point found by a whole warp: 32 probes per round instead of one, so a run of 64K scores takes four
+// rounds of global loads instead of sixteen.  All lanes return the result.
+__device__ __forceinline__ int merge_path_warp(const float* A, int la, const float* B, int lb, int diag) {
+  const int lane = threadIdx.x & 31;
+  int lo = max(0, diag - lb), hi = min(diag, la);
+  while (lo < hi) {
+    const int step = (hi - lo + 31) / 32;
+    const int q = lo + (lane + 1) * step - 1;                 // probe positions, ascending with the lane
+    const bool in = q < hi;
+    const bool ge = in && A[q] >= B[diag - 1 - q];            // true on a prefix of the lanes
+    const unsigned m = __ballot_sync(0xffffffffu, ge);
+    const int c = __popc(m);                                   // the split lies beyond the first c probes
+    const int q_c = lo + (c + 1) * step - 1;                   // first probe that failed (if it exists)
+    lo = lo + c * step;
+    if (c < 32 && q_c < hi) hi = q_c;
+    if (lo > hi) lo = hi;
+  }
+  return lo;
+}
+
 __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const ScoreParams p, const float* src, float* dst,
                                                              int run) {
   __shared__ float s_in[kMergeTile];
@@ -573,7 +593,11 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const ScoreParams 
   const float* B = A + run;
   const int d0 = o0 - pair0;
   const int d1 = min(d0 + kMergeTile, la + lb);
-  if (threadIdx.x < 2) s_split[threadIdx.x] = merge_path(A, la, B, lb, threadIdx.x == 0 ? d0 : d1);
+  if (threadIdx.x < 64) {                      // warp 0 finds the tile's start, warp 1 its end
+    const int w = threadIdx.x >> 5;
+    const int split = merge_path_warp(A, la, B, lb, w == 0 ? d0 : d1);
+    if ((threadIdx.x & 31) == 0) s_split[w] = split;
+  }
   __syncthreads();
   const int a0 = s_split[0], a1 = s_split[1];
   const int b0 = d0 - a0, b1 = d1 - a1;
