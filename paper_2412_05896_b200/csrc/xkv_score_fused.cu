@@ -341,8 +341,6 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
         tmem_wait_ld();
         const int key = (sh.tile_begin + ti) * kTcKeyTile + etid;
         const bool masked = key + p.window >= sh.t;          // a window key (causal inside the window) or past the end
-#pragma unroll
-        for (int i = 0; i < 32; ++i) x[i] *= p.scale_log2;
         if (masked) {
           const int lim0 = sh.t - p.window;                  // row i sees the keys up to lim0 + i % W
 #pragma unroll
@@ -353,10 +351,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
           const float4 r4 = ref4[i >> 2];
-          y[i] = x[i] - r4.x;
-          y[i + 1] = x[i + 1] - r4.y;
-          y[i + 2] = x[i + 2] - r4.z;
-          y[i + 3] = x[i + 3] - r4.w;
+          y[i] = fmaf(x[i], p.scale_log2, -r4.x);            // raw logit * (log2 e / sqrt(d)) - reference
+          y[i + 1] = fmaf(x[i + 1], p.scale_log2, -r4.y);
+          y[i + 2] = fmaf(x[i + 2], p.scale_log2, -r4.z);
+          y[i + 3] = fmaf(x[i + 3], p.scale_log2, -r4.w);
           dmax = fmaxf(fmaxf(dmax, fmaxf(y[i], y[i + 1])), fmaxf(y[i + 2], y[i + 3]));
         }
         if (__any_sync(0xffffffffu, first || dmax > kLazyRaise || r_run == -INFINITY)) {
@@ -364,7 +362,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
           // tells the other lanes by how much the sums gathered so far shrink
           float tcopy[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) tcopy[i] = x[i];
+          for (int i = 0; i < 32; ++i) tcopy[i] = x[i] * p.scale_log2;
           const float tmax = warp_transpose_reduce(tcopy, lane, [](float a, float b) { return fmaxf(a, b); });
           float shrink = 1.f;
           if (tmax > r_run) {
@@ -378,10 +376,10 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
             const float4 r4 = ref4[i >> 2];
-            y[i] = x[i] - r4.x;
-            y[i + 1] = x[i + 1] - r4.y;
-            y[i + 2] = x[i + 2] - r4.z;
-            y[i + 3] = x[i + 3] - r4.w;
+            y[i] = fmaf(x[i], p.scale_log2, -r4.x);
+            y[i + 1] = fmaf(x[i + 1], p.scale_log2, -r4.y);
+            y[i + 2] = fmaf(x[i + 2], p.scale_log2, -r4.z);
+            y[i + 3] = fmaf(x[i + 3], p.scale_log2, -r4.w);
           }
           if (!first) {
 #pragma unroll
