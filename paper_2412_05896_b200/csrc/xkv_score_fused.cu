@@ -21,9 +21,10 @@
 //      unit after next.
 // The producer and the MMA issuer run up to a whole unit ahead of the epilogue, and the epilogue runs steps X
 // (the wait) and B of a unit after step A of the next one, so neither the keys nor the epilogue wait for the
-// exchange; the statistics of up to four units can sit in a CTA's shared memory.  The only waits on other CTAs are those of step X, within a cluster, whose
-// CTAs the hardware schedules together; they are bounded like every other wait here, and a CTA leaves only
-// after a cluster-wide barrier, so no store can reach the shared memory of a CTA that has gone.
+// exchange; the statistics of up to four units can sit in a CTA's shared memory.  The only waits on other
+// CTAs are those of step X, within a cluster, whose CTAs the hardware schedules together; they are bounded
+// like every other wait here, and a CTA leaves only after a cluster-wide barrier, so no store can reach the
+// shared memory of a CTA that has gone.
 #include "tc_common.cuh"
 
 namespace xkv {
