@@ -7,7 +7,7 @@
  *                         scores per KV head, their descending sort, and the layer's
  *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
  *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
- *      xkv_average_budgets  host: the averaged list of the online scenario           (Sec. IV-D)
+ *      xkv_average_budgets  host: the averaged list of the online scenario           (Sec. IV-C)
  *   3. xkv_select_compact per layer: top-k per (sequence, KV head) and gather of the kept K/V
  *                         rows into a ragged paged cache                             (Alg. 2 steps 5-7)
  *   4. xkv_decode_attn    per generation step: attention over the ragged compacted caches,
@@ -22,8 +22,13 @@
  *   - Device pointers must be 16-byte aligned; violations are rejected with XKV_ERR_INVALID_ARG.
  *   - Arguments are validated on the host and rejected before anything is enqueued. A negative
  *     return value means nothing was launched. Conditions only the device can see (a cache slot
- *     beyond its page table, a bounded wait that expired) are recorded in a status word at the
- *     start of the workspace; read it with xkv_read_device_status after the call.
+ *     beyond its page table, a bounded wait that expired, a prompt longer than max_seqlen) are
+ *     recorded in a status word, the first four bytes of the workspace. The word is sticky: a call
+ *     never clears it, it keeps the first error recorded since it was last read, so one workspace
+ *     can serve many calls (the layers of a phase) and be checked once. xkv_read_device_status
+ *     returns the word and resets it. A workspace must be zero-filled before its first use.
+ *   - The first call of an entry point on a device does one-time set-up (kernel attributes, symbol
+ *     addresses); these steps are idempotent and safe from several host threads.
  *   - Sequences are packed: token c of sequence b is row cu_seqlens[b] + c. t_b = cu_seqlens[b+1]
  *     - cu_seqlens[b] is the prompt length, W = dims.window, P_b = max(t_b - W, 0) the prefix
  *     length (the tokens that can be evicted); the last min(W, t_b) tokens are always kept.
@@ -112,7 +117,9 @@ typedef struct xkv_cache {
  * k          dev bf16, token row cu_seqlens[b]+c, head g at element offset
  *            (cu_seqlens[b]+c)*kv_stride_token + g*kv_stride_head
  * cu_seqlens dev int32 [B+1], non-decreasing, cu_seqlens[0] = 0, cu_seqlens[B] = total_tokens
- * total_tokens, max_seqlen  host values: T and an upper bound of every t_b
+ * total_tokens, max_seqlen  host values: T and an upper bound of every t_b. The launch grids and buffers are
+ *            sized from max_seqlen: a prompt found longer on the device is processed as if cut to
+ *            max_seqlen tokens and the device status becomes XKV_ERR_INVALID_ARG.
  * scores     dev out fp32 [Hkv][T]: w at column cu_seqlens[b]+c for c < P_b; window columns are 0
  * sorted     dev out fp32 [Hkv][T]: per (g, b) the P_b values of w in descending order at columns
  *            cu_seqlens[b] .. cu_seqlens[b]+P_b-1; window columns are 0. NULL skips the sort and
@@ -152,7 +159,7 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
                              int32_t* budgets, double* r_avg);
 
 /*
- * xkv_average_budgets -- the averaged allocation list of the online scenario (Sec. IV-D), host only.
+ * xkv_average_budgets -- the averaged allocation list of the online scenario (Sec. IV-C), host only.
  *
  * The lists that xkv_alloc_budgets produced for a sample of tasks of one type are averaged layer by
  * layer; later tasks of that type skip the allocation and are evicted under the averaged list.
@@ -177,7 +184,10 @@ xkv_status xkv_average_budgets(const int32_t* lists, int32_t n_tasks, int32_t n_
  * bit-exactly from k and v into cache slots 0 .. kb + (t_b - P_b) - 1 of (layer, b) and
  * seq_lens[layer][b] is set to that count.
  *
- * budget     host int32 [1] (per_sequence = 0) or [B] (per_sequence = 1), each >= 0
+ * budget     host int32 [1] (per_sequence = 0) or [B] (per_sequence = 1), each >= 0. With per_sequence = 1
+ *            the array is copied to the device on `stream`: from pageable memory that copy waits
+ *            for the stream's earlier work; from pinned memory it is asynchronous, and the array
+ *            must then stay alive and unchanged until the stream has passed this call.
  * scores     dev fp32 [Hkv][T] (w of xkv_score, or any non-negative finite scores)
  * sorted     dev fp32 [Hkv][T] (descending per (g,b), as xkv_score writes it)
  * k, v       dev bf16, same layout and strides (dims.kv_stride_*)
@@ -210,11 +220,14 @@ xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t
  * lse        dev out fp32 [Lr][B][Hq], may be NULL: natural-log sum of exp of the scaled logits
  * chunk_rows 0 = chosen on the device from the cache lengths; otherwise a multiple of 64
  * workspace  dev, at least xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...) bytes
- * Device status XKV_ERR_CAPACITY if an append does not fit its page table (that row is skipped).
- * Launches: up to 2048 (layer, sequence) units the call is one small memset and one kernel, launched
- * cooperatively with one block per SM (the blocks append, meet once and plan their work themselves),
- * so the device must be able to hold that grid at once -- other work on the GPU delays the launch, it
- * does not break it. Larger problems run a separate append-and-plan kernel first.
+ * Device status XKV_ERR_CAPACITY if an append does not fit its page table (that row is neither stored
+ * nor attended to and its seq_lens entry stays), XKV_ERR_WORKSPACE if the work items planned on the
+ * device exceed what the workspace was sized for, XKV_ERR_TIMEOUT if a bounded wait expired.
+ * Launches: up to 2048 (layer, sequence) units the call is one small memset and one kernel whose blocks
+ * plan their work themselves from the lengths before the call; the block that handles the end of a
+ * cache takes the new row from k_new / v_new and stores it, and seq_lens is advanced when the last
+ * block leaves. No block waits for another one to start, so the launch needs no particular
+ * residency. Larger problems run a separate append-and-plan kernel first.
  */
 xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin,
                            int32_t layer_end, const void* q, const void* k_new, const void* v_new,
@@ -235,10 +248,16 @@ xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t
  *
  * Arguments and results are those of xkv_decode_attn without workspace/workspace_bytes, plus
  *   status_out  dev out int32 [1], may be NULL: receives the device status word of this call
- *               (XKV_OK, XKV_ERR_CAPACITY, XKV_ERR_TIMEOUT) in stream order; copy it to the host to read it.
+ *               (XKV_OK, XKV_ERR_CAPACITY, XKV_ERR_WORKSPACE, XKV_ERR_TIMEOUT) in stream order; copy it to
+ *               the host to read it. Unlike a caller's workspace the array's status word is cleared by
+ *               every call.
  * Limits and rules
  *   - Returns XKV_ERR_WORKSPACE, launching nothing, when the scratch this problem needs
- *     (xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...)) exceeds XKV_STATIC_SCRATCH_BYTES.
+ *     (xkv_workspace_bytes(XKV_OP_DECODE_ATTN, ...)) exceeds XKV_STATIC_SCRATCH_BYTES. With
+ *     chunk_rows = 0 the library reserves room for about 14 000 chunks beyond one per (layer,
+ *     sequence, KV head), which alone passes the limit once G * head_dim >= 256 (any grouped-query
+ *     model with head_dim 128): such callers pass an explicit chunk_rows, which sizes the scratch
+ *     from the longest cache instead.
  *   - The first call on a device looks up the array's device address (a one-time set-up step);
  *     make that first call outside any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents; each call
@@ -262,11 +281,11 @@ size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen,
                            int32_t chunk_rows);
 
 /*
- * Copies the device status word of `workspace` to the host, waits for `stream`, and returns it:
- * XKV_OK, or the first XKV_ERR_* a kernel of the last call on that workspace recorded.
- * This is the only entry point that synchronises.
+ * Copies the device status word of `workspace` to the host, resets the word to XKV_OK, waits for
+ * `stream`, and returns what it read: XKV_OK, or the first XKV_ERR_* a kernel recorded in any call
+ * on that workspace since the word was last read. This is the only entry point that synchronises.
  */
-xkv_status xkv_read_device_status(const void* workspace, void* stream);
+xkv_status xkv_read_device_status(void* workspace, void* stream);
 
 /*
  * Profiling hook (no counterpart in the paper): while both events are set, every xkv_decode_attn call
@@ -275,6 +294,14 @@ xkv_status xkv_read_device_status(const void* workspace, void* stream);
  * owned by the caller; pass NULL, NULL to switch the hook off (the default). Not thread-safe.
  */
 void xkv_profile_events(void* start, void* stop);
+
+/*
+ * Test hook (no counterpart in the paper), process-wide: the limit of every bounded wait inside the kernels
+ * (nanoseconds; <= 0 restores the default of two seconds), and the index of one decode work item whose
+ * split-K merge ticket is never published (-1: none), so that a test can watch a wait run out: the kernel
+ * returns, the device status reads XKV_ERR_TIMEOUT and the workspace stays usable.
+ */
+void xkv_test_hooks(int64_t wait_limit_ns, int32_t withhold_decode_item);
 
 /* Number of kernel launches the library enqueued since it was loaded (all entry points). */
 int64_t xkv_launch_count(void);

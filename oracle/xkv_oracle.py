@@ -185,51 +185,51 @@ def retained_mass(gains: np.ndarray) -> np.ndarray:
 def adaptive_allocation(gains: list[np.ndarray], N: int | None = None, R_avg: float | None = None,
                         n_min: int = 0, n_max: int | None = None,
                         capacity: list[int] | None = None) -> tuple[list[int], float]:
-    """Algorithm 1.  gains[i][j] is layer i's (j+1)-th largest normalised score.
+    """Algorithm 1 (adaptive allocation).  gains[i][j] is layer i's (j+1)-th largest normalised score,
+    i.e. the increase of R_i (Eq. 4) when layer i keeps one more token (Eq. 21).
 
-    Mode N (Eq. 17): hand out N slots.  Mode R_avg (Eq. 18): stop at the first iteration where the
-    mean over layers of the granted normalised scores reaches R_avg.
-    Returns (List_A, mean over layers of the retained ratio).
+    Every layer offers the gain of the next token it would keep; one slot at a time goes to the layer whose
+    offer is largest (the lowest layer among equal offers), and that layer then offers its following token.
+    Mode N (Eq. 17): stop after N slots.  Mode R_avg (Eq. 18): stop as soon as the mean over layers of the
+    retained ratio reaches R_avg.  Returns (slots per layer, mean over layers of the retained ratio).
     """
-    L = len(gains)
-    cap = [len(g) for g in gains] if capacity is None else list(capacity)
+    n_layers = len(gains)
+    room = [len(g) for g in gains] if capacity is None else list(capacity)
     if n_max is not None:
-        cap = [min(c, n_max) for c in cap]
+        room = [min(c, n_max) for c in room]
 
-    def wait_value(i: int, pos: int) -> float:
-        # normalised score of the token layer i would keep next, after holding pos slots
-        if pos >= cap[i]:
+    def offer(i: int) -> float:
+        # gain of the token layer i would keep next; a full layer offers nothing, ranks past the curve add 0
+        if held[i] >= room[i]:
             return NEG_INF
-        return float(gains[i][pos]) if pos < len(gains[i]) else 0.0
+        return float(gains[i][held[i]]) if held[i] < len(gains[i]) else 0.0
 
-    List_A = [min(n_min, cap[i]) for i in range(L)]
-    R_total = sum(float(np.sum(np.asarray(gains[i][: List_A[i]], dtype=np.float64))) for i in range(L))
-    List_W = [wait_value(i, List_A[i]) for i in range(L)]
+    held = [min(n_min, room[i]) for i in range(n_layers)]
+    retained = sum(float(np.sum(np.asarray(gains[i][: held[i]], dtype=np.float64))) for i in range(n_layers))
 
-    def grant() -> None:
-        nonlocal R_total
-        maximum = max(List_W)
-        if maximum == NEG_INF:
+    def give_one_slot() -> None:
+        nonlocal retained
+        offers = [offer(i) for i in range(n_layers)]
+        best = max(offers)
+        if best == NEG_INF:
             raise ValueError("budget exceeds capacity")
-        index = List_W.index(maximum)          # first layer holding the maximum
-        List_A[index] += 1
-        R_total += maximum
-        pos = List_A[index]
-        List_W[index] = wait_value(index, pos)
+        winner = offers.index(best)            # lowest layer index among equal offers
+        held[winner] += 1
+        retained += best
 
     if N is not None:
-        if N < sum(List_A):
+        if N < sum(held):
             raise ValueError("N below the n_min floor")
-        for _ in range(N - sum(List_A)):
-            grant()
+        while sum(held) < N:
+            give_one_slot()
     elif R_avg is not None:
         if not (0.0 < R_avg <= 1.0 + 1e-12):
             raise ValueError("R_avg target out of range")
-        while R_total / L < R_avg:
-            grant()
+        while retained / n_layers < R_avg:
+            give_one_slot()
     else:
         raise ValueError("give N or R_avg")
-    return List_A, R_total / L
+    return held, retained / n_layers
 
 
 def allocation_objective(gains: list[np.ndarray], List_A: list[int]) -> float:
@@ -238,7 +238,7 @@ def allocation_objective(gains: list[np.ndarray], List_A: list[int]) -> float:
 
 
 def averaged_allocation(lists: list[list[int]]) -> list[int]:
-    """Online scenario (Sec. IV-D): the allocation lists recorded for the sampled tasks are averaged layer by
+    """Online scenario (Sec. IV-C): the allocation lists recorded for the sampled tasks are averaged layer by
     layer and the averaged list is applied to later tasks of the same type.
 
     The paper does not say how the averages become integers.  Reading taken here: every layer gets the floor of

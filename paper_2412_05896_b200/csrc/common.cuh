@@ -21,7 +21,7 @@ struct WorkspaceHeader {
   int32_t prep_ticket;   // decode: CTAs of the prepare kernel that have finished
   int32_t n_multi;       // decode: (layer, sequence) units cut into more than one chunk
   int32_t merge_counter; // decode: next split-K merge job to hand to a warp
-  int32_t grid_arrivals; // decode: CTAs of the self-planning launch that have finished appending
+  int32_t grid_arrivals; // decode: CTAs of the self-planning launch that have finished all their work
   int32_t reserved[56];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
@@ -34,6 +34,10 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 void count_launch(int n = 1);
 xkv_status check_launch();
 int sm_count();
+// Limit, in nanoseconds, of every bounded wait inside a kernel (two seconds unless a test shortened it).
+uint64_t wait_limit_ns();
+// Test hook: index of the decode work item whose merge ticket is withheld (-1: none).
+int32_t debug_withhold_item();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -99,13 +103,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Waits for the phase with the given parity; gives up after kWaitLimit polls and returns false.
-constexpr uint32_t kWaitLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* ptr) {
+  int32_t v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+  return v;
+}
+
+// Waits for the phase with the given parity for at most limit_ns of wall time; false on expiry.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint64_t limit_ns) {
+  for (int i = 0; i < 128; ++i)
     if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (global_timer_ns() - t0 > limit_ns) return false;
   }
-  return false;
+}
+
+// Polls a counter in global memory until it reaches `target`, for at most limit_ns; false on expiry.
+__device__ __forceinline__ bool spin_until_ge(const int32_t* ptr, int32_t target, uint64_t limit_ns, unsigned sleep_ns) {
+  if (ld_acquire_gpu(ptr) >= target) return true;
+  const uint64_t t0 = global_timer_ns();
+  while (ld_acquire_gpu(ptr) < target) {
+    if (global_timer_ns() - t0 > limit_ns) return false;
+    __nanosleep(sleep_ns);
+  }
+  return true;
 }
 
 // 2-D tiled TMA load global -> shared, completion counted on an mbarrier.  x is the innermost

@@ -21,7 +21,7 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
 size_t decode_workspace_bytes(const xkv_dims* d, int n_layers, int max_cache_len, int chunk_rows);
 xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end, const void* q,
                        const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,
-                       void* workspace, size_t workspace_bytes, cudaStream_t st);
+                       void* workspace, size_t workspace_bytes, cudaStream_t st, bool clear_status = false);
 
 xkv_status decode_attn_static(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end,
                               const void* q, const void* k_new, const void* v_new, void* out, float* lse,

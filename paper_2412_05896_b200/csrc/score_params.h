@@ -26,7 +26,9 @@ struct ScoreParams {
   int32_t batch, n_q_heads, n_kv_heads, group, window, M, pool_kernel, pool_mode;
   int32_t M_real;      // G*W; M is M_real rounded up to a multiple of 16 (the padding rows never contribute)
   int32_t split_keys, n_splits, n_chunks, curve_len;
+  int32_t max_seqlen;  // host bound of every prompt length; longer prompts are cut to it and reported
   float scale_log2;
+  uint64_t wait_ns;    // limit of every bounded wait
 };
 
 // tcgen05 variant of the two logit passes (xkv_score_tc.cu).  Returns XKV_ERR_UNSUPPORTED when the shape
@@ -35,8 +37,9 @@ xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, c
 // Key split the tcgen05 variant uses (0 if it does not cover the shape).
 int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen);
 
-// Single-launch variant (xkv_score_fused.cu): both passes by thread-block clusters, the second one fed from L2.
-// Covers G*W in {32, 64, 128} while the keys of the units in flight fit in L2.
+// Single-launch variant (xkv_score_fused.cu): a thread-block cluster per unit keeps the unit's logits in tensor
+// memory between the statistics and the column sums, so the keys are read once.  Covers G*W = 32 and prompts of
+// at most 8192 tokens.
 bool score_fused_covers(int M, int head_dim, int units, int max_seqlen);
 xkv_status score_fused_pass(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st);
 

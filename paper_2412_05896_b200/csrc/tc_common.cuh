@@ -102,11 +102,6 @@ __device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_
                : "memory");
 }
 
-__device__ __forceinline__ uint64_t tc_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
 constexpr int kWsThreads = 320;
 constexpr int kEpiThreads = 128;     // threads of one epilogue group
 constexpr int kWsStages = 4;       // shared-memory ring of key tiles
@@ -169,15 +164,15 @@ __device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int
   m = m_new;
 }
 
-// Bounded mbarrier wait (two seconds) that also gives up when another role has raised the abort flag.
-__device__ __forceinline__ bool ws_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded mbarrier wait that also gives up when another role has raised the abort flag.
+__device__ __forceinline__ bool ws_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
   for (int i = 0; i < 64; ++i)
     if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = tc_timer_ns();
+  const uint64_t t0 = global_timer_ns();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (tc_timer_ns() - t0 > 2000000000ull) {
+    if (global_timer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       return false;
     }

@@ -22,16 +22,22 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 xkv_status check_launch() { return cudaGetLastError() == cudaSuccess ? XKV_OK : XKV_ERR_CUDA; }
 
 int sm_count() {
-  static int cached[64] = {};
+  static std::atomic<int> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (cached[dev] == 0) {
-    int n = 0;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    cached[dev] = n;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
-  return cached[dev];
+  return n;
 }
+
+static std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+static std::atomic<int32_t> g_withhold_item{-1};
+
+uint64_t wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+int32_t debug_withhold_item() { return g_withhold_item.load(std::memory_order_relaxed); }
 
 namespace {
 
@@ -189,12 +195,13 @@ size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen,
   }
 }
 
-xkv_status xkv_read_device_status(const void* workspace, void* stream) {
+xkv_status xkv_read_device_status(void* workspace, void* stream) {
   if (workspace == nullptr) return XKV_ERR_INVALID_ARG;
   int32_t status = 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemcpyAsync(&status, workspace, sizeof(status), cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return XKV_ERR_CUDA;
+  if (cudaMemsetAsync(workspace, 0, sizeof(status), st) != cudaSuccess) return XKV_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return XKV_ERR_CUDA;
   return status;
 }
@@ -204,6 +211,11 @@ void xkv_profile_events(void* start, void* stop) {
 }
 
 int64_t xkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void xkv_test_hooks(int64_t wait_limit_ns, int32_t withhold_decode_item) {
+  g_wait_limit_ns.store(wait_limit_ns > 0 ? (uint64_t)wait_limit_ns : 2000000000ull, std::memory_order_relaxed);
+  g_withhold_item.store(withhold_decode_item, std::memory_order_relaxed);
+}
 
 const char* xkv_status_string(xkv_status status) {
   switch (status) {

@@ -2,11 +2,18 @@
 // compacted per-layer caches.
 //
 // Kernels, in stream order:
-//   decode_prepare_kernel  one CTA per (layer, sequence): store the new K/V row of every KV head in
-//                          slot seq_lens[l][b] and advance seq_lens; the last CTA to finish then cuts
-//                          every (layer, sequence, KV head) cache into chunks of rows and writes the
-//                          work-item table (the chunk size is chosen from the total cached length).
-//   decode_attn_kernel     persistent CTAs of eight independent warps.  A warp takes work items
+//   decode_prepare_kernel  only for more than 2048 (layer, sequence) units: one CTA per unit stores the
+//                          new K/V row of every KV head in slot seq_lens[l][b] and advances seq_lens;
+//                          the last CTA to finish then cuts every (layer, sequence, KV head) cache into
+//                          chunks of rows and writes the work-item table.
+//   decode_attn_kernel     persistent CTAs of eight independent warps.  Up to 2048 units every CTA plans
+//                          for itself from the lengths as they were before the call (chunk size from the
+//                          total cached length, chunks before each unit as a prefix table in shared
+//                          memory) and nothing waits for anything: the warp that owns the last chunk of a
+//                          (unit, KV head) takes the new K/V row from the call's arguments, patches it
+//                          into its shared-memory tile and stores it to the page; seq_lens is advanced
+//                          by the last CTA to leave, so a CTA that starts late still plans from the old
+//                          lengths.  A warp takes work items
 //                          from a global counter and streams its item's K and V rows through its own
 //                          ring of shared-memory stages: 16-row TMA tensor boxes (128-byte swizzle)
 //                          that complete on an mbarrier, issued by the warp itself a few tiles ahead
@@ -30,6 +37,8 @@
 
 #include <cmath>
 #include <mutex>
+
+#include <atomic>
 
 #include "common.cuh"
 #include "ops.h"
@@ -62,8 +71,10 @@ struct DecodeParams {
   int32_t layer_begin, n_layers, batch, n_q_heads, n_kv_heads, group;
   int32_t page_size, max_pages_per_seq, n_pages;
   int32_t chunk_rows_forced, max_items;
-  int32_t fused_plan, do_append;   // fused_plan: the attention kernel appends and plans in its own prologue
+  int32_t fused_plan, do_append;   // fused_plan: the attention kernel plans in its own prologue and appends itself
+  int32_t withhold_item;           // test hook: the merge ticket of this work item is never published (-1: none)
   float scale_log2;
+  uint64_t wait_ns;                // limit of every bounded wait
   WorkspaceHeader* hdr;
   int32_t* tickets;   // [n_layers*batch*n_kv_heads]
   int2* unit_info;    // [n_layers*batch]: {first item of head 0, chunks per head}
@@ -236,29 +247,6 @@ __global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodePara
 }
 
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t global_timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* ptr) {
-  int32_t v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
-  return v;
-}
-
-// Bounded wait: two seconds of wall time at most.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (int i = 0; i < 128; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_timer_ns();
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (global_timer_ns() - t0 > 2000000000ull) return false;
-  }
-}
-
 template <int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
@@ -289,32 +277,17 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 
   const bool fused = p.fused_plan != 0;
   const int n_units = p.n_layers * p.batch;
+  // Length of unit e as this launch sees it: the stored length, plus the row this call appends when it fits the
+  // page table.  seq_lens itself is only advanced by the last CTA to leave, so this reads the same at any time.
+  const int cap_rows = p.max_pages_per_seq * p.page_size;
+  const bool self_append = fused && p.do_append != 0;
+  auto unit_len = [&](int e) -> int {
+    int n = __ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]);
+    n = n > 0 ? n : 0;
+    return n + ((self_append && n < cap_rows) ? 1 : 0);
+  };
   if (fused) {
-    // ---- prologue of the self-planning launch: append, meet, plan
-    for (int e = blockIdx.x; e < n_units; e += gridDim.x) {
-      if (p.do_append) append_unit(p, D, e, &s_plan[3]);
-      for (int h = tid; h < p.n_kv_heads; h += kAttnThreads) p.tickets[e * p.n_kv_heads + h] = 0;
-    }
-    // every CTA of the grid is resident (cooperative launch): wait until all have appended
-    __threadfence();
-    __syncthreads();
-    int met = 1;
-    if (tid == 0) {
-      atomicAdd(&p.hdr->grid_arrivals, 1);
-      const uint64_t t0 = global_timer_ns();
-      while (ld_acquire_gpu(&p.hdr->grid_arrivals) < (int)gridDim.x) {
-        if (global_timer_ns() - t0 > 2000000000ull) {
-          met = 0;
-          record_status(p.hdr, XKV_ERR_TIMEOUT);
-          break;
-        }
-        __nanosleep(64);
-      }
-      __threadfence();
-    }
-    if (!__syncthreads_and(met)) return;
-    // the rows other CTAs stored with ordinary writes are read below by TMA (the asynchronous proxy)
-    asm volatile("fence.proxy.async.global;" ::: "memory");
+    // ---- prologue of the self-planning launch
     // the plan, computed by every CTA for itself: chunk size from the total length, then the number of chunks
     // before each unit (and the list of units with more than one)
     constexpr int kPer = kMaxPlanUnits / kAttnThreads;
@@ -323,9 +296,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
     for (int i = 0; i < kPer; ++i) {
       const int e = tid * kPer + i;
-      int n = 0;
-      if (e < n_units) n = __ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]);
-      nloc[i] = n > 0 ? n : 0;
+      nloc[i] = e < n_units ? unit_len(e) : 0;
       rows += nloc[i];
     }
 #pragma unroll
@@ -408,8 +379,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int first_chunk = s_excl[lo], nc = s_excl[lo + 1] - first_chunk;
     const int local = idx - first_chunk * p.n_kv_heads;
     const int h = local / nc, c = local % nc;
-    int n = __ldcg(&p.seq_lens[(p.layer_begin + lo / p.batch) * p.batch + lo % p.batch]);
-    n = n > 0 ? n : 0;
+    const int n = unit_len(lo);
     const int rb = c * plan_chunk;
     return make_int4(lo, h, rb, min(n, rb + plan_chunk));
   };
@@ -503,7 +473,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (aborted) return;
     const int s = idx % C::kStages;
     const uint32_t ph = (idx / C::kStages) & 1u;
-    const bool ok = ((int32_t)(issued - idx) > 0) && mbar_wait_bounded(&full_bar[s], ph);
+    const bool ok = ((int32_t)(issued - idx) > 0) && mbar_wait_bounded(&full_bar[s], ph, p.wait_ns);
     if (!__all_sync(0xffffffffu, ok)) {
       aborted = true;
       no_more = true;
@@ -557,9 +527,41 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     };
 
     const int n_tiles = (I.w - I.z + kTileRows - 1) / kTileRows;
+    // The row this call appends to (e, h) is the last row of the unit's last chunk.  Its page slot still holds
+    // old bytes when the tile is copied in, so the owner of that chunk takes the row from k_new / v_new:
+    // into the landed tile (16-byte pieces at their swizzled places; lanes 0-15 carry K, lanes 16-31 V) and into
+    // the page, where the next call's copies will find it.
+    int new_slot = -1;                                   // cache slot of the appended row if this item owns it
+    if (self_append && I.w > I.z) {
+      const int n_old = max(__ldcg(&p.seq_lens[(p.layer_begin + e / p.batch) * p.batch + e % p.batch]), 0);
+      if (n_old < cap_rows && I.w == n_old + 1) new_slot = n_old;
+    }
+    auto patch_new_row = [&](uint32_t idx) {
+      constexpr int kPieces = D / 8;                     // 16-byte pieces of one row
+      const int r = (new_slot - I.z) % kTileRows;
+      uint8_t* ks = ring + (size_t)(idx % C::kStages) * C::kStageBytes;
+      const size_t src = ((size_t)e * p.n_kv_heads + h) * D;
+      const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
+      const int page = p.block_table[(size_t)le * p.max_pages_per_seq + new_slot / p.page_size];
+      const bool page_ok = page >= 0 && page < p.n_pages;
+      if (!page_ok && lane == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
+      for (int i = lane; i < 2 * kPieces; i += 32) {
+        const int is_v = i / kPieces, c = i % kPieces;
+        const uint4 val = *reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8);
+        *reinterpret_cast<uint4*>(ks + is_v * C::kTileBytes + (c >> 3) * C::kBoxBytes + r * 128 +
+                                  (((c & 7) ^ (r & 7)) << 4)) = val;
+        if (page_ok) {
+          const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + new_slot % p.page_size) * D + c * 8;
+          *reinterpret_cast<uint4*>((is_v ? p.v_pages : p.k_pages) + dst) = val;
+        }
+      }
+      fence_proxy_async_smem();       // the stage is written again by a later copy
+      __syncwarp();
+    };
     float s_next[4] = {0.f, 0.f, 0.f, 0.f};
     if (n_tiles > 0) {
       wait_tile(consumed);
+      if (!aborted && new_slot >= 0 && n_tiles == 1) patch_new_row(consumed);
       if (!aborted) qk_tile(consumed, s_next);
     }
     for (int t = 0; t < n_tiles; ++t) {
@@ -570,6 +572,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int wrows = min(kTileRows, I.w - (I.z + t * kTileRows));
       if (t + 1 < n_tiles) {          // the next tile's scores do not depend on this tile's softmax
         wait_tile(consumed + 1);
+        if (!aborted && new_slot >= 0 && t + 2 == n_tiles) patch_new_row(consumed + 1);
         if (!aborted) qk_tile(consumed + 1, s_next);
       }
       if (!aborted) {
@@ -680,7 +683,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
                 make_float2(m_ref[hh], l_part[hh]);
       }
       __syncwarp();                 // the lanes' partial results are ordered before lane 0's fence (cumulative)
-      if (lane == 0) {
+      if (lane == 0 && item != p.withhold_item) {
         __threadfence();
         atomicAdd(&p.tickets[e * p.n_kv_heads + h], 1);     // one more chunk of this unit is published
       }
@@ -705,19 +708,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     const int2 ui = unit_info(e);
     const int nc = ui.y, first = ui.x + h * nc;
     int ready = 1;
-    if (lane == 0) {
-      const int32_t* tk = &p.tickets[e * p.n_kv_heads + h];
-      if (ld_acquire_gpu(tk) < nc) {
-        const uint64_t t0 = global_timer_ns();
-        while (ld_acquire_gpu(tk) < nc) {
-          if (global_timer_ns() - t0 > 2000000000ull) {
-            ready = 0;
-            break;
-          }
-          __nanosleep(200);
-        }
-      }
-    }
+    if (lane == 0) ready = spin_until_ge(&p.tickets[e * p.n_kv_heads + h], nc, p.wait_ns, 200) ? 1 : 0;
     ready = __shfl_sync(0xffffffffu, ready, 0);
     if (!ready) {
       if (lane == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
@@ -784,6 +775,25 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     // let copies already issued land before this CTA's shared memory can be handed on
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
   }
+  if (self_append) {
+    // the last CTA to get here advances the lengths of the units whose new row was stored
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_plan[3] = (atomicAdd(&p.hdr->grid_arrivals, 1) == (int)gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (s_plan[3]) {
+      for (int e = tid; e < n_units; e += kAttnThreads) {
+        const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
+        const int n_old = max(p.seq_lens[le], 0);
+        if (n_old < cap_rows) {
+          const int page = p.block_table[(size_t)le * p.max_pages_per_seq + n_old / p.page_size];
+          if (page >= 0 && page < p.n_pages) p.seq_lens[le] = n_old + 1;
+        } else {
+          record_status(p.hdr, XKV_ERR_CAPACITY);
+        }
+      }
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -832,9 +842,8 @@ bool decode_layout(const xkv_dims* d, int n_layers, int max_cache_len, int chunk
     const int64_t per = max_cache_len > 0 ? ((int64_t)max_cache_len + chunk_rows - 1) / chunk_rows : 1;
     max_items = units * (per > 0 ? per : 1);
   } else {
-    max_items = units + (int64_t)(kTargetItems + 1) * 1;
     // ceil() adds at most one item per unit, the rows themselves at most kTargetItems
-    max_items += 0;
+    max_items = units + (int64_t)kTargetItems + 1;
   }
   if (max_items > (int64_t)1 << 28) return false;
   const int G = d->n_q_heads / d->n_kv_heads;
@@ -858,34 +867,16 @@ xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const Decod
   // opt in to the large dynamic shared-memory carve-out once per process and device in use
   int dev = 0;
   cudaGetDevice(&dev);
-  static bool done[64] = {};
+  static std::atomic<bool> done[64];   // idempotent set-up: two threads doing it twice is harmless
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
-  if (!done[dev]) {
+  if (!done[dev].load(std::memory_order_acquire)) {
     attr_err = cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     Cfg<D>::kSmemBytes);
     if (attr_err != cudaSuccess) return XKV_ERR_CUDA;
-    done[dev] = true;
+    done[dev].store(true, std::memory_order_release);
   }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_start, st);
-  if (p.fused_plan) {
-    // the prologue's grid-wide meeting needs every CTA resident: a cooperative launch guarantees it
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)sm_count());
-    cfg.blockDim = dim3(kAttnThreads);
-    cfg.dynamicSmemBytes = Cfg<D>::kSmemBytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, decode_attn_kernel<D>, tk, tv, p) != cudaSuccess) {
-      cudaGetLastError();
-      return XKV_ERR_CUDA;
-    }
-  } else {
-    decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
-  }
+  decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_stop, st);
   count_launch();
   return check_launch();
@@ -906,7 +897,7 @@ size_t decode_workspace_bytes(const xkv_dims* d, int n_layers, int max_cache_len
 
 xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end, const void* q,
                        const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,
-                       void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                       void* workspace, size_t workspace_bytes, cudaStream_t st, bool clear_status) {
   const int Lr = layer_end - layer_begin;
   const int G = d->n_q_heads / d->n_kv_heads;
   if (G > kMaxGroup) return XKV_ERR_UNSUPPORTED;
@@ -947,6 +938,8 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   p.max_items = (int32_t)L.max_items;
   const float scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
+  p.wait_ns = wait_limit_ns();
+  p.withhold_item = debug_withhold_item();
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   p.tickets = reinterpret_cast<int32_t*>(ws + L.tickets);
   p.unit_info = reinterpret_cast<int2*>(ws + L.unit_info);
@@ -957,14 +950,15 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
 
   const int n_units = Lr * d->batch;
   const int do_append = k_new != nullptr ? 1 : 0;
-  // Up to kMaxPlanUnits units the attention kernel appends and plans in its own prologue (one launch);
-  // beyond that a separate kernel appends and writes the work-item table.
+  // Up to kMaxPlanUnits units the attention kernel plans in its own prologue and appends as it goes (one
+  // launch); beyond that a separate kernel appends and writes the work-item table.
   p.fused_plan = n_units <= kMaxPlanUnits ? 1 : 0;
   p.do_append = do_append;
-  if (p.fused_plan) {
-    if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;   // status, counters
-  } else {
-    if (cudaMemsetAsync(ws, 0, L.unit_info, st) != cudaSuccess) return XKV_ERR_CUDA;    // header + tickets
+  // counters and tickets start at zero; the status word (the first four bytes) is left alone unless asked, so an
+  // error of an earlier call on this workspace stays until it is read
+  const size_t keep = clear_status ? 0 : sizeof(int32_t);
+  if (cudaMemsetAsync(ws + keep, 0, L.unit_info - keep, st) != cudaSuccess) return XKV_ERR_CUDA;
+  if (!p.fused_plan) {
     decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append);
     count_launch();
     xkv_status s = check_launch();
@@ -986,13 +980,15 @@ xkv_status decode_attn_static(const xkv_dims* d, const xkv_cache* c, int layer_b
                               int chunk_rows, int32_t* status_out, cudaStream_t st) {
   // In host code g_static_scratch is only a handle for the symbol; the device address has to be
   // asked for, once per device, while that device is current.
-  static void* scratch_ptr[64] = {};
+  static std::atomic<void*> scratch_ptr[64];   // resolving the address twice from two threads gives the same value
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return XKV_ERR_CUDA;
-  if (scratch_ptr[dev] == nullptr) {
+  void* scratch = scratch_ptr[dev].load(std::memory_order_acquire);
+  if (scratch == nullptr) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return XKV_ERR_CUDA;
-    scratch_ptr[dev] = ptr;
+    scratch_ptr[dev].store(ptr, std::memory_order_release);
+    scratch = ptr;
   }
   const int max_cache_len = c->max_pages_per_seq * c->page_size;
   const size_t need = decode_workspace_bytes(d, layer_end - layer_begin, max_cache_len, chunk_rows);
@@ -1000,10 +996,10 @@ xkv_status decode_attn_static(const xkv_dims* d, const xkv_cache* c, int layer_b
   if (need > kStaticScratchBytes) return XKV_ERR_WORKSPACE;   // problem too large for the fixed scratch
   // decode_attn clears the part of the scratch that must start at zero (status word, tickets)
   xkv_status s = decode_attn(d, c, layer_begin, layer_end, q, k_new, v_new, out, lse, chunk_rows,
-                             scratch_ptr[dev], kStaticScratchBytes, st);
+                             scratch, kStaticScratchBytes, st, /*clear_status=*/true);
   if (s != XKV_OK) return s;
   if (status_out != nullptr &&
-      cudaMemcpyAsync(status_out, scratch_ptr[dev], sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      cudaMemcpyAsync(status_out, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
     return XKV_ERR_CUDA;
   return XKV_OK;
 }

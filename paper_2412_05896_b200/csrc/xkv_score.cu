@@ -24,6 +24,8 @@
 // row normalisers must be final before a column sum can be formed.
 #include <cmath>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "ops.h"
 #include "score_params.h"
@@ -58,18 +60,6 @@ __device__ __forceinline__ uint32_t swz(int r, int c, int row_bytes) {
   return (uint32_t)(r * row_bytes + ((c >> 3) << 7) + (((c & 7) ^ (r & 7)) << 4));
 }
 
-__device__ __forceinline__ int ld_acquire(const int* ptr) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
-  return v;
-}
-
-__device__ __forceinline__ uint64_t timer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
 struct UnitShape {
   int b, g, cu, t, P;
 };
@@ -79,7 +69,7 @@ __device__ __forceinline__ UnitShape unit_shape(const ScoreParams& p, int unit) 
   s.b = unit / p.n_kv_heads;
   s.g = unit % p.n_kv_heads;
   s.cu = p.cu_seqlens[s.b];
-  s.t = p.cu_seqlens[s.b + 1] - s.cu;
+  s.t = min(p.cu_seqlens[s.b + 1] - s.cu, p.max_seqlen);
   s.P = max(s.t - p.window, 0);
   return s;
 }
@@ -269,21 +259,11 @@ __device__ __forceinline__ void publish_stats(const ScoreParams& p, const UnitSh
   }
 }
 
-// Bounded wait (two seconds) for a unit's row normalisers.  Thread 0 polls; returns false on expiry.
+// Bounded wait for a unit's row normalisers.  Thread 0 polls; returns false on expiry.
 __device__ __forceinline__ bool wait_unit_ready(const ScoreParams& p, int unit, int* s_flag) {
   if (threadIdx.x == 0) {
-    int ok = 1;
-    if (ld_acquire(&p.unit_ready[unit]) == 0) {
-      const uint64_t t0 = timer_ns();
-      while (ld_acquire(&p.unit_ready[unit]) == 0) {
-        __nanosleep(100);
-        if (timer_ns() - t0 > 2000000000ull) {
-          ok = 0;
-          record_status(p.hdr, XKV_ERR_TIMEOUT);
-          break;
-        }
-      }
-    }
+    const int ok = spin_until_ge(&p.unit_ready[unit], 1, p.wait_ns, 100) ? 1 : 0;
+    if (!ok) record_status(p.hdr, XKV_ERR_TIMEOUT);
     *s_flag = ok;
   }
   __syncthreads();
@@ -433,7 +413,10 @@ __global__ void __launch_bounds__(kSortThreads) pool_sort_kernel(const ScorePara
   const int unit = blockIdx.x, chunk = blockIdx.y;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
   const int cu = p.cu_seqlens[b];
-  const int t = p.cu_seqlens[b + 1] - cu;
+  const int t_given = p.cu_seqlens[b + 1] - cu;
+  const int t = min(t_given, p.max_seqlen);
+  if (t_given > p.max_seqlen && chunk == 0 && g == 0 && threadIdx.x == 0)
+    record_status(p.hdr, XKV_ERR_INVALID_ARG);       // a prompt longer than the bound the grids were sized for
   const int P = max(t - p.window, 0);
   const int c0 = chunk * kSortChunk;
   const int tid = threadIdx.x;
@@ -581,7 +564,7 @@ __global__ void __launch_bounds__(kMergeThreads) merge_kernel(const ScoreParams 
   const int unit = blockIdx.x;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
   const int cu = p.cu_seqlens[b];
-  const int t = p.cu_seqlens[b + 1] - cu;
+  const int t = min(p.cu_seqlens[b + 1] - cu, p.max_seqlen);
   const int P = max(t - p.window, 0);
   const int o0 = blockIdx.y * kMergeTile;
   if (o0 >= P) return;
@@ -625,7 +608,7 @@ __global__ void gains_kernel(const ScoreParams p) {
   extern __shared__ float s_inv[];   // [Hkv]
   const int b = blockIdx.y;
   const int cu = p.cu_seqlens[b];
-  const int t = p.cu_seqlens[b + 1] - cu;
+  const int t = min(p.cu_seqlens[b + 1] - cu, p.max_seqlen);
   const int P = max(t - p.window, 0);
   for (int g = threadIdx.x; g < p.n_kv_heads; g += blockDim.x) {
     const float* ps = p.part_sum + ((size_t)b * p.n_kv_heads + g) * p.n_chunks;
@@ -738,18 +721,18 @@ void score_layout(const xkv_dims* d, int max_seqlen, int64_t T, ScoreLayout* L) 
 template <int D>
 xkv_status launch_passes(const ScoreParams& p, const ScoreLayout& L, cudaStream_t st) {
   const size_t smem = PassCfg<D>::smem_bytes(p.M, L.slice_tiles);
-  static bool done[64] = {};
+  static std::atomic<bool> done[64];   // idempotent set-up: two threads doing it twice is harmless
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
-  if (!done[dev]) {
+  if (!done[dev].load(std::memory_order_acquire)) {
     const int max_smem = 227 * 1024;
     if (cudaFuncSetAttribute(score_stream_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) !=
             cudaSuccess ||
         cudaFuncSetAttribute(score_resident_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) !=
             cudaSuccess)
       return XKV_ERR_CUDA;
-    done[dev] = true;
+    done[dev].store(true, std::memory_order_release);
   }
   int grid = sm_count() * L.ctas_per_sm;
   if (grid > p.n_work) grid = p.n_work;
@@ -814,8 +797,11 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
   p.n_work = (L.resident ? 1 : 2) * units * L.n_splits;
   const float scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
   p.scale_log2 = scale * 1.4426950408889634f;
+  p.max_seqlen = max_seqlen;
+  p.wait_ns = wait_limit_ns();
 
-  if (cudaMemsetAsync(ws, 0, L.u, st) != cudaSuccess) return XKV_ERR_CUDA;   // header, tickets, ready flags
+  // counters, tickets and ready flags start at zero; the status word (first four bytes) keeps an unread error
+  if (cudaMemsetAsync(ws + 4, 0, L.u - 4, st) != cudaSuccess) return XKV_ERR_CUDA;
   xkv_status s;
   if (L.use_tc && score_fused_covers(p.M, d->head_dim, units, max_seqlen)) {
     s = score_fused_pass(p, d->head_dim, max_seqlen, st);      // both passes in one cluster kernel, keys read once

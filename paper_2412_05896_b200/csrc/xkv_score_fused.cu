@@ -25,6 +25,8 @@
 // CTAs are those of step X, within a cluster, whose CTAs the hardware schedules together; they are bounded
 // like every other wait here, and a CTA leaves only after a cluster-wide barrier, so no store can reach the
 // shared memory of a CTA that has gone.
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace xkv {
@@ -119,7 +121,7 @@ __device__ __forceinline__ bool unit_shape(const ScoreParams& p, int n, uint32_t
   u->b = unit / p.n_kv_heads;
   u->g = unit % p.n_kv_heads;
   u->cu = p.cu_seqlens[u->b];
-  u->t = p.cu_seqlens[u->b + 1] - u->cu;
+  u->t = min(p.cu_seqlens[u->b + 1] - u->cu, p.max_seqlen);
   u->P = max(u->t - p.window, 0);
   const int nt1 = (u->t + kTcKeyTile - 1) / kTcKeyTile, nt2 = (u->P + kTcKeyTile - 1) / kTcKeyTile;
   const int per = (nt1 + CS - 1) / CS;              // <= kSlotsPerUnit: the host checks max_seqlen
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
       for (int n = 0; ok && unit_shape<CS>(p, n, cluster, n_clusters, rank, &sh); ++n) {
         if (sh.n1 == 0) continue;
         const uint32_t qb = it & 1u;
-        ok = ws_wait(&qempty_bar[qb], ((it >> 1) & 1u) ^ 1u, s_abort);
+        ok = ws_wait(&qempty_bar[qb], ((it >> 1) & 1u) ^ 1u, s_abort, p.wait_ns);
         if (!ok) break;
         mbar_arrive_expect_tx(&qfull_bar[qb], (uint32_t)C::kQBytes);
         const int qrow0 = (sh.b * p.n_q_heads + sh.g * p.group) * p.window;
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
           tma_load_2d(q_s + (size_t)qb * C::kQBytes + hf * C::kQHalfBytes, &tmap_q, hf * 64, qrow0, &qfull_bar[qb]);
         for (int ti = 0; ti < sh.n1; ++ti, ++gt) {
           const uint32_t s = gt % C::kStages;
-          ok = ws_wait(&empty_bar[s], ((gt / C::kStages) & 1u) ^ 1u, s_abort);
+          ok = ws_wait(&empty_bar[s], ((gt / C::kStages) & 1u) ^ 1u, s_abort, p.wait_ns);
           if (!ok) break;
           mbar_arrive_expect_tx(&full_bar[s], (uint32_t)C::kKTileBytes);
 #pragma unroll
@@ -225,14 +227,14 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
       for (int n = 0; ok && unit_shape<CS>(p, n, cluster, n_clusters, rank, &sh); ++n) {
         if (sh.n1 == 0) continue;
         const uint32_t qb = it & 1u;
-        ok = ws_wait(&qfull_bar[qb], (it >> 1) & 1u, s_abort);
+        ok = ws_wait(&qfull_bar[qb], (it >> 1) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         const uint32_t qa = q_base + qb * C::kQBytes;
         for (int ti = 0; ti < sh.n1; ++ti, ++gt) {
           const uint32_t s = gt % C::kStages;
           const uint32_t slot = (it & 1u) * kSlotsPerUnit + (uint32_t)ti;
-          ok = ws_wait(&full_bar[s], (gt / C::kStages) & 1u, s_abort) &&
-               ws_wait(&resempty_bar[slot], ((slot_uses >> slot) & 1u) ^ 1u, s_abort);
+          ok = ws_wait(&full_bar[s], (gt / C::kStages) & 1u, s_abort, p.wait_ns) &&
+               ws_wait(&resempty_bar[slot], ((slot_uses >> slot) & 1u) ^ 1u, s_abort, p.wait_ns);
           if (!ok) break;
           slot_uses ^= 1u << slot;
           tc_fence_after_sync();
@@ -274,7 +276,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
     auto finish = [&](const UnitShape& u, uint32_t q, uint32_t slot0) {
       const uint32_t st = q % kStatSlots, st_phase = (q / kStatSlots) & 1u;
       const uint32_t par = q & 1u, phase = (q >> 1) & 1u;
-      ok = __all_sync(0xffffffffu, ws_wait(&stats_bar[st], st_phase, s_abort));
+      ok = __all_sync(0xffffffffu, ws_wait(&stats_bar[st], st_phase, s_abort, p.wait_ns));
       if (!ok) return;
       // row normalisers: thread r < 32 merges every entry of query row r (entries r, r + 32, ... of each CTA)
       if (eall < kRows) {
@@ -292,7 +294,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
       __syncwarp();
       if (lane == 0) mbar_arrive(&mrow_bar[par]);
       if (u.n1 == 0) return;
-      ok = __all_sync(0xffffffffu, ws_wait(&mrow_bar[par], phase, s_abort));
+      ok = __all_sync(0xffffffffu, ws_wait(&mrow_bar[par], phase, s_abort, p.wait_ns));
       if (!ok) return;
       // ---- B: column sums out of TMEM; a thread owns one key
       float* uo = p.u + (size_t)u.g * p.total_tokens + u.cu;
@@ -334,7 +336,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
       bool first = true;
       for (int ti = (int)group; ti < sh.n1; ti += 2) {
         const uint32_t slot = slot0 + (uint32_t)ti;
-        ok = __all_sync(0xffffffffu, ws_wait(&resfull_bar[slot], (slot_uses >> slot) & 1u, s_abort));
+        ok = __all_sync(0xffffffffu, ws_wait(&resfull_bar[slot], (slot_uses >> slot) & 1u, s_abort, p.wait_ns));
         if (!ok) break;
         tc_fence_after_sync();
         float x[32];
@@ -436,7 +438,7 @@ template <int D, int CS>
 xkv_status fused_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScoreParams& p, cudaStream_t st) {
   using F = FusedCfg<D, CS>;
   const size_t smem = F::kSmemBytes;             // > 113 KB: one CTA per SM, which owns all 512 TMEM columns
-  static int max_clusters[64] = {};
+  static std::atomic<int> max_clusters[64];   // the occupancy query gives the same answer from any thread
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
@@ -451,7 +453,7 @@ xkv_status fused_launch(const CUtensorMap& tq, const CUtensorMap& tk, const Scor
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (max_clusters[dev] == 0) {
+  if (max_clusters[dev].load(std::memory_order_acquire) == 0) {
     if (cudaFuncSetAttribute(score_fused_kernel<D, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return XKV_ERR_CUDA;
@@ -462,9 +464,9 @@ xkv_status fused_launch(const CUtensorMap& tq, const CUtensorMap& tk, const Scor
       cudaGetLastError();
       return XKV_ERR_CUDA;
     }
-    max_clusters[dev] = n;
+    max_clusters[dev].store(n, std::memory_order_release);
   }
-  int n_clusters = max_clusters[dev];
+  int n_clusters = max_clusters[dev].load(std::memory_order_acquire);
   const int units = p.batch * p.n_kv_heads;
   if (n_clusters > units) n_clusters = units;
   cfg.gridDim = dim3((unsigned)(n_clusters * CS));

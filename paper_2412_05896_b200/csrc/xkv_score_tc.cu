@@ -14,6 +14,8 @@
 //           exp2(s*c - normaliser[row]) over the query rows straight out of TMEM -> column score u[key].
 //           Items are walked in reverse so that the keys pass 1 streamed last are re-read from L2.
 // No CTA ever waits for another one; every mbarrier wait is bounded.
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace xkv {
@@ -50,7 +52,7 @@ __device__ __forceinline__ bool item_shape(const ScoreParams& p, int n, ItemShap
   it->b = it->unit / p.n_kv_heads;
   it->g = it->unit % p.n_kv_heads;
   it->cu = p.cu_seqlens[it->b];
-  it->t = p.cu_seqlens[it->b + 1] - it->cu;
+  it->t = min(p.cu_seqlens[it->b + 1] - it->cu, p.max_seqlen);
   it->P = max(it->t - p.window, 0);
   it->key_begin = it->split * p.split_keys;
   it->key_end = min(it->key_begin + p.split_keys, PASS == 1 ? it->t : it->P);
@@ -114,7 +116,7 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
       for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
         if (sh.n_tiles == 0) continue;
         const uint32_t qb = it % C::kQBufs;
-        ok = ws_wait(&qempty_bar[qb], ((it / C::kQBufs) & 1u) ^ 1u, s_abort);
+        ok = ws_wait(&qempty_bar[qb], ((it / C::kQBufs) & 1u) ^ 1u, s_abort, p.wait_ns);
         if (!ok) break;
         mbar_arrive_expect_tx(&qfull_bar[qb], C::kQTxBytes + (PASS == 2 ? (uint32_t)(M * 4) : 0u));
         if (PASS == 2)     // the item's row normalisers ride on the same barrier; slot reuse distance is four items
@@ -128,7 +130,7 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
                         &qfull_bar[qb]);
         for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
           const uint32_t s = gt % kWsStages;
-          ok = ws_wait(&empty_bar[s], ((gt / kWsStages) & 1u) ^ 1u, s_abort);
+          ok = ws_wait(&empty_bar[s], ((gt / kWsStages) & 1u) ^ 1u, s_abort, p.wait_ns);
           if (!ok) break;
           mbar_arrive_expect_tx(&full_bar[s], (uint32_t)C::kKTileBytes);
 #pragma unroll
@@ -149,13 +151,13 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
       for (int n = 0; ok && item_shape<PASS>(p, n, &sh); ++n) {
         if (sh.n_tiles == 0) continue;
         const uint32_t qb = it % C::kQBufs;
-        ok = ws_wait(&qfull_bar[qb], (it / C::kQBufs) & 1u, s_abort);
+        ok = ws_wait(&qfull_bar[qb], (it / C::kQBufs) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         const uint32_t qa = q_base + qb * C::kQBytes;
         for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
           const uint32_t s = gt % kWsStages, ab = gt % kAccBufs;
-          ok = ws_wait(&full_bar[s], (gt / kWsStages) & 1u, s_abort) &&
-               ws_wait(&accempty_bar[ab], ((gt / kAccBufs) & 1u) ^ 1u, s_abort);
+          ok = ws_wait(&full_bar[s], (gt / kWsStages) & 1u, s_abort, p.wait_ns) &&
+               ws_wait(&accempty_bar[ab], ((gt / kAccBufs) & 1u) ^ 1u, s_abort, p.wait_ns);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t kt = k_base + s * C::kKTileBytes;
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
       for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
         const uint32_t ab = gt % kAccBufs;
         if (ab != group) continue;               // the other group's tile
-        ok = __all_sync(0xffffffffu, ws_wait(&accfull_bar[ab], (gt / kAccBufs) & 1u, s_abort));
+        ok = __all_sync(0xffffffffu, ws_wait(&accfull_bar[ab], (gt / kAccBufs) & 1u, s_abort, p.wait_ns));
         if (!ok) break;
         tc_fence_after_sync();
         const int tile_c0 = sh.key_begin + ti * kTcKeyTile;
@@ -310,7 +312,7 @@ __global__ void __launch_bounds__(1024) tc_merge_kernel(const ScoreParams p) {
   const int per_split = kAccBufs * group_reps;               // partial statistics of this row per split
   const int entries = kAccBufs * group_entries;
   const int b = unit / p.n_kv_heads;
-  const int t = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+  const int t = min(p.cu_seqlens[b + 1] - p.cu_seqlens[b], p.max_seqlen);
   const int n_splits_u = (t + p.split_keys - 1) / p.split_keys;
   const float2* part = p.stats_part + (size_t)unit * p.n_splits * entries + r;
   const int n = n_splits_u * per_split;
@@ -363,15 +365,15 @@ xkv_status tc_launch(const CUtensorMap& tq, const CUtensorMap& tk, const ScorePa
   using C = TcCfg<D, M>;
   size_t smem = C::kSmemBytes;
   if (smem < 120 * 1024) smem = 120 * 1024;      // one CTA per SM: it may hold all 512 TMEM columns
-  static bool done[64] = {};
+  static std::atomic<bool> done[64];   // idempotent set-up: two threads doing it twice is harmless
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
-  if (!done[dev]) {
+  if (!done[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(score_tc_kernel<D, M, PASS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)smem) != cudaSuccess)      // the kernel also has a few KB of static shared memory
       return XKV_ERR_CUDA;
-    done[dev] = true;
+    done[dev].store(true, std::memory_order_release);
   }
   int grid = sm_count();
   if (grid > p.n_work) grid = p.n_work;

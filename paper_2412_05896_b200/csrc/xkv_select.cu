@@ -40,13 +40,13 @@ struct SelectParams {
   int64_t total_tokens, stride_token, stride_head;
   int32_t batch, n_kv_heads, head_dim, window, page_size, max_pages_per_seq, n_pages;
   int2* counts;                // [units][n_chunks] scores above / equal to the threshold per chunk (chunked path)
-  int32_t n_chunks;
+  int32_t n_chunks, max_seqlen;
   WorkspaceHeader* hdr;
 };
 
 __device__ __forceinline__ void unit_shape(const SelectParams& p, int b, int* cu, int* t, int* P, int* kb) {
   *cu = p.cu_seqlens[b];
-  *t = p.cu_seqlens[b + 1] - *cu;
+  *t = min(p.cu_seqlens[b + 1] - *cu, p.max_seqlen);     // a longer prompt is cut to the bound the buffers were sized for
   *P = max(*t - p.window, 0);
   const int budget = p.budget_dev != nullptr ? p.budget_dev[b] : p.budget;
   *kb = min(budget, *P);
@@ -344,8 +344,9 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
   p.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
   p.counts = reinterpret_cast<int2*>(ws + L.counts);
   p.n_chunks = L.n_chunks;
+  p.max_seqlen = max_seqlen;
 
-  if (cudaMemsetAsync(ws, 0, kHeaderBytes, st) != cudaSuccess) return XKV_ERR_CUDA;
+  if (cudaMemsetAsync(ws + 4, 0, kHeaderBytes - 4, st) != cudaSuccess) return XKV_ERR_CUDA;   // the status word stays
   if (per_sequence) {
     if (cudaMemcpyAsync(ws + L.budget, budget, (size_t)d->batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return XKV_ERR_CUDA;

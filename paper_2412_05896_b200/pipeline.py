@@ -1,7 +1,7 @@
 """The call a user makes: one object that owns the device buffers of a batch (torch tensors for
 memory and streams only) and drives the four library entry points in order.
 
-    sess = XkvSession(...); sess.prefill(q_win, k, v, total_budget=...); sess.decode(q, k_new, v_new)
+    sess = XkvSession(...); sess.prefill(q_win, k, v, total=...); sess.decode(q, k_new, v_new)
 
 Every computation happens inside libxkv.so; this file allocates, copies and calls.
 """
@@ -227,10 +227,13 @@ class XkvSession:
         return out
 
     def device_status(self, which: str = "decode") -> int:
+        """First error any call of that kind recorded since the last check (the status words are sticky and
+        reading resets them), XKV_OK otherwise."""
         self.join()
         ws = {"decode": [self.ws_decode], "score": self.ws_score, "select": self.ws_select}[which]
+        first = xkv.OK
         for w in ws:
             st = xkv.read_device_status(w)
-            if st != xkv.OK:
-                return st
-        return xkv.OK
+            if st != xkv.OK and first == xkv.OK:
+                first = st
+        return first

@@ -24,7 +24,7 @@ STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
            "xkv_workspace_bytes",
-           "xkv_read_device_status", "xkv_profile_events", "xkv_launch_count", "xkv_status_string",
+           "xkv_read_device_status", "xkv_profile_events", "xkv_test_hooks", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
 
 
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
     L.xkv_read_device_status.argtypes = [vp, vp]
     L.xkv_profile_events.restype = None
     L.xkv_profile_events.argtypes = [vp, vp]
+    L.xkv_test_hooks.restype = None
+    L.xkv_test_hooks.argtypes = [i64, i32]
     L.xkv_launch_count.restype = i64
     L.xkv_launch_count.argtypes = []
     L.xkv_status_string.restype = ctypes.c_char_p
@@ -208,5 +210,12 @@ def profile_events(start, stop) -> None:
                              None if stop is None else stop.cuda_event)
 
 
+def test_hooks(wait_limit_ns: int = 0, withhold_decode_item: int = -1) -> None:
+    """Shortens every bounded device wait and/or withholds one decode merge ticket (tests of the expiry path);
+    test_hooks() restores the defaults."""
+    lib().xkv_test_hooks(wait_limit_ns, withhold_decode_item)
+
+
 def read_device_status(workspace, stream=None) -> int:
+    """The workspace's sticky status word (first error since the last read); reading resets it."""
     return lib().xkv_read_device_status(_ptr(workspace), _stream(stream))

@@ -171,7 +171,7 @@ def test_alloc_budgets_ties_and_unsorted_curves(seed):
 
 
 def test_average_budgets_matches_oracle_and_keeps_the_total():
-    """Online scenario (Sec. IV-D): layer-wise average of the recorded lists."""
+    """Online scenario (Sec. IV-C): layer-wise average of the recorded lists."""
     # by hand: means 4, 14/3, 22/3; recorded totals 16 each -> floors 4, 4, 7 and one slot to the larger fraction 2/3
     assert O.averaged_allocation([[3, 5, 8], [4, 4, 8], [5, 5, 6]]) == [4, 5, 7]
     assert xkv.average_budgets([[3, 5, 8], [4, 4, 8], [5, 5, 6]]).tolist() == [4, 5, 7]

@@ -22,7 +22,7 @@ def _run_case(L, B, Hq, Hkv, d, lens, page_size, chunk_rows, append, seed, stres
     handle = cache.handle()
     ws_bytes = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L,
                                    max_cache_len=cache.max_pages * page_size, chunk_rows=chunk_rows)
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=DEV)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=DEV)
     out = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
     lse = torch.empty(L, B, Hq, dtype=torch.float32, device=DEV)
     g = torch.Generator(device="cpu").manual_seed(seed + 1000)
@@ -104,7 +104,7 @@ def test_decode_score_profiles_along_the_cache(profile):
     G = Hq // Hkv
     q = torch.stack([u[h // G] for h in range(Hq)])[None, None].repeat(L, B, 1, 1).to(torch.bfloat16)
     for chunk_rows in (0, 128):
-        ws = torch.empty(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=cache.max_pages * ps,
+        ws = torch.zeros(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=cache.max_pages * ps,
                                              chunk_rows=chunk_rows), dtype=torch.uint8, device=DEV)
         out = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
         lse = torch.empty(L, B, Hq, dtype=torch.float32, device=DEV)
@@ -141,7 +141,7 @@ def test_decode_capacity_overflow_is_reported_not_faulted():
     cache = DirectCache(L, B, Hkv, d, [[16, 5]], ps, extra_rows=0, device=DEV, seed=1)
     assert cache.max_pages == 1                      # sequence 0 is exactly full
     dims = xkv.Dims(B, Hq, Hkv, d, 16, 1, 0, 0.0, Hkv * d, d)
-    ws = torch.empty(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=ps),
+    ws = torch.zeros(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=ps),
                      dtype=torch.uint8, device=DEV)
     q = torch.randn(L, B, Hq, d, device=DEV).to(torch.bfloat16)
     kn = torch.randn(L, B, Hkv, d, device=DEV).to(torch.bfloat16)
@@ -150,3 +150,36 @@ def test_decode_capacity_overflow_is_reported_not_faulted():
     torch.cuda.synchronize()
     assert xkv.read_device_status(ws) == xkv.ERR_CAPACITY
     assert cache.seq_lens.cpu().tolist() == [[16, 6]]
+
+
+def test_bounded_wait_expires_with_a_status_and_the_workspace_stays_usable():
+    """Failure detection without a fault: the split-K merge of one head waits for a chunk whose ticket a test
+    hook withholds, with the wait limit shortened to a millisecond.  The kernel must return, the status word
+    must read XKV_ERR_TIMEOUT, and the next ordinary call on the same workspace must be clean and correct."""
+    require_lib()
+    L, B, Hq, Hkv, d, ps, chunk_rows = 1, 2, 4, 2, 128, 16, 64
+    lens = [[300, 40]]
+    cache = DirectCache(L, B, Hkv, d, lens, ps, extra_rows=1, device=DEV, seed=31)
+    dims = xkv.Dims(B, Hq, Hkv, d, 16, 1, 0, 0.0, Hkv * d, d)
+    ws = torch.zeros(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=cache.max_pages * ps,
+                                         chunk_rows=chunk_rows), dtype=torch.uint8, device=DEV)
+    q = torch.randn(L, B, Hq, d, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).to(DEV)
+    out = torch.zeros(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
+    try:
+        xkv.test_hooks(wait_limit_ns=1_000_000, withhold_decode_item=2)    # a chunk of sequence 0, KV head 0
+        xkv.decode_attn(dims, cache.handle(), 0, L, q, None, None, out, None, chunk_rows, ws)
+        torch.cuda.synchronize()
+    finally:
+        xkv.test_hooks()
+    assert xkv.read_device_status(ws) == xkv.ERR_TIMEOUT
+    assert xkv.read_device_status(ws) == xkv.OK                            # reading reset the word
+    xkv.decode_attn(dims, cache.handle(), 0, L, q, None, None, out, None, chunk_rows, ws)
+    torch.cuda.synchronize()
+    assert xkv.read_device_status(ws) == xkv.OK
+    G = Hq // Hkv
+    ref = np.zeros((L, B, Hq, d))
+    for b in range(B):
+        K, V = f64(cache.K[(0, b)]), f64(cache.V[(0, b)])
+        for h in range(Hq):
+            ref[0, b, h], _ = O.decode_attention(f64(q[0, b, h]), K[:, h // G], V[:, h // G])
+    check_attention(out, ref, "call after the expired wait")

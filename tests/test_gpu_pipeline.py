@@ -147,7 +147,7 @@ def test_full_budget_reproduces_full_attention():
 
 
 def test_online_scenario_averaged_list_applied_to_a_new_task():
-    """Sec. IV-D: allocation lists recorded on a few sampled tasks are averaged, and a later task of the same type
+    """Sec. IV-C: allocation lists recorded on a few sampled tasks are averaged, and a later task of the same type
     is evicted under the averaged list without running the allocation.  Uses the paper's own defaults (observation
     window 8, average pooling of size 7)."""
     require_lib()

@@ -69,6 +69,13 @@ CASES = [
     ([4096, 31, 32, 33, 160], 3, 3, 64, 32, 5, 1),   # G*W = 32, clusters of four, lengths around the window
     ([300, 1000, 5], 4, 4, 64, 8, 7, 1),         # G*W = 8 (MHA with the paper's window of 8): padded to 16 rows
     ([700, 129], 6, 2, 128, 8, 7, 0),            # G*W = 24: padded to 32 rows
+    # the two-pass tensor-core kernels in every shape the dispatcher can pick (query rows x head dimension)
+    ([2300, 900], 8, 1, 128, 8, 7, 1),           # G*W = 64, d = 128 (eight query heads per KV head, the paper's window of 8)
+    ([1800, 2600], 4, 2, 64, 32, 5, 0),          # G*W = 64, d = 64
+    ([9100, 300], 2, 2, 128, 32, 7, 0),          # G*W = 32, d = 128, a prompt beyond what the single-read kernel holds
+    ([8300, 1000], 1, 1, 64, 32, 3, 0),          # G*W = 32, d = 64, likewise
+    ([2100, 640], 8, 2, 64, 32, 7, 0),           # G*W = 128, d = 64
+    ([1700, 130], 8, 1, 64, 32, 5, 1),           # G*W = 256, d = 64
 ]
 
 
@@ -194,7 +201,7 @@ def test_select_per_sequence_budgets_and_capacity_status():
     assert sess.seq_lens[0].cpu().tolist() == [0, 0]
 
 
-@pytest.mark.parametrize("lengths,Hq,Hkv,d,W,ps,mode", CASES[:5])
+@pytest.mark.parametrize("lengths,Hq,Hkv,d,W,ps,mode", CASES[:5] + CASES[11:])
 def test_selection_from_gpu_scores_matches_oracle_outside_near_ties(lengths, Hq, Hkv, d, W, ps, mode):
     """End to end through scoring: kept sets equal the oracle's wherever no other score lies within
     1e-5 (relative) of the k-th largest; inside that band only the band itself may differ."""
@@ -223,3 +230,35 @@ def test_selection_from_gpu_scores_matches_oracle_outside_near_ties(lengths, Hq,
                 else:
                     assert np.array_equal(got, keep), (budget, b, g)
     print(f"near-tie heads: {near} of {total}")
+
+
+def test_status_of_an_early_layer_survives_the_later_layers_of_the_phase():
+    """Layers share a few workspaces.  A layer whose budget does not fit its page table must still show in the
+    phase's status after later layers, which fit, have run on the same workspace."""
+    require_lib()
+    lengths, Hkv, W, d, L = [600, 900], 2, 16, 64, 6
+    q, k, v = _inputs(3, lengths, Hkv, Hkv, d, W)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    sess = XkvSession(L, Hkv, Hkv, d, W, 5, lengths, device=DEV, max_budget=200, n_lanes=2)
+    sess.score_layers([qd] * L, [kd] * L)
+    assert sess.device_status("score") == xkv.OK
+    budgets = np.array([50, 800, 60, 70, 80, 90], dtype=np.int32)       # layer 1 overflows its 200-token page table
+    sess.assign_pages(np.minimum(budgets, 200))
+    sess.select_layers(budgets, [kd] * L, [vd] * L)
+    torch.cuda.synchronize()
+    assert sess.device_status("select") == xkv.ERR_CAPACITY
+    assert sess.device_status("select") == xkv.OK                        # read once, then clean
+    lens = sess.seq_lens.cpu().numpy()
+    assert lens[1].tolist() == [0, 0] and lens[0].tolist() == [50 + W, 50 + W] and lens[5].tolist() == [90 + W, 90 + W]
+
+
+def test_prompt_longer_than_max_seqlen_is_reported_not_waited_for():
+    """max_seqlen sizes the grids; a longer prompt on the device is cut to it and flagged, with no stall."""
+    require_lib()
+    lengths, Hq, Hkv, d, W = [1500, 400], 4, 2, 128, 16
+    q, k, v = _inputs(9, lengths, Hq, Hkv, d, W)
+    sess = XkvSession(1, Hq, Hkv, d, W, 5, lengths, device=DEV)
+    sess.max_seqlen = 1024                                                # a wrong bound, below the first prompt
+    sess.score_layer(0, q.to(DEV), k.to(DEV))
+    torch.cuda.synchronize()
+    assert sess.device_status("score") == xkv.ERR_INVALID_ARG

@@ -88,8 +88,16 @@ def test_allocation_single_layer_and_batch_mean():
     g = O.head_gains(np.array([1.0, 2.0, 3.0]))
     A, r = O.adaptive_allocation([g], N=2)
     assert A == [2] and abs(r - 5.0 / 6.0) < 1e-15
-    x = np.arange(24, dtype=np.float64).reshape(2, 3, 4)
-    assert np.allclose(O.batch_mean_gains(x), x.mean(axis=1))
+    # batch mean of the curves, numbers written out by hand: 2 layers x 2 sequences x 3 ranks
+    x = np.array([[[0.50, 0.25, 0.25], [0.70, 0.20, 0.00]],
+                  [[1.00, 0.00, 0.00], [0.40, 0.35, 0.25]]])
+    want = np.array([[0.60, 0.225, 0.125],
+                     [0.70, 0.175, 0.125]])
+    got = O.batch_mean_gains(x)
+    assert got.shape == (2, 3) and np.max(np.abs(got - want)) < 1e-15
+    # a sequence shorter than the others contributes zeros beyond its prefix: the mean is over all B sequences
+    y = np.array([[[0.9, 0.1, 0.0, 0.0], [0.4, 0.3, 0.2, 0.1], [1.0, 0.0, 0.0, 0.0]]])
+    assert np.max(np.abs(O.batch_mean_gains(y) - np.array([[2.3 / 3, 0.4 / 3, 0.2 / 3, 0.1 / 3]]))) < 1e-15
 
 
 # ------------------------------------------------------------------ TopK / EvictByIndex

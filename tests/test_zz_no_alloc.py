@@ -9,9 +9,10 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import xkv_oracle as O
 from paper_2412_05896_b200 import xkv
 
-from gpu_util import ATOL, RTOL, DirectCache, require_lib
+from gpu_util import ATOL, RTOL, DirectCache, check_attention, f64, require_lib
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -29,7 +30,7 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
     need = xkv.workspace_bytes(xkv.OP_DECODE_ATTN, dims, n_layers=L, max_cache_len=ref_cache.max_pages * ps,
                                chunk_rows=chunk_rows)
     assert need <= xkv.STATIC_SCRATCH_BYTES
-    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    ws = torch.zeros(need, dtype=torch.uint8, device=DEV)
     out_ref = torch.empty(L, B, Hq, d, dtype=torch.bfloat16, device=DEV)
     out_sta = torch.empty_like(out_ref)
     lse_ref = torch.empty(L, B, Hq, dtype=torch.float32, device=DEV)
@@ -52,6 +53,15 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
         fin = np.isfinite(la)
         assert np.array_equal(fin, np.isfinite(lb)) and np.allclose(la[fin], lb[fin], atol=2e-3, rtol=1e-4)
         assert torch.equal(ref_cache.seq_lens, sta_cache.seq_lens)
+        # and against the fp64 attention of Eq. 1 over the same rows, so that this file stands on its own
+        sta_cache.append_host(kn, vn)
+        want = np.zeros((L, B, Hq, d))
+        for l in range(L):
+            for bb in range(B):
+                K, V = f64(sta_cache.K[(l, bb)]), f64(sta_cache.V[(l, bb)])
+                for h in range(Hq):
+                    want[l, bb, h], _ = O.decode_attention(f64(q[l, bb, h]), K[:, h // (Hq // Hkv)], V[:, h // (Hq // Hkv)])
+        check_attention(out_sta, want, f"call {call} against the oracle")
 
 
 def test_static_scratch_rejects_problems_beyond_its_size():
