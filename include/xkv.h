@@ -6,6 +6,7 @@
  *   1. xkv_score          per layer: observation-window attention weights -> pooled importance
  *                         scores per KV head, their descending sort, and the layer's
  *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
+ *      xkv_batch_curves   device: one curve per layer from the batch's curves         (Alg. 1, input W)
  *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
  *      xkv_average_budgets  host: the averaged list of the online scenario           (Sec. IV-C)
  *   3. xkv_select_compact per layer: top-k per (sequence, KV head) and gather of the kept K/V
@@ -159,6 +160,23 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
                              int32_t* budgets, double* r_avg);
 
 /*
+ * xkv_batch_curves -- the batch's curve of every layer, formed on the device (Alg. 1 takes one w per
+ * layer: for a batch that is the mean over its sequences of the per-sequence curves xkv_score wrote).
+ *
+ *   out[l][j] = (sum over b of gains[l][b][j]) / divisor      summed in the order of b, in double precision
+ *
+ * gains      dev fp32 [n_layers][batch][curve_len]
+ * divisor    batch for the mean of one GPU's batch; the total number of sequences of all ranks when the
+ *            per-rank results are afterwards summed across ranks
+ * out        dev out fp32 [n_layers][curve_len]; copied to the host it is the `gains` argument of
+ *            xkv_alloc_budgets with batch = 1 and prefix_len = max_b P_b, which gives the list that
+ *            per_sequence = 0 gives on the full array (up to the rounding of the mean to fp32), while only
+ *            n_layers * curve_len numbers cross to the host.
+ */
+xkv_status xkv_batch_curves(const float* gains, int32_t n_layers, int32_t batch, int32_t curve_len, int32_t divisor,
+                            float* out, void* stream);
+
+/*
  * xkv_average_budgets -- the averaged allocation list of the online scenario (Sec. IV-C), host only.
  *
  * The lists that xkv_alloc_budgets produced for a sample of tasks of one type are averaged layer by
@@ -203,6 +221,16 @@ xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t
                               int64_t total_tokens, int32_t max_seqlen, const xkv_cache* cache,
                               int32_t* sel, int32_t sel_stride,
                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * xkv_build_block_table -- fills cache->block_table for runs of consecutive pages (no counterpart in the
+ * paper: bookkeeping of the reduced caches whose sizes differ per layer, Sec. IV-A).
+ *   block_table[l][b][i] = first_page[l][b] + i  for i < n_pages_lb[l][b],  0 otherwise
+ * first_page, n_pages_lb  dev int32 [n_layers][batch]; which pages a (layer, sequence) gets is the caller's
+ *            decision (it owns the pool), the library only expands it on the device.
+ */
+xkv_status xkv_build_block_table(const int32_t* first_page, const int32_t* n_pages_lb, const xkv_cache* cache,
+                                 int32_t batch, void* stream);
 
 /*
  * xkv_decode_attn -- one generation step of attention over the reduced caches of layers

@@ -137,6 +137,23 @@ xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t
                         static_cast<cudaStream_t>(stream));
 }
 
+xkv_status xkv_batch_curves(const float* gains, int32_t n_layers, int32_t batch, int32_t curve_len, int32_t divisor,
+                            float* out, void* stream) {
+  if (gains == nullptr || out == nullptr || !aligned16(gains) || !aligned16(out)) return XKV_ERR_INVALID_ARG;
+  if (n_layers <= 0 || batch <= 0 || curve_len <= 0 || divisor <= 0) return XKV_ERR_INVALID_ARG;
+  return batch_curves(gains, n_layers, batch, curve_len, 1.0 / (double)divisor, out, static_cast<cudaStream_t>(stream));
+}
+
+xkv_status xkv_build_block_table(const int32_t* first_page, const int32_t* n_pages_lb, const xkv_cache* cache,
+                                 int32_t batch, void* stream) {
+  if (first_page == nullptr || n_pages_lb == nullptr || cache == nullptr || cache->block_table == nullptr)
+    return XKV_ERR_INVALID_ARG;
+  if (!aligned16(first_page) || !aligned16(n_pages_lb) || !aligned16(cache->block_table)) return XKV_ERR_INVALID_ARG;
+  if (batch <= 0 || cache->n_layers <= 0 || cache->max_pages_per_seq <= 0) return XKV_ERR_INVALID_ARG;
+  return build_block_table(first_page, n_pages_lb, cache->n_layers * batch, cache->block_table,
+                           cache->max_pages_per_seq, static_cast<cudaStream_t>(stream));
+}
+
 xkv_status xkv_decode_attn(const xkv_dims* dims, const xkv_cache* cache, int32_t layer_begin, int32_t layer_end,
                            const void* q, const void* k_new, const void* v_new, void* out, float* lse,
                            int32_t chunk_rows, void* workspace, size_t workspace_bytes, void* stream) {

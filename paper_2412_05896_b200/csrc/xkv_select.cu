@@ -278,6 +278,27 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
   }
 }
 
+// block_table[l][b][i] = first_page[l][b] + i for i < n_pages_lb[l][b], else 0.  grid = (L*B), any block size.
+__global__ void block_table_kernel(const int32_t* first_page, const int32_t* n_pages_lb, int32_t* block_table,
+                                   int max_pages_per_seq) {
+  const int lb = blockIdx.x;
+  const int first = first_page[lb], n = n_pages_lb[lb];
+  int32_t* row = block_table + (size_t)lb * max_pages_per_seq;
+  for (int i = threadIdx.x; i < max_pages_per_seq; i += blockDim.x) row[i] = i < n ? first + i : 0;
+}
+
+// out[l][j] = scale * sum over b of gains[l][b][j], summed in the order of b in double precision (the same
+// result on every run).  grid = (tiles of 256 ranks, L).
+__global__ void batch_curves_kernel(const float* gains, int batch, int curve_len, double scale, float* out) {
+  const int l = blockIdx.y;
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= curve_len) return;
+  const float* g = gains + (size_t)l * batch * curve_len + j;
+  double acc = 0.0;
+  for (int b = 0; b < batch; ++b) acc += (double)g[(size_t)b * curve_len];
+  out[(size_t)l * curve_len + j] = (float)(acc * scale);
+}
+
 struct SelectLayout {
   size_t budget, sel, counts, total;
   int sel_stride, n_chunks;
@@ -294,6 +315,20 @@ void select_layout(const xkv_dims* d, int max_seqlen, SelectLayout* L) {
 }
 
 }  // namespace
+
+xkv_status build_block_table(const int32_t* first_page, const int32_t* n_pages_lb, int n_lb, int32_t* block_table,
+                             int max_pages_per_seq, cudaStream_t st) {
+  block_table_kernel<<<n_lb, 128, 0, st>>>(first_page, n_pages_lb, block_table, max_pages_per_seq);
+  count_launch();
+  return check_launch();
+}
+
+xkv_status batch_curves(const float* gains, int n_layers, int batch, int curve_len, double scale, float* out,
+                        cudaStream_t st) {
+  batch_curves_kernel<<<dim3((curve_len + 255) / 256, n_layers), 256, 0, st>>>(gains, batch, curve_len, scale, out);
+  count_launch();
+  return check_launch();
+}
 
 size_t select_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens) {
   (void)total_tokens;

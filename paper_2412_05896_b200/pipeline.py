@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import math
+import time
 
 import numpy as np
 import torch
@@ -47,7 +48,11 @@ class XkvSession:
         self.scores = torch.empty(n_layers, n_kv_heads, self.T, **f32)
         self.sorted = torch.empty(n_layers, n_kv_heads, self.T, **f32)
         self.gains = torch.empty(n_layers, self.B, self.curve_len, **f32)
-        self.gains_host = torch.empty(n_layers, self.B, self.curve_len, dtype=torch.float32, pin_memory=True)
+        # what crosses to the host for the solver: one curve per layer (the batch mean, formed on the device);
+        # the per-sequence curves cross only when every sequence gets its own list
+        self.layer_gains = torch.empty(n_layers, self.curve_len, **f32)
+        self.layer_gains_host = torch.empty(n_layers, self.curve_len, dtype=torch.float32, pin_memory=True)
+        self.gains_host = None
         # Layers are independent in the scoring and in the eviction phase, so consecutive layers go to
         # n_lanes side streams, each with its own workspace: the short latency-bound kernels of one layer
         # (sort, curves, selection) then run under the HBM-bound ones of the next.
@@ -77,8 +82,9 @@ class XkvSession:
         self.v_pages = torch.zeros(self.n_pages, n_kv_heads, page_size, head_dim, **bf16)
         self.block_table = torch.zeros(n_layers, self.B, self.max_pages_per_seq, dtype=torch.int32,
                                        device=self.device)
-        self.block_table_host = torch.zeros(n_layers, self.B, self.max_pages_per_seq, dtype=torch.int32,
-                                            pin_memory=(self.device.type == "cuda"))
+        # page runs of every (layer, sequence): [0] first page, [1] number of pages; expanded on the device
+        self.page_runs_host = [torch.zeros(n_layers, self.B, dtype=torch.int32, pin_memory=True) for _ in range(2)]
+        self.page_runs = [torch.zeros(n_layers, self.B, dtype=torch.int32, device=self.device) for _ in range(2)]
         self.seq_lens = torch.zeros(n_layers, self.B, dtype=torch.int32, device=self.device)
         self.cache = xkv.Cache(self.k_pages.data_ptr(), self.v_pages.data_ptr(), self.block_table.data_ptr(),
                                self.seq_lens.data_ptr(), n_layers, page_size, self.max_pages_per_seq,
@@ -90,6 +96,7 @@ class XkvSession:
         self.out = torch.empty(n_layers, self.B, n_q_heads, head_dim, **bf16)
         self.lse = torch.empty(n_layers, self.B, n_q_heads, **f32)
         self.budgets: np.ndarray | None = None
+        self.last_solver_ms: float | None = None      # host time of the last xkv_alloc_budgets call
         self.r_avg: float | None = None
 
     def _ws(self, nbytes: int) -> torch.Tensor:
@@ -169,18 +176,32 @@ class XkvSession:
 
     def solve_budgets(self, total: int | None = None, r_target: float = 0.0, n_min: int = 0, n_max: int = 0,
                       per_sequence: bool = False):
-        """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host."""
+        """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host.  For one list per
+        batch the curves are averaged over the sequences on the device first, so L x curve_len numbers cross."""
         self.join()
-        self.gains_host.copy_(self.gains, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        budgets, r_avg = xkv.alloc_budgets(self.gains_host.numpy(), np.asarray(self.prefix, dtype=np.int32),
-                                           per_sequence=per_sequence, total=-1 if total is None else total,
+        if per_sequence:
+            if self.gains_host is None:
+                self.gains_host = torch.empty(self.L, self.B, self.curve_len, dtype=torch.float32, pin_memory=True)
+            self.gains_host.copy_(self.gains, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            gains, prefix = self.gains_host.numpy(), np.asarray(self.prefix, dtype=np.int32)
+        else:
+            xkv.batch_curves(self.gains, self.L, self.B, self.curve_len, self.B, self.layer_gains)
+            self.layer_gains_host.copy_(self.layer_gains, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            gains = self.layer_gains_host.numpy().reshape(self.L, 1, self.curve_len)
+            prefix = np.asarray([self.max_prefix], dtype=np.int32)
+        t0 = time.perf_counter()
+        budgets, r_avg = xkv.alloc_budgets(gains, prefix, per_sequence=per_sequence,
+                                           total=-1 if total is None else total,
                                            r_target=r_target, n_min=n_min, n_max=n_max)
+        self.last_solver_ms = 1e3 * (time.perf_counter() - t0)
         self.budgets, self.r_avg = budgets, r_avg
         return budgets, r_avg
 
     def assign_pages(self, budgets) -> None:
-        """Hand consecutive pool pages to every (layer, sequence) for its kept rows plus new tokens."""
+        """Hand consecutive pool pages to every (layer, sequence) for its kept rows plus new tokens: the runs are
+        computed here (2 x L x B integers), the page table is expanded from them on the device."""
         budgets = np.asarray(budgets)
         k_lb = budgets.T if budgets.ndim == 2 else np.broadcast_to(budgets[:, None], (self.L, self.B))   # [L, B]
         prefix = np.asarray(self.prefix)[None, :]
@@ -190,10 +211,10 @@ class XkvSession:
         start = np.concatenate([[0], np.cumsum(n.ravel())[:-1]]).reshape(self.L, self.B)
         if int(start.ravel()[-1] + n.ravel()[-1]) > self.n_pages:
             raise RuntimeError("page pool too small for these budgets")
-        idx = np.arange(self.max_pages_per_seq, dtype=np.int64)[None, None, :]
-        bt = self.block_table_host.numpy()
-        bt[:] = np.where(idx < n[:, :, None], start[:, :, None] + idx, 0).astype(np.int32)
-        self.block_table.copy_(self.block_table_host, non_blocking=True)
+        for dst, host, src in zip(self.page_runs, self.page_runs_host, (start, n)):
+            host.numpy()[:] = src
+            dst.copy_(host, non_blocking=True)
+        xkv.build_block_table(self.page_runs[0], self.page_runs[1], self.cache, self.B)
 
     def select_layer(self, layer: int, budget, k: torch.Tensor, v: torch.Tensor, sel: torch.Tensor | None = None,
                      per_sequence: bool = False) -> None:

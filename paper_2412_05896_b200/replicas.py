@@ -65,18 +65,22 @@ def whole_job_rate(units_local: float, ms_local: float, device="cpu") -> tuple[f
     return total / (ms_max * 1e-3), ms_max, total
 
 
-def batch_mean_curves_over_ranks(gains, device="cpu"):
-    """One budget list for the sequences of all ranks (instead of one list per replica): the curves the solver
-    averages over a batch are averaged over every rank's batch.  gains: float [L, B_local, curve_len] as written by
-    xkv_score (torch tensor or array; every rank must use the same L and curve_len).  Returns a torch float64
-    tensor [L, 1, curve_len] that xkv.alloc_budgets takes as a batch of one: the mean over all sequences of the
-    job.  This is the only exchange a sharded run of the path needs -- L x curve_len numbers, before the host
-    solver; K, V and the scores never leave their GPU.
+def count_over_ranks(n_local: int, device="cpu") -> int:
+    """Sum of an integer count over the ranks (e.g. the sequences of the whole job)."""
+    return int(round(sum_over_ranks(float(n_local), device)))
+
+
+def sum_curves_over_ranks(local_curves: torch.Tensor) -> torch.Tensor:
+    """One budget list for the units of all ranks (instead of one list per replica).  This is the only exchange a
+    sharded run of the path needs -- L x curve_len numbers, before the host solver; K, V and the scores never leave
+    their GPU.
+
+    local_curves: float tensor [L, curve_len], this rank's share of the job's curves, already weighted so that the
+    shares add up to the job's curve: xkv.batch_curves(..., divisor = sequences of all ranks) when the ranks hold
+    different sequences, or the rank's own mean divided by the number of ranks when they hold equal shares of the
+    KV heads.  Summed in place over the ranks (all-reduce) and returned; every rank then runs the same
+    deterministic host solver on it as a batch of one.  No arithmetic of the method happens here.
     """
-    g = torch.as_tensor(gains).to(device=device, dtype=torch.float64)
-    total = g.sum(dim=1, keepdim=True)
-    count = torch.tensor([float(g.shape[1])], device=device, dtype=torch.float64)
     if dist.is_initialized() and dist.get_world_size() > 1:
-        dist.all_reduce(total, op=dist.ReduceOp.SUM)
-        dist.all_reduce(count, op=dist.ReduceOp.SUM)
-    return total / count
+        dist.all_reduce(local_curves, op=dist.ReduceOp.SUM)
+    return local_curves

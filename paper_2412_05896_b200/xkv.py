@@ -22,7 +22,7 @@ OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("xkv_score", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
+EXPORTS = ("xkv_score", "xkv_batch_curves", "xkv_build_block_table", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
            "xkv_workspace_bytes",
            "xkv_read_device_status", "xkv_profile_events", "xkv_test_hooks", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
@@ -63,6 +63,10 @@ def lib() -> ctypes.CDLL:
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     L.xkv_score.restype = i32
     L.xkv_score.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.xkv_batch_curves.restype = i32
+    L.xkv_batch_curves.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+    L.xkv_build_block_table.restype = i32
+    L.xkv_build_block_table.argtypes = [vp, vp, ctypes.POINTER(Cache), i32, vp]
     L.xkv_alloc_budgets.restype = i32
     L.xkv_alloc_budgets.argtypes = [vp, i32, i32, i32, vp, i32, i64, ctypes.c_double, i32, i32, vp, vp]
     L.xkv_average_budgets.restype = i32
@@ -151,6 +155,17 @@ def score(dims: Dims, q_win, k, cu_seqlens, total_tokens: int, max_seqlen: int, 
     _check(lib().xkv_score(ctypes.byref(dims), _ptr(q_win), _ptr(k), _ptr(cu_seqlens), total_tokens, max_seqlen,
                            _ptr(scores), _ptr(sorted_scores), _ptr(gains), _ptr(mass), curve_len,
                            _ptr(workspace), _nbytes(workspace), _stream(stream)), "xkv_score")
+
+
+def batch_curves(gains, n_layers: int, batch: int, curve_len: int, divisor: int, out, stream=None) -> None:
+    """gains dev [L, B, curve_len] -> out dev [L, curve_len] = sum over b / divisor."""
+    _check(lib().xkv_batch_curves(_ptr(gains), n_layers, batch, curve_len, divisor, _ptr(out), _stream(stream)),
+           "xkv_batch_curves")
+
+
+def build_block_table(first_page, n_pages_lb, cache: Cache, batch: int, stream=None) -> None:
+    _check(lib().xkv_build_block_table(_ptr(first_page), _ptr(n_pages_lb), ctypes.byref(cache), batch,
+                                       _stream(stream)), "xkv_build_block_table")
 
 
 def alloc_budgets(gains: np.ndarray, prefix_len, per_sequence: bool = False, total: int = -1,

@@ -75,7 +75,11 @@ def _curve_worker(rank: int, world: int, port: int, out):
     all_curves = np.stack([[O.head_gains(rng.random(n) ** (2 + l)) for _ in range(5)] for l in range(L)])   # [L, 5, n]
     mine = all_curves[:, :2] if rank == 0 else all_curves[:, 2:]
     assert mine.shape[1] == b_local
-    shared = replicas.batch_mean_curves_over_ranks(mine.astype(np.float32)).numpy()
+    n_seq = replicas.count_over_ranks(b_local)
+    assert n_seq == 5
+    # this rank's share of the job's curve (on a GPU xkv_batch_curves forms it with divisor = n_seq)
+    share = torch.from_numpy(mine.astype(np.float32).astype(np.float64).sum(axis=1) / n_seq)
+    shared = replicas.sum_curves_over_ranks(share).numpy()[:, None, :]
     budgets, r = xkv.alloc_budgets(shared.astype(np.float32), [n], total=60, n_min=2)
     whole, r_whole = xkv.alloc_budgets(all_curves.astype(np.float32), [n] * 5, total=60, n_min=2)
     out.put((rank, budgets.tolist(), whole.tolist(), float(np.abs(shared[:, 0] - all_curves.astype(np.float32).mean(1)).max())))
