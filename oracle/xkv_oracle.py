@@ -278,6 +278,26 @@ def bruteforce_allocation(gains: list[np.ndarray], N: int, n_min: int = 0,
     return best, best_val
 
 
+def head_level_allocation(w_layers: list[list[np.ndarray]], N: int | None = None, R_avg: float | None = None,
+                          n_min: int = 0, n_max: int | None = None) -> tuple[list[list[int]], float]:
+    """Head-level budgets inside the layers (Sec. II-C: cache sizes pre-set per attention head work together with
+    the layer-centric allocation).  Reading taken here: the unit that waits for slots in Algorithm 1 is a
+    (layer, KV head) pair instead of a layer, each with its own curve Sort(w)/Sum(w) (Eq. 21 for that head);
+    N is then the number of cached prefix tokens summed over all heads of all layers, and the objective is the
+    mean over all heads of Eq. 4.  Units are ordered layer-major, so ties go to the lower layer, then the lower
+    head.
+
+    w_layers[l][g]: pooled score vector of KV head g of layer l (one sequence).  Returns (n[l][g], mean R).
+    """
+    flat = [head_gains(w) for heads in w_layers for w in heads]
+    held, r = adaptive_allocation(flat, N=N, R_avg=R_avg, n_min=n_min, n_max=n_max)
+    out, i = [], 0
+    for heads in w_layers:
+        out.append(held[i: i + len(heads)])
+        i += len(heads)
+    return out, r
+
+
 def batch_mean_gains(gains_lb: np.ndarray) -> np.ndarray:
     """gains_lb [L, B, curve_len] -> [L, curve_len]: mean over the sequences of a batch."""
     return np.mean(np.asarray(gains_lb, dtype=np.float64), axis=1)

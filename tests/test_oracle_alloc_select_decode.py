@@ -100,6 +100,59 @@ def test_allocation_single_layer_and_batch_mean():
     assert np.max(np.abs(O.batch_mean_gains(y) - np.array([[2.3 / 3, 0.4 / 3, 0.2 / 3, 0.1 / 3]]))) < 1e-15
 
 
+# ------------------------------------------------------------------ head-level budgets (Sec. II-C)
+def _bruteforce_heads(w_layers, N):
+    """Every split of N over the (layer, head) units; best mean over the units of Eq. 4, written out here."""
+    units = [np.sort(w)[::-1] / np.sum(w) for heads in w_layers for w in heads]
+    best = -1.0
+    for split in itertools.product(*[range(len(u) + 1) for u in units]):
+        if sum(split) == N:
+            best = max(best, sum(float(np.sum(u[:n])) for u, n in zip(units, split)) / len(units))
+    return best
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_head_level_allocation_matches_bruteforce(seed):
+    rng = np.random.default_rng(100 + seed)
+    w_layers = [[rng.random(int(rng.integers(2, 5))) ** 3 for _ in range(2)] for _ in range(2)]   # 2 layers x 2 heads
+    total = sum(len(w) for heads in w_layers for w in heads)
+    for N in range(0, total + 1):
+        n, r = O.head_level_allocation(w_layers, N=N)
+        assert sum(sum(row) for row in n) == N
+        assert [len(row) for row in n] == [2, 2]
+        assert abs(r - _bruteforce_heads(w_layers, N)) < 1e-13
+
+
+def test_head_level_allocation_against_the_layer_level_one():
+    rng = np.random.default_rng(7)
+    L, H, P = 3, 4, 12
+    # heads that differ: the head-level optimum is at least the layer-level one spread over the heads (which is a
+    # feasible point of the head-level problem with H times the slots), and strictly better for these scores
+    w_layers = [[rng.random(P) ** 4 for _ in range(H)] for _ in range(L)]
+    layer_curves = [O.layer_gains(heads, P) for heads in w_layers]
+    for N in (3, 9, 20):
+        A, r_layer = O.adaptive_allocation(layer_curves, N=N)
+        n, r_head = O.head_level_allocation(w_layers, N=H * N)
+        spread = sum(float(np.sum(O.head_gains(w)[:A[l]])) for l in range(L) for w in w_layers[l]) / (L * H)
+        assert abs(spread - r_layer) < 1e-13                       # the layer curve is the mean of its heads' curves
+        assert r_head >= r_layer - 1e-15
+    assert r_head > r_layer + 1e-6
+    # identical heads inside every layer: each head gets exactly its layer's count
+    w_same = [[w] * H for w in (rng.random(P) ** 3 for _ in range(L))]
+    curves = [O.head_gains(heads[0]) for heads in w_same]
+    for N in (1, 7, 15, 30):
+        A, r_layer = O.adaptive_allocation(curves, N=N)
+        n, r_head = O.head_level_allocation(w_same, N=H * N)
+        assert n == [[a] * H for a in A] and abs(r_head - r_layer) < 1e-13
+    # by hand: one layer, two heads w0 = (6, 3, 1) and w1 = (5, 5): the curves are (.6, .3, .1) and (.5, .5); three
+    # slots go to .6, then .5 (head 1), then .5 (head 1)
+    n, r = O.head_level_allocation([[np.array([1.0, 6.0, 3.0]), np.array([5.0, 5.0])]], N=3)
+    assert n == [[1, 2]] and abs(r - (0.6 + 1.0) / 2) < 1e-15
+    # the box applies per head
+    n, _ = O.head_level_allocation([[np.array([1.0, 6.0, 3.0]), np.array([5.0, 5.0])]], N=3, n_min=1, n_max=2)
+    assert n == [[1, 2]]
+
+
 # ------------------------------------------------------------------ TopK / EvictByIndex
 def test_topk_matches_bruteforce_sort():
     rng = np.random.default_rng(20)
