@@ -7,6 +7,7 @@
  *                         scores per KV head, their descending sort, and the layer's
  *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
  *      xkv_batch_curves   device: one curve per layer from the batch's curves         (Alg. 1, input W)
+ *      xkv_head_curves    device: one curve per (layer, KV head) for head-level budgets      (Sec. II-C)
  *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
  *      xkv_average_budgets  host: the averaged list of the online scenario           (Sec. IV-C)
  *   3. xkv_select_compact per layer: top-k per (sequence, KV head) and gather of the kept K/V
@@ -58,6 +59,11 @@ typedef int32_t xkv_status;
 #define XKV_POOL_MAX 0
 #define XKV_POOL_AVG 1
 
+/* What the `budget` argument of xkv_select_compact holds. */
+#define XKV_BUDGET_PER_LAYER    0 /* [1]: one count for every sequence and KV head of the layer (Alg. 1's n_i) */
+#define XKV_BUDGET_PER_SEQUENCE 1 /* [B]: one count per sequence (the paper's offline mode, one list per task) */
+#define XKV_BUDGET_PER_HEAD     2 /* [B][Hkv]: head-level budgets inside the layer (Sec. II-C)                 */
+
 #define XKV_OP_SCORE          0
 #define XKV_OP_SELECT_COMPACT 1
 #define XKV_OP_DECODE_ATTN    2
@@ -85,6 +91,15 @@ typedef struct xkv_dims {
  *   seq_lens          : dev int32 [n_layers][B], number of filled slots; written by
  *                       xkv_select_compact, advanced by xkv_decode_attn when it appends
  * page_size is a multiple of 16 (at most 256).
+ *
+ * Head-level budgets (XKV_BUDGET_PER_HEAD) give every KV head of a sequence a cache of its own length. The same
+ * structure then describes B*Hkv caches of one KV head each per layer:
+ *   k_pages / v_pages : dev bf16 [n_pages][1][page_size][d]
+ *   block_table       : dev int32 [n_layers][B*Hkv][max_pages_per_seq], cache index b*Hkv + g
+ *   seq_lens          : dev int32 [n_layers][B*Hkv]
+ * xkv_select_compact fills it when called with XKV_BUDGET_PER_HEAD, and xkv_decode_attn reads it when called
+ * with dims {batch = B*Hkv, n_q_heads = G, n_kv_heads = 1}: q, k_new, v_new, out and lse keep their memory
+ * layout ([Lr][B][Hq][d] is [Lr][B*Hkv][G][d]).
  */
 typedef struct xkv_cache {
   void*    k_pages;
@@ -177,6 +192,24 @@ xkv_status xkv_batch_curves(const float* gains, int32_t n_layers, int32_t batch,
                             float* out, void* stream);
 
 /*
+ * xkv_head_curves -- the curve of every KV head of one layer on its own: what Algorithm 1 consumes when the
+ * unit that waits for slots is a (layer, KV head) pair instead of a layer (head-level cache sizes working
+ * together with the layer-level allocation, Sec. II-C; per head the curve is Sort(w)/Sum(w) of Eq. 21).
+ *
+ *   head_gains[g][b][j] = sorted[g][cu_seqlens[b] + j] / sum over c < P_b of scores[g][cu_seqlens[b] + c]
+ *                         for j < min(P_b, curve_len), 0 for the other j < curve_len
+ *
+ * scores, sorted  dev fp32 [Hkv][T] as xkv_score wrote them for this layer
+ * head_gains      dev out fp32 [Hkv][B][curve_len]. The arrays of all layers, stacked, are [L*Hkv][B][curve_len]:
+ *                 the `gains` argument of xkv_batch_curves / xkv_alloc_budgets with n_layers = L*Hkv, whose
+ *                 budgets [L*Hkv] are then one count per (layer, KV head) and whose total is the number of
+ *                 cached prefix tokens summed over all heads of all layers.
+ */
+xkv_status xkv_head_curves(const xkv_dims* dims, const float* scores, const float* sorted,
+                           const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen,
+                           float* head_gains, int32_t curve_len, void* stream);
+
+/*
  * xkv_average_budgets -- the averaged allocation list of the online scenario (Sec. IV-C), host only.
  *
  * The lists that xkv_alloc_budgets produced for a sample of tasks of one type are averaged layer by
@@ -202,10 +235,13 @@ xkv_status xkv_average_budgets(const int32_t* lists, int32_t n_tasks, int32_t n_
  * bit-exactly from k and v into cache slots 0 .. kb + (t_b - P_b) - 1 of (layer, b) and
  * seq_lens[layer][b] is set to that count.
  *
- * budget     host int32 [1] (per_sequence = 0) or [B] (per_sequence = 1), each >= 0. With per_sequence = 1
- *            the array is copied to the device on `stream`: from pageable memory that copy waits
+ * per_sequence  XKV_BUDGET_PER_LAYER (0), XKV_BUDGET_PER_SEQUENCE (1) or XKV_BUDGET_PER_HEAD (2)
+ * budget     host int32 [1], [B] or [B][Hkv] accordingly, each >= 0. Arrays of more than one entry are
+ *            copied to the device on `stream`: from pageable memory that copy waits
  *            for the stream's earlier work; from pinned memory it is asynchronous, and the array
  *            must then stay alive and unchanged until the stream has passed this call.
+ *            With XKV_BUDGET_PER_HEAD, `cache` is the per-head form described at xkv_cache, kb and the
+ *            slot count are those of (b, g), and seq_lens[layer][b*Hkv + g] is set.
  * scores     dev fp32 [Hkv][T] (w of xkv_score, or any non-negative finite scores)
  * sorted     dev fp32 [Hkv][T] (descending per (g,b), as xkv_score writes it)
  * k, v       dev bf16, same layout and strides (dims.kv_stride_*)

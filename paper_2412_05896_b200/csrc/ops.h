@@ -23,6 +23,9 @@ xkv_status build_block_table(const int32_t* first_page, const int32_t* n_pages_l
 xkv_status batch_curves(const float* gains, int n_layers, int batch, int curve_len, double scale, float* out,
                         cudaStream_t st);
 
+xkv_status head_curves(const xkv_dims* d, const float* scores, const float* sorted, const int32_t* cu_seqlens,
+                       int64_t total_tokens, int max_seqlen, float* out, int curve_len, cudaStream_t st);
+
 size_t decode_workspace_bytes(const xkv_dims* d, int n_layers, int max_cache_len, int chunk_rows);
 xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, int layer_end, const void* q,
                        const void* k_new, const void* v_new, void* out, float* lse, int chunk_rows,

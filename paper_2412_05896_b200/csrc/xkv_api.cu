@@ -122,9 +122,13 @@ xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t
   if (layer < 0 || layer >= cache->n_layers) return XKV_ERR_INVALID_ARG;
   if (total_tokens <= 0 || total_tokens >= (1ll << 31) || max_seqlen <= 0 || max_seqlen > total_tokens)
     return XKV_ERR_INVALID_ARG;
-  if (per_sequence != 0 && per_sequence != 1) return XKV_ERR_INVALID_ARG;
+  if (per_sequence != XKV_BUDGET_PER_LAYER && per_sequence != XKV_BUDGET_PER_SEQUENCE &&
+      per_sequence != XKV_BUDGET_PER_HEAD)
+    return XKV_ERR_INVALID_ARG;
+  const int n_budgets = per_sequence == XKV_BUDGET_PER_HEAD ? dims->batch * dims->n_kv_heads
+                                                            : (per_sequence ? dims->batch : 1);
   int32_t max_budget = 0;
-  for (int i = 0; i < (per_sequence ? dims->batch : 1); ++i) {
+  for (int i = 0; i < n_budgets; ++i) {
     if (budget[i] < 0) return XKV_ERR_BUDGET;
     if (budget[i] > max_budget) max_budget = budget[i];
   }
@@ -142,6 +146,22 @@ xkv_status xkv_batch_curves(const float* gains, int32_t n_layers, int32_t batch,
   if (gains == nullptr || out == nullptr || !aligned16(gains) || !aligned16(out)) return XKV_ERR_INVALID_ARG;
   if (n_layers <= 0 || batch <= 0 || curve_len <= 0 || divisor <= 0) return XKV_ERR_INVALID_ARG;
   return batch_curves(gains, n_layers, batch, curve_len, 1.0 / (double)divisor, out, static_cast<cudaStream_t>(stream));
+}
+
+xkv_status xkv_head_curves(const xkv_dims* dims, const float* scores, const float* sorted, const int32_t* cu_seqlens,
+                           int64_t total_tokens, int32_t max_seqlen, float* head_gains, int32_t curve_len,
+                           void* stream) {
+  xkv_status s = check_prefill_dims(dims);
+  if (s != XKV_OK) return s;
+  if (scores == nullptr || sorted == nullptr || cu_seqlens == nullptr || head_gains == nullptr)
+    return XKV_ERR_INVALID_ARG;
+  if (!aligned16(scores) || !aligned16(sorted) || !aligned16(cu_seqlens) || !aligned16(head_gains))
+    return XKV_ERR_INVALID_ARG;
+  if (total_tokens <= 0 || total_tokens >= (1ll << 31) || max_seqlen <= 0 || max_seqlen > total_tokens ||
+      curve_len < 1)
+    return XKV_ERR_INVALID_ARG;
+  return head_curves(dims, scores, sorted, cu_seqlens, total_tokens, max_seqlen, head_gains, curve_len,
+                     static_cast<cudaStream_t>(stream));
 }
 
 xkv_status xkv_build_block_table(const int32_t* first_page, const int32_t* n_pages_lb, const xkv_cache* cache,

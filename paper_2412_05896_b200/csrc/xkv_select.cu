@@ -27,11 +27,12 @@ struct SelectParams {
   const float* scores;
   const float* sorted;
   const int32_t* cu_seqlens;
-  const int32_t* budget_dev;   // [B] when per-sequence, else null
+  const int32_t* budget_dev;   // [B] per sequence, [B][Hkv] per head, else null
   int32_t budget;              // shared budget otherwise
+  int32_t head_level;          // 1: budgets, cache lengths and page lists are per (sequence, KV head)
   int32_t* sel;                // [B][Hkv][sel_stride]
   int32_t sel_stride;
-  int32_t* seq_lens_layer;     // seq_lens + layer*B
+  int32_t* seq_lens_layer;     // seq_lens + layer*B (layer*B*Hkv when head_level)
   const int32_t* block_table_layer;
   const __nv_bfloat16* k;
   const __nv_bfloat16* v;
@@ -44,13 +45,21 @@ struct SelectParams {
   WorkspaceHeader* hdr;
 };
 
-__device__ __forceinline__ void unit_shape(const SelectParams& p, int b, int* cu, int* t, int* P, int* kb) {
+__device__ __forceinline__ void unit_shape(const SelectParams& p, int b, int g, int* cu, int* t, int* P, int* kb) {
   *cu = p.cu_seqlens[b];
   *t = min(p.cu_seqlens[b + 1] - *cu, p.max_seqlen);     // a longer prompt is cut to the bound the buffers were sized for
   *P = max(*t - p.window, 0);
-  const int budget = p.budget_dev != nullptr ? p.budget_dev[b] : p.budget;
+  const int budget = p.budget_dev == nullptr ? p.budget
+                                             : (p.head_level ? p.budget_dev[b * p.n_kv_heads + g] : p.budget_dev[b]);
   *kb = min(budget, *P);
 }
+
+// Index of the cache (its seq_lens entry and page list) that holds KV head g of sequence b, and whether this
+// (b, g) is the one that writes the entry: with head-level budgets every head has a cache of its own.
+__device__ __forceinline__ int cache_index(const SelectParams& p, int b, int g) {
+  return p.head_level ? b * p.n_kv_heads + g : b;
+}
+__device__ __forceinline__ bool writes_len(const SelectParams& p, int g) { return p.head_level || g == 0; }
 
 // Exclusive block scan of one int per thread (kSelThreads threads); returns the exclusive prefix
 // and writes the block total to *total.
@@ -85,11 +94,11 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectParams p) {
   __shared__ int s_warp[33];
   const int b = blockIdx.x / p.n_kv_heads, g = blockIdx.x % p.n_kv_heads;
   int cu, t, P, kb;
-  unit_shape(p, b, &cu, &t, &P, &kb);
+  unit_shape(p, b, g, &cu, &t, &P, &kb);
   const int n_keep = kb + (t - P);
   const bool fits = n_keep <= p.max_pages_per_seq * p.page_size;
-  if (threadIdx.x == 0 && g == 0) {
-    p.seq_lens_layer[b] = fits ? n_keep : 0;
+  if (threadIdx.x == 0 && writes_len(p, g)) {
+    p.seq_lens_layer[cache_index(p, b, g)] = fits ? n_keep : 0;
     if (!fits) record_status(p.hdr, XKV_ERR_CAPACITY);
   }
   if (!fits) return;
@@ -149,7 +158,7 @@ __global__ void __launch_bounds__(kSelThreads) select_count_kernel(SelectParams 
   const int unit = blockIdx.x, chunk = blockIdx.y;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
   int cu, t, P, kb;
-  unit_shape(p, b, &cu, &t, &P, &kb);
+  unit_shape(p, b, g, &cu, &t, &P, &kb);
   if (kb == 0 || kb == P || chunk * kSelChunk >= P) return;      // nothing to count: no selection by score
   const float* w = p.scores + (size_t)g * p.total_tokens + cu;
   const float thr = p.sorted[(size_t)g * p.total_tokens + cu + kb - 1];
@@ -173,11 +182,11 @@ __global__ void __launch_bounds__(kSelThreads) select_chunk_kernel(SelectParams 
   const int unit = blockIdx.x, chunk = blockIdx.y;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
   int cu, t, P, kb;
-  unit_shape(p, b, &cu, &t, &P, &kb);
+  unit_shape(p, b, g, &cu, &t, &P, &kb);
   const int n_keep = kb + (t - P);
   const bool fits = n_keep <= p.max_pages_per_seq * p.page_size;
-  if (chunk == 0 && threadIdx.x == 0 && g == 0) {
-    p.seq_lens_layer[b] = fits ? n_keep : 0;
+  if (chunk == 0 && threadIdx.x == 0 && writes_len(p, g)) {
+    p.seq_lens_layer[cache_index(p, b, g)] = fits ? n_keep : 0;
     if (!fits) record_status(p.hdr, XKV_ERR_CAPACITY);
   }
   if (!fits) return;
@@ -252,13 +261,14 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
   const int unit = blockIdx.x;
   const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
   int cu, t, P, kb;
-  unit_shape(p, b, &cu, &t, &P, &kb);
+  unit_shape(p, b, g, &cu, &t, &P, &kb);
   const int n_keep = kb + (t - P);
   if (n_keep > p.max_pages_per_seq * p.page_size) return;
   const int row0 = blockIdx.y * kGatherRows;
   if (row0 >= n_keep) return;
   const int32_t* sel = p.sel + (size_t)unit * p.sel_stride;
-  const int32_t* bt = p.block_table_layer + (size_t)b * p.max_pages_per_seq;
+  const int32_t* bt = p.block_table_layer + (size_t)cache_index(p, b, g) * p.max_pages_per_seq;
+  const int page_heads = p.head_level ? 1 : p.n_kv_heads, page_head = p.head_level ? 0 : g;
   const int lanes_per_row = p.head_dim / 8;                   // 16-byte lanes per row
   const int rows_per_pass = kGatherThreads / lanes_per_row;
   const int lr = threadIdx.x / lanes_per_row, lc = threadIdx.x % lanes_per_row;
@@ -270,7 +280,7 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
       continue;
     }
     const size_t src = (size_t)(cu + pos) * p.stride_token + (size_t)g * p.stride_head + lc * 8;
-    const size_t dst = (((size_t)page * p.n_kv_heads + g) * p.page_size + r % p.page_size) * p.head_dim + lc * 8;
+    const size_t dst = (((size_t)page * page_heads + page_head) * p.page_size + r % p.page_size) * p.head_dim + lc * 8;
     const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k + src));
     const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v + src));
     *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
@@ -299,6 +309,34 @@ __global__ void batch_curves_kernel(const float* gains, int batch, int curve_len
   out[(size_t)l * curve_len + j] = (float)(acc * scale);
 }
 
+// out[g][b][j] = sorted[g][cu_b + j] / sum over the prefix of scores[g][cu_b + c] (0 for j >= P_b).  grid = B*Hkv.
+// The sum runs in double precision in a fixed order (per-thread strided partial sums, then a tree), so the result
+// is the same on every run.
+__global__ void __launch_bounds__(1024) head_curves_kernel(const float* scores, const float* sorted,
+                                                           const int32_t* cu_seqlens, int64_t total_tokens,
+                                                           int max_seqlen, int window, int batch, int n_kv_heads,
+                                                           int curve_len, float* out) {
+  __shared__ double s_sum[1024];
+  const int b = blockIdx.x / n_kv_heads, g = blockIdx.x % n_kv_heads;
+  const int cu = cu_seqlens[b];
+  const int t = min(cu_seqlens[b + 1] - cu, max_seqlen);
+  const int P = max(t - window, 0);
+  const float* w = scores + (size_t)g * total_tokens + cu;
+  double acc = 0.0;
+  for (int c = threadIdx.x; c < P; c += 1024) acc += (double)w[c];
+  s_sum[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = 512; o > 0; o >>= 1) {
+    if (threadIdx.x < o) s_sum[threadIdx.x] += s_sum[threadIdx.x + o];
+    __syncthreads();
+  }
+  const double total = s_sum[0];
+  const double inv = total > 0.0 ? 1.0 / total : 0.0;
+  const float* srt = sorted + (size_t)g * total_tokens + cu;
+  float* o = out + ((size_t)g * batch + b) * curve_len;
+  for (int j = threadIdx.x; j < curve_len; j += 1024) o[j] = j < P ? (float)((double)srt[j] * inv) : 0.f;
+}
+
 struct SelectLayout {
   size_t budget, sel, counts, total;
   int sel_stride, n_chunks;
@@ -306,7 +344,7 @@ struct SelectLayout {
 
 void select_layout(const xkv_dims* d, int max_seqlen, SelectLayout* L) {
   size_t off = kHeaderBytes;
-  L->budget = off; off = align_up(off + (size_t)d->batch * 4, 256);
+  L->budget = off; off = align_up(off + (size_t)d->batch * d->n_kv_heads * 4, 256);
   L->sel_stride = (max_seqlen + 3) / 4 * 4;
   L->sel = off;    off = align_up(off + (size_t)d->batch * d->n_kv_heads * L->sel_stride * 4, 256);
   L->n_chunks = (max_seqlen + kSelChunk - 1) / kSelChunk;
@@ -330,6 +368,14 @@ xkv_status batch_curves(const float* gains, int n_layers, int batch, int curve_l
   return check_launch();
 }
 
+xkv_status head_curves(const xkv_dims* d, const float* scores, const float* sorted, const int32_t* cu_seqlens,
+                       int64_t total_tokens, int max_seqlen, float* out, int curve_len, cudaStream_t st) {
+  head_curves_kernel<<<d->batch * d->n_kv_heads, 1024, 0, st>>>(scores, sorted, cu_seqlens, total_tokens, max_seqlen,
+                                                                d->window, d->batch, d->n_kv_heads, curve_len, out);
+  count_launch();
+  return check_launch();
+}
+
 size_t select_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens) {
   (void)total_tokens;
   SelectLayout L;
@@ -346,8 +392,11 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
   if (workspace_bytes < L.total) return XKV_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
 
+  const int head_level = per_sequence == XKV_BUDGET_PER_HEAD ? 1 : 0;
+  const int n_budgets = head_level ? d->batch * d->n_kv_heads : (per_sequence ? d->batch : 1);
+  const int n_caches = head_level ? d->batch * d->n_kv_heads : d->batch;       // caches of one layer
   int max_budget = 0;
-  for (int i = 0; i < (per_sequence ? d->batch : 1); ++i) max_budget = budget[i] > max_budget ? budget[i] : max_budget;
+  for (int i = 0; i < n_budgets; ++i) max_budget = budget[i] > max_budget ? budget[i] : max_budget;
   const int64_t max_keep64 = (int64_t)max_budget + d->window;
   const int max_keep = (int)(max_keep64 < max_seqlen ? max_keep64 : max_seqlen);
   if (sel != nullptr && sel_stride < max_keep) return XKV_ERR_INVALID_ARG;
@@ -360,8 +409,9 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
   p.budget = budget[0];
   p.sel = sel != nullptr ? sel : reinterpret_cast<int32_t*>(ws + L.sel);
   p.sel_stride = sel != nullptr ? sel_stride : L.sel_stride;
-  p.seq_lens_layer = c->seq_lens + (size_t)layer * d->batch;
-  p.block_table_layer = c->block_table + (size_t)layer * d->batch * c->max_pages_per_seq;
+  p.head_level = head_level;
+  p.seq_lens_layer = c->seq_lens + (size_t)layer * n_caches;
+  p.block_table_layer = c->block_table + (size_t)layer * n_caches * c->max_pages_per_seq;
   p.k = static_cast<const __nv_bfloat16*>(k);
   p.v = static_cast<const __nv_bfloat16*>(v);
   p.k_pages = static_cast<__nv_bfloat16*>(c->k_pages);
@@ -383,7 +433,7 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
 
   if (cudaMemsetAsync(ws + 4, 0, kHeaderBytes - 4, st) != cudaSuccess) return XKV_ERR_CUDA;   // the status word stays
   if (per_sequence) {
-    if (cudaMemcpyAsync(ws + L.budget, budget, (size_t)d->batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    if (cudaMemcpyAsync(ws + L.budget, budget, (size_t)n_budgets * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return XKV_ERR_CUDA;
     p.budget_dev = reinterpret_cast<const int32_t*>(ws + L.budget);
   }

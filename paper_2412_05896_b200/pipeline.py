@@ -22,8 +22,13 @@ class XkvSession:
                  pool_kernel: int, lengths: list[int], pool_mode: int = xkv.POOL_MAX, page_size: int = 16,
                  max_new_tokens: int = 0, max_budget: int | None = None, total_budget: int | None = None,
                  curve_len: int | None = None, device="cuda:0", scale: float = 0.0,
-                 decode_chunk_rows: int = 0, n_lanes: int = 3):
+                 decode_chunk_rows: int = 0, n_lanes: int = 3, head_level: bool = False):
+        """head_level: budgets, cache lengths and page lists per (layer, sequence, KV head) instead of per (layer,
+        sequence); total_budget and the solver's total then count prefix tokens over all heads of all layers, and
+        max_budget bounds one head."""
         self.L, self.Hq, self.Hkv, self.d, self.W = n_layers, n_q_heads, n_kv_heads, head_dim, window
+        self.head_level = bool(head_level)
+        self.G = n_q_heads // n_kv_heads
         self.B = len(lengths)
         self.lengths = list(lengths)
         self.device = torch.device(device)
@@ -43,15 +48,23 @@ class XkvSession:
 
         # per-layer scores, their sort and the curves (kept for all layers: the solver needs every curve
         # before the first layer can be compacted)
-        self.curve_len = max(1, min(curve_len or self.max_prefix, max(self.max_prefix, 1)))
+        # (a multiple of four ranks, so that every layer's slice of the stacked arrays starts on a 16-byte boundary;
+        # ranks beyond the longest prefix read zero)
+        self.curve_len = (max(1, min(curve_len or self.max_prefix, max(self.max_prefix, 1))) + 3) // 4 * 4
         f32 = dict(dtype=torch.float32, device=self.device)
-        self.scores = torch.empty(n_layers, n_kv_heads, self.T, **f32)
-        self.sorted = torch.empty(n_layers, n_kv_heads, self.T, **f32)
+        self._layer_stride = (n_kv_heads * self.T + 3) // 4 * 4           # floats between the layers' score arrays
+        self.scores = torch.empty(n_layers, self._layer_stride, **f32)[:, : n_kv_heads * self.T].view(
+            n_layers, n_kv_heads, self.T)
+        self.sorted = torch.empty(n_layers, self._layer_stride, **f32)[:, : n_kv_heads * self.T].view(
+            n_layers, n_kv_heads, self.T)
         self.gains = torch.empty(n_layers, self.B, self.curve_len, **f32)
         # what crosses to the host for the solver: one curve per layer (the batch mean, formed on the device);
         # the per-sequence curves cross only when every sequence gets its own list
-        self.layer_gains = torch.empty(n_layers, self.curve_len, **f32)
-        self.layer_gains_host = torch.empty(n_layers, self.curve_len, dtype=torch.float32, pin_memory=True)
+        # units of the solver: layers, or (layer, KV head) pairs with head-level budgets
+        self.n_solver_units = n_layers * (n_kv_heads if self.head_level else 1)
+        self.head_gains = torch.empty(n_layers, n_kv_heads, self.B, self.curve_len, **f32) if self.head_level else None
+        self.layer_gains = torch.empty(self.n_solver_units, self.curve_len, **f32)
+        self.layer_gains_host = torch.empty(self.n_solver_units, self.curve_len, dtype=torch.float32, pin_memory=True)
         self.gains_host = None
         # Layers are independent in the scoring and in the eviction phase, so consecutive layers go to
         # n_lanes side streams, each with its own workspace: the short latency-bound kernels of one layer
@@ -69,28 +82,37 @@ class XkvSession:
         per_layer_cap = min(max_budget if max_budget else self.max_prefix, self.max_prefix)
         self.max_cache_len = per_layer_cap + window + max_new_tokens
         self.max_pages_per_seq = max(1, math.ceil(self.max_cache_len / page_size))
+        n_units = self.n_solver_units
         if total_budget is None:
-            total_budget = n_layers * per_layer_cap
-        total_budget = min(total_budget, n_layers * per_layer_cap)
+            total_budget = n_units * per_layer_cap
+        total_budget = min(total_budget, n_units * per_layer_cap)
+        # caches per layer and the KV heads one page holds: B caches of Hkv heads, or B*Hkv caches of one head
+        self.n_caches = self.B * (n_kv_heads if self.head_level else 1)
+        page_heads = 1 if self.head_level else n_kv_heads
         n_pages = 0
         for P, t in zip(self.prefix, lengths):
-            rows = min(total_budget, n_layers * P) + n_layers * (min(window, t) + max_new_tokens + page_size)
+            rows = min(total_budget, n_units * P) + n_units * (min(window, t) + max_new_tokens + page_size)
             n_pages += math.ceil(rows / page_size)
         self.n_pages = max(n_pages, 1)
         bf16 = dict(dtype=torch.bfloat16, device=self.device)
-        self.k_pages = torch.zeros(self.n_pages, n_kv_heads, page_size, head_dim, **bf16)
-        self.v_pages = torch.zeros(self.n_pages, n_kv_heads, page_size, head_dim, **bf16)
-        self.block_table = torch.zeros(n_layers, self.B, self.max_pages_per_seq, dtype=torch.int32,
+        self.k_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, **bf16)
+        self.v_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, **bf16)
+        self.block_table = torch.zeros(n_layers, self.n_caches, self.max_pages_per_seq, dtype=torch.int32,
                                        device=self.device)
-        # page runs of every (layer, sequence): [0] first page, [1] number of pages; expanded on the device
-        self.page_runs_host = [torch.zeros(n_layers, self.B, dtype=torch.int32, pin_memory=True) for _ in range(2)]
-        self.page_runs = [torch.zeros(n_layers, self.B, dtype=torch.int32, device=self.device) for _ in range(2)]
-        self.seq_lens = torch.zeros(n_layers, self.B, dtype=torch.int32, device=self.device)
+        # page runs of every (layer, cache): [0] first page, [1] number of pages; expanded on the device
+        self.page_runs_host = [torch.zeros(n_layers, self.n_caches, dtype=torch.int32, pin_memory=True)
+                               for _ in range(2)]
+        self.page_runs = [torch.zeros(n_layers, self.n_caches, dtype=torch.int32, device=self.device)
+                          for _ in range(2)]
+        self.seq_lens = torch.zeros(n_layers, self.n_caches, dtype=torch.int32, device=self.device)
         self.cache = xkv.Cache(self.k_pages.data_ptr(), self.v_pages.data_ptr(), self.block_table.data_ptr(),
                                self.seq_lens.data_ptr(), n_layers, page_size, self.max_pages_per_seq,
                                self.n_pages)
+        # decode sees the head-level caches as B*Hkv sequences of one KV head with G query heads each
+        self.dec_dims = self.dims if not self.head_level else xkv.Dims(
+            self.n_caches, self.G, 1, head_dim, window, pool_kernel, pool_mode, scale, head_dim, head_dim)
         self.chunk_rows = decode_chunk_rows
-        self.ws_decode = self._ws(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, self.dims, n_layers=n_layers,
+        self.ws_decode = self._ws(xkv.workspace_bytes(xkv.OP_DECODE_ATTN, self.dec_dims, n_layers=n_layers,
                                                       max_cache_len=self.max_pages_per_seq * page_size,
                                                       chunk_rows=decode_chunk_rows))
         self.out = torch.empty(n_layers, self.B, n_q_heads, head_dim, **bf16)
@@ -130,6 +152,9 @@ class XkvSession:
         xkv.score(self.dims, q_win, k, self.cu, self.T, self.max_seqlen, self.scores[layer],
                   self.sorted[layer] if want_curves else None, self.gains[layer] if want_curves else None,
                   mass, self.curve_len, self.ws_score[i], stream=stream)
+        if self.head_level and want_curves:
+            xkv.head_curves(self.dims, self.scores[layer], self.sorted[layer], self.cu, self.T, self.max_seqlen,
+                            self.head_gains[layer], self.curve_len, stream=stream)
 
     def score_layers(self, q_win: list[torch.Tensor], k: list[torch.Tensor]) -> None:
         """score_layer for every layer, with one fork and one join of the side streams for the whole phase (the
@@ -139,7 +164,7 @@ class XkvSession:
         for s in self.lanes:
             s.wait_stream(cur)
         lib, dims, cu = xkv.lib(), ctypes.byref(self.dims), self.cu.data_ptr()
-        esz = self.scores[0].numel() * 4
+        esz = self._layer_stride * 4
         gsz = self.gains[0].numel() * 4
         for l in range(self.L):
             i = l % len(streams)
@@ -150,22 +175,34 @@ class XkvSession:
                                streams[i].cuda_stream)
             if st < 0:
                 raise xkv.XkvError(st, "xkv_score")
+            if self.head_level:
+                xkv.head_curves(self.dims, self.scores[l], self.sorted[l], self.cu, self.T, self.max_seqlen,
+                                self.head_gains[l], self.curve_len, stream=streams[i])
         self._lanes_busy = bool(self.lanes)
         self.join()
 
     def select_layers(self, budgets, k: list[torch.Tensor], v: list[torch.Tensor]) -> None:
-        """select_layer for every layer under one budget per layer, forked and joined once like score_layers."""
+        """select_layer for every layer under one budget per layer ([L]), or per (layer, KV head) ([L, Hkv]) with
+        head-level budgets; forked and joined once like score_layers."""
         cur = torch.cuda.current_stream()
         streams = self.lanes if self.lanes else [cur]
         for s in self.lanes:
             s.wait_stream(cur)
         lib, dims, cu, cache = xkv.lib(), ctypes.byref(self.dims), self.cu.data_ptr(), ctypes.byref(self.cache)
-        esz = self.scores[0].numel() * 4
-        b32 = np.ascontiguousarray(budgets, dtype=np.int32)
+        esz = self._layer_stride * 4
+        if self.head_level:
+            # the same count for every sequence: [L, Hkv] -> [L, B, Hkv]; kept alive until the streams are joined
+            b32 = np.ascontiguousarray(np.broadcast_to(np.asarray(budgets, dtype=np.int32).reshape(self.L, 1, self.Hkv),
+                                                       (self.L, self.B, self.Hkv)))
+            mode, step = xkv.BUDGET_PER_HEAD, 4 * self.B * self.Hkv
+        else:
+            b32 = np.ascontiguousarray(budgets, dtype=np.int32)
+            mode, step = xkv.BUDGET_PER_LAYER, 4
+        self._budget_keepalive = b32
         for l in range(self.L):
             i = l % len(streams)
             ws = self.ws_select[i]
-            st = lib.xkv_select_compact(dims, l, b32.ctypes.data + 4 * l, 0, self.scores.data_ptr() + l * esz,
+            st = lib.xkv_select_compact(dims, l, b32.ctypes.data + step * l, mode, self.scores.data_ptr() + l * esz,
                                         self.sorted.data_ptr() + l * esz, k[l].data_ptr(), v[l].data_ptr(), cu,
                                         self.T, self.max_seqlen, cache, None, 0, ws.data_ptr(), ws.numel(),
                                         streams[i].cuda_stream)
@@ -179,6 +216,8 @@ class XkvSession:
         """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host.  For one list per
         batch the curves are averaged over the sequences on the device first, so L x curve_len numbers cross."""
         self.join()
+        if per_sequence and self.head_level:
+            raise ValueError("per-sequence lists are not combined with head-level budgets in this session")
         if per_sequence:
             if self.gains_host is None:
                 self.gains_host = torch.empty(self.L, self.B, self.curve_len, dtype=torch.float32, pin_memory=True)
@@ -186,16 +225,19 @@ class XkvSession:
             torch.cuda.current_stream().synchronize()
             gains, prefix = self.gains_host.numpy(), np.asarray(self.prefix, dtype=np.int32)
         else:
-            xkv.batch_curves(self.gains, self.L, self.B, self.curve_len, self.B, self.layer_gains)
+            src = self.head_gains if self.head_level else self.gains        # [units, B, curve_len] either way
+            xkv.batch_curves(src, self.n_solver_units, self.B, self.curve_len, self.B, self.layer_gains)
             self.layer_gains_host.copy_(self.layer_gains, non_blocking=True)
             torch.cuda.current_stream().synchronize()
-            gains = self.layer_gains_host.numpy().reshape(self.L, 1, self.curve_len)
+            gains = self.layer_gains_host.numpy().reshape(self.n_solver_units, 1, self.curve_len)
             prefix = np.asarray([self.max_prefix], dtype=np.int32)
         t0 = time.perf_counter()
         budgets, r_avg = xkv.alloc_budgets(gains, prefix, per_sequence=per_sequence,
                                            total=-1 if total is None else total,
                                            r_target=r_target, n_min=n_min, n_max=n_max)
         self.last_solver_ms = 1e3 * (time.perf_counter() - t0)
+        if self.head_level:
+            budgets = budgets.reshape(self.L, self.Hkv)          # one count per (layer, KV head)
         self.budgets, self.r_avg = budgets, r_avg
         return budgets, r_avg
 
@@ -203,22 +245,30 @@ class XkvSession:
         """Hand consecutive pool pages to every (layer, sequence) for its kept rows plus new tokens: the runs are
         computed here (2 x L x B integers), the page table is expanded from them on the device."""
         budgets = np.asarray(budgets)
-        k_lb = budgets.T if budgets.ndim == 2 else np.broadcast_to(budgets[:, None], (self.L, self.B))   # [L, B]
         prefix = np.asarray(self.prefix)[None, :]
         window = np.minimum(self.W, np.asarray(self.lengths))[None, :]
-        rows = np.minimum(k_lb, prefix) + window + self.max_new
+        if self.head_level:                                  # budgets [L, Hkv] -> one cache per (layer, b, g)
+            k_lb = np.broadcast_to(budgets.reshape(self.L, 1, self.Hkv), (self.L, self.B, self.Hkv))
+            rows = (np.minimum(k_lb, prefix[:, :, None]) + window[:, :, None] + self.max_new).reshape(self.L, -1)
+        else:
+            k_lb = budgets.T if budgets.ndim == 2 else np.broadcast_to(budgets[:, None], (self.L, self.B))   # [L, B]
+            rows = np.minimum(k_lb, prefix) + window + self.max_new
         n = np.minimum(-(-rows // self.page_size), self.max_pages_per_seq).astype(np.int64)               # pages
-        start = np.concatenate([[0], np.cumsum(n.ravel())[:-1]]).reshape(self.L, self.B)
+        start = np.concatenate([[0], np.cumsum(n.ravel())[:-1]]).reshape(self.L, self.n_caches)
         if int(start.ravel()[-1] + n.ravel()[-1]) > self.n_pages:
             raise RuntimeError("page pool too small for these budgets")
         for dst, host, src in zip(self.page_runs, self.page_runs_host, (start, n)):
             host.numpy()[:] = src
             dst.copy_(host, non_blocking=True)
-        xkv.build_block_table(self.page_runs[0], self.page_runs[1], self.cache, self.B)
+        xkv.build_block_table(self.page_runs[0], self.page_runs[1], self.cache, self.n_caches)
 
     def select_layer(self, layer: int, budget, k: torch.Tensor, v: torch.Tensor, sel: torch.Tensor | None = None,
                      per_sequence: bool = False) -> None:
+        """budget: one count, [B] with per_sequence, or [Hkv] / [B, Hkv] in a head-level session."""
         stream, i = self._lane(layer, k, v, sel)
+        if self.head_level:
+            budget = np.ascontiguousarray(np.broadcast_to(np.asarray(budget, dtype=np.int32), (self.B, self.Hkv)))
+            per_sequence = xkv.BUDGET_PER_HEAD
         xkv.select_compact(self.dims, layer, budget, per_sequence, self.scores[layer], self.sorted[layer], k, v,
                            self.cu, self.T, self.max_seqlen, self.cache, sel,
                            0 if sel is None else sel.shape[-1], self.ws_select[i], stream=stream)
@@ -242,7 +292,7 @@ class XkvSession:
         self.join()
         out = self.out if out is None else out
         layer_end = self.L if layer_end is None else layer_end
-        xkv.decode_attn(self.dims, self.cache, layer_begin, layer_end, q, k_new, v_new, out,
+        xkv.decode_attn(self.dec_dims, self.cache, layer_begin, layer_end, q, k_new, v_new, out,
                         self.lse if lse is None else lse,
                         self.chunk_rows if chunk_rows is None else chunk_rows, self.ws_decode)
         return out

@@ -19,10 +19,11 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET = -1, -2, -3, -4
 ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = -5, -6, -7
 POOL_MAX, POOL_AVG = 0, 1
 OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
+BUDGET_PER_LAYER, BUDGET_PER_SEQUENCE, BUDGET_PER_HEAD = 0, 1, 2
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("xkv_score", "xkv_batch_curves", "xkv_build_block_table", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
+EXPORTS = ("xkv_score", "xkv_batch_curves", "xkv_head_curves", "xkv_build_block_table", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
            "xkv_workspace_bytes",
            "xkv_read_device_status", "xkv_profile_events", "xkv_test_hooks", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
@@ -65,6 +66,8 @@ def lib() -> ctypes.CDLL:
     L.xkv_score.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, vp, vp, vp, i32, vp, sz, vp]
     L.xkv_batch_curves.restype = i32
     L.xkv_batch_curves.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+    L.xkv_head_curves.restype = i32
+    L.xkv_head_curves.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, i32, vp]
     L.xkv_build_block_table.restype = i32
     L.xkv_build_block_table.argtypes = [vp, vp, ctypes.POINTER(Cache), i32, vp]
     L.xkv_alloc_budgets.restype = i32
@@ -163,6 +166,13 @@ def batch_curves(gains, n_layers: int, batch: int, curve_len: int, divisor: int,
            "xkv_batch_curves")
 
 
+def head_curves(dims: Dims, scores, sorted_scores, cu_seqlens, total_tokens: int, max_seqlen: int, head_gains,
+                curve_len: int, stream=None) -> None:
+    """scores, sorted dev [Hkv, T] of one layer -> head_gains dev [Hkv, B, curve_len]."""
+    _check(lib().xkv_head_curves(ctypes.byref(dims), _ptr(scores), _ptr(sorted_scores), _ptr(cu_seqlens), total_tokens,
+                                 max_seqlen, _ptr(head_gains), curve_len, _stream(stream)), "xkv_head_curves")
+
+
 def build_block_table(first_page, n_pages_lb, cache: Cache, batch: int, stream=None) -> None:
     _check(lib().xkv_build_block_table(_ptr(first_page), _ptr(n_pages_lb), ctypes.byref(cache), batch,
                                        _stream(stream)), "xkv_build_block_table")
@@ -192,7 +202,7 @@ def average_budgets(lists) -> np.ndarray:
     return out
 
 
-def select_compact(dims: Dims, layer: int, budget, per_sequence: bool, scores, sorted_scores, k, v, cu_seqlens,
+def select_compact(dims: Dims, layer: int, budget, per_sequence, scores, sorted_scores, k, v, cu_seqlens,
                    total_tokens: int, max_seqlen: int, cache: Cache, sel, sel_stride: int, workspace,
                    stream=None) -> None:
     budget = np.ascontiguousarray(np.atleast_1d(budget), dtype=np.int32)
