@@ -348,6 +348,51 @@ def decode_attention(q: np.ndarray, K_c: np.ndarray, V_c: np.ndarray,
 
 
 # ----------------------------------------------------------------------------------------------
+# Eq. 1 / Eq. 2 over the whole prompt: the prefill attention whose last ows rows are W_attn of Alg. 2 step 1
+# ----------------------------------------------------------------------------------------------
+def prefill_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray,
+                      scale: float | None = None) -> tuple[np.ndarray, np.ndarray]:
+    """Causal attention of one head over a prompt of t tokens: Z = softmax(Q K^T / sqrt(d_k)) V (Eq. 1 with the
+    weights of Eq. 2), row i seeing keys 0..i.  Q, K, V: [t, d].  Returns (Z [t, d], lse [t]) where lse[i] is the
+    natural log of the sum over the visible keys of exp(scaled logit): the softmax normaliser of row i, which
+    for the last ows rows is the normaliser of the observation-window weights (Alg. 2 step 1)."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    t, d = K.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    Z = attention_weights(Q, K, scale) @ V
+    S = (Q @ K.T) * scale
+    lse = np.empty(t, dtype=np.float64)
+    for i in range(t):
+        row = S[i, : i + 1]
+        m = np.max(row)
+        lse[i] = m + math.log(np.sum(np.exp(row - m)))
+    return Z, lse
+
+
+def column_scores_from_lse(Q_win_group: np.ndarray, K: np.ndarray, lse_rows: np.ndarray, ows: int,
+                           scale: float | None = None) -> np.ndarray:
+    """Select + Merge when the prefill attention has already produced the normalisers of the window rows
+    (Alg. 2 step 1 takes W_attn from the layer's own attention): u[c] = sum over the group's query heads and
+    window rows of exp(scaled logit - lse).  Q_win_group [G, ows, d], K [t, d], lse_rows [G, ows] (rows of
+    positions t-ows .. t-1).  Returns [max(t-ows, 0)]."""
+    K = np.asarray(K, dtype=np.float64)
+    t, d = K.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    P = max(t - ows, 0)
+    u = np.zeros(P, dtype=np.float64)
+    for Qh, lh in zip(np.asarray(Q_win_group, dtype=np.float64), np.asarray(lse_rows, dtype=np.float64)):
+        for r in range(ows):
+            if t - ows + r < 0:
+                continue
+            u += np.exp((K[:P] @ Qh[r]) * scale - lh[r])
+    return u
+
+
+# ----------------------------------------------------------------------------------------------
 # The path end to end on packed batches (same layouts the C ABI uses, numpy arrays)
 # ----------------------------------------------------------------------------------------------
 def score_layer(q_win: np.ndarray, k: np.ndarray, cu_seqlens: np.ndarray, ows: int, ps: int,

@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
         const uint32_t qb = it & 1u;
         ok = ws_wait(&qfull_bar[qb], (it >> 1) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
-        const uint32_t qa = q_base + qb * C::kQBytes;
+        const uint64_t q_desc = umma_desc_k128(q_base + qb * C::kQBytes);   // k-steps only move the start-address field
         for (int ti = 0; ti < sh.n1; ++ti, ++gt) {
           const uint32_t s = gt % C::kStages;
           const uint32_t slot = (it & 1u) * kSlotsPerUnit + (uint32_t)ti;
@@ -238,12 +238,11 @@ __global__ void __launch_bounds__(kWsThreads, 1) score_fused_kernel(const __grid
           if (!ok) break;
           slot_uses ^= 1u << slot;
           tc_fence_after_sync();
-          const uint32_t kt = k_base + s * C::kKTileBytes;
+          const uint64_t k_desc = umma_desc_k128(k_base + s * C::kKTileBytes);
 #pragma unroll
           for (int k = 0; k < C::kSteps; ++k) {
-            const uint32_t ko = (uint32_t)(k % 4) * 32u;
-            const uint64_t kd = umma_desc_k128(kt + (k / 4) * C::kKHalfBytes + ko);
-            const uint64_t qd = umma_desc_k128(qa + (k / 4) * C::kQHalfBytes + ko);
+            const uint64_t kd = k_desc + (uint64_t)(((k / 4) * C::kKHalfBytes + (k % 4) * 32) >> 4);
+            const uint64_t qd = q_desc + (uint64_t)(((k / 4) * C::kQHalfBytes + (k % 4) * 32) >> 4);
             umma_bf16(tmem_base + slot * kRows, kd, qd, umma_idesc(kTcKeyTile, kRows), k > 0 ? 1u : 0u);
           }
           umma_commit(&empty_bar[s]);           // the ring stage is free once these MMAs have read it

@@ -153,27 +153,28 @@ __global__ void __launch_bounds__(kWsThreads) score_tc_kernel(const __grid_const
         const uint32_t qb = it % C::kQBufs;
         ok = ws_wait(&qfull_bar[qb], (it / C::kQBufs) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
-        const uint32_t qa = q_base + qb * C::kQBytes;
+        // One descriptor per operand buffer; a k-step (16 bf16 = 32 bytes inside the swizzled 128-byte row, the
+        // next 64 columns one half-tile further) only moves the start-address field, which is in 16-byte units
+        // and cannot carry out of its 14 bits for addresses inside shared memory.
+        const uint64_t q_desc = umma_desc_k128(q_base + qb * C::kQBytes);
         for (int ti = 0; ti < sh.n_tiles; ++ti, ++gt) {
           const uint32_t s = gt % kWsStages, ab = gt % kAccBufs;
           ok = ws_wait(&full_bar[s], (gt / kWsStages) & 1u, s_abort, p.wait_ns) &&
                ws_wait(&accempty_bar[ab], ((gt / kAccBufs) & 1u) ^ 1u, s_abort, p.wait_ns);
           if (!ok) break;
           tc_fence_after_sync();
-          const uint32_t kt = k_base + s * C::kKTileBytes;
+          const uint64_t k_desc = umma_desc_k128(k_base + s * C::kKTileBytes);
           const uint32_t d_tmem = tmem_base + ab * C::kBufCols;
 #pragma unroll
           for (int k = 0; k < C::kSteps; ++k) {
-            const uint32_t ko = (uint32_t)(k % 4) * 32u;      // 16 bf16 along K inside the swizzled 128-byte row
-            const uint64_t kd = umma_desc_k128(kt + (k / 4) * C::kKHalfBytes + ko);
+            const uint64_t kd = k_desc + (uint64_t)(((k / 4) * C::kKHalfBytes + (k % 4) * 32) >> 4);
+            const uint64_t qd = q_desc + (uint64_t)(((k / 4) * C::kQHalfBytes + (k % 4) * 32) >> 4);
             if (PASS == 1) {
 #pragma unroll
-              for (int rb = 0; rb < (M == 256 ? 2 : 1); ++rb) {
-                const uint64_t qd = umma_desc_k128(qa + (k / 4) * C::kQHalfBytes + rb * 128 * 128 + ko);
-                umma_bf16(d_tmem + rb * 128u, qd, kd, umma_idesc(128, kTcKeyTile), k > 0 ? 1u : 0u);
-              }
+              for (int rb = 0; rb < (M == 256 ? 2 : 1); ++rb)
+                umma_bf16(d_tmem + rb * 128u, qd + (uint64_t)((rb * 128 * 128) >> 4), kd, umma_idesc(128, kTcKeyTile),
+                          k > 0 ? 1u : 0u);
             } else {
-              const uint64_t qd = umma_desc_k128(qa + (k / 4) * C::kQHalfBytes + ko);
               umma_bf16(d_tmem, kd, qd, umma_idesc(kTcKeyTile, M), k > 0 ? 1u : 0u);
             }
           }

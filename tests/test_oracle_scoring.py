@@ -195,3 +195,48 @@ def test_score_layer_packed_batch_matches_per_unit():
     assert curves.shape == (2, 12)
     assert abs(curves[0].sum() - 1.0) < 1e-13 and abs(curves[1].sum() - 1.0) < 1e-13
     assert np.all(curves[0, 6:] == 0.0)
+
+
+# ------------------------------------------------------------------ prefill attention (Eq. 1 / Eq. 2 over the prompt)
+def test_prefill_attention_closed_forms_and_library():
+    rng = np.random.default_rng(40)
+    t, d = 37, 16
+    Q, K, V = rng.standard_normal((t, d)), rng.standard_normal((t, d)), rng.standard_normal((t, d))
+    Z, lse = O.prefill_attention(Q, K, V)
+    # library cross-check: torch fp64 causal scaled-dot-product attention on the CPU
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(Q)[None], torch.from_numpy(K)[None],
+                                                           torch.from_numpy(V)[None], is_causal=True)[0].numpy()
+    assert np.max(np.abs(Z - ref)) < 1e-12
+    # identical keys: uniform weights over the visible keys, so row i is the running mean of V and lse = s + ln(i+1)
+    Kc = np.tile(K[:1], (t, 1))
+    Zc, lc = O.prefill_attention(Q, Kc, V)
+    running = np.cumsum(V, axis=0) / np.arange(1, t + 1)[:, None]
+    assert np.max(np.abs(Zc - running)) < 1e-12
+    s_const = (Q @ K[0]) / math.sqrt(d)
+    assert np.max(np.abs(lc - (s_const + np.log(np.arange(1, t + 1))))) < 1e-12
+    # row 0 sees only itself: z_0 = v_0, lse_0 = its one logit
+    assert np.max(np.abs(Z[0] - V[0])) < 1e-15 and abs(lse[0] - (Q[0] @ K[0]) / math.sqrt(d)) < 1e-13
+    # the last rows of each decode step: attending with q_i over keys 0..i is decode_attention on that prefix
+    for i in (0, 5, t - 1):
+        z, l = O.decode_attention(Q[i], K[: i + 1], V[: i + 1])
+        assert np.max(np.abs(z - Z[i])) < 1e-13 and abs(l - lse[i]) < 1e-12
+
+
+def test_window_scores_from_the_prefill_normalisers_equal_the_definition():
+    rng = np.random.default_rng(41)
+    t, d, ows, G = 53, 8, 6, 2
+    K = rng.standard_normal((t, d))
+    Qfull = rng.standard_normal((G, t, d)) * 2.0
+    lse = np.stack([O.prefill_attention(Qfull[h], K, K)[1] for h in range(G)])            # [G, t]
+    Qwin = Qfull[:, t - ows:]
+    u_def = O.column_scores(Qwin, K, ows)
+    u_lse = O.column_scores_from_lse(Qwin, K, lse[:, t - ows:], ows)
+    assert np.max(np.abs(u_def - u_lse)) < 1e-13
+    # exp(logit - lse) of a window row is that row of W_attn (Eq. 2): compare with the full matrix
+    Wfull = O.attention_weights(Qfull[1], K)
+    r = 3
+    row = np.exp((K[: t - ows] @ Qwin[1, r]) / math.sqrt(d) - lse[1, t - ows + r])
+    assert np.max(np.abs(row - Wfull[t - ows + r, : t - ows])) < 1e-14
+    # a wrong normaliser (shifted by ln 2) halves the scores: the function really uses what it is given
+    u_half = O.column_scores_from_lse(Qwin, K, lse[:, t - ows:] + math.log(2.0), ows)
+    assert np.max(np.abs(u_half - 0.5 * u_def)) < 1e-13
