@@ -3,9 +3,13 @@
  * KV-cache budgets) on one NVIDIA B200 (sm_100a).
  *
  * The path, in call order:
+ *   0. xkv_prefill_attn   optional, the step before the path: causal attention of the whole prompt, which also
+ *                         yields the softmax normalisers of the window rows   (Eq. 1, Eq. 2; Alg. 2 step 1)
  *   1. xkv_score          per layer: observation-window attention weights -> pooled importance
  *                         scores per KV head, their descending sort, and the layer's
  *                         retained-importance curve               (Eq. 2, Eq. 3, Eq. 4; Alg. 2 steps 1-4)
+ *      xkv_score_lse      the same from normalisers that xkv_prefill_attn (or the model's own attention)
+ *                         already produced: one pass over the keys instead of two      (Alg. 2 steps 1-4)
  *      xkv_batch_curves   device: one curve per layer from the batch's curves         (Alg. 1, input W)
  *      xkv_head_curves    device: one curve per (layer, KV head) for head-level budgets      (Sec. II-C)
  *   2. xkv_alloc_budgets  host: greedy split of a global budget across layers        (Alg. 1; Eq. 17, Eq. 18)
@@ -67,6 +71,7 @@ typedef int32_t xkv_status;
 #define XKV_OP_SCORE          0
 #define XKV_OP_SELECT_COMPACT 1
 #define XKV_OP_DECODE_ATTN    2
+#define XKV_OP_PREFILL_ATTN   3
 
 /* Problem shape shared by the device entry points. */
 typedef struct xkv_dims {
@@ -149,6 +154,46 @@ xkv_status xkv_score(const xkv_dims* dims, const void* q_win, const void* k,
                      const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen,
                      float* scores, float* sorted, float* gains, float* mass, int32_t curve_len,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * xkv_prefill_attn -- causal attention of the prompt (Eq. 1 with the weights of Eq. 2), the layer's own attention
+ * in which the paper computes W_attn (Alg. 2 step 1; Sec. IV-A, prefill phase).
+ *
+ * For every sequence b, query head h and position i < t_b:
+ *   out[i,h,:] = softmax over the keys c <= i of scale * q[i,h,:] . k[c,g,:]  times  v[c,g,:]     (g = h / G)
+ *   lse[h][i]  = natural log of the sum over c <= i of exp(scale * q[i,h,:] . k[c,g,:])
+ * bf16 inputs, fp32 accumulation, the weights rounded to bf16 before they multiply v, bf16 output.
+ * The lse entries of the last W positions of a sequence are the normalisers of the observation-window rows
+ * of W_attn; xkv_score_lse takes them instead of recomputing them with a pass over the keys.
+ *
+ * q          dev bf16 [T][Hq][d], packed like k (row cu_seqlens[b] + i)
+ * k, v       dev bf16, layout and strides of xkv_score (dims.kv_stride_*)
+ * out        dev out bf16 [T][Hq][d]
+ * lse        dev out fp32 [Hq][T], may be NULL
+ * workspace  dev, at least xkv_workspace_bytes(XKV_OP_PREFILL_ATTN, ...) bytes (the status word), 256-byte aligned
+ * dims.window, pool_kernel and pool_mode are not used. Device status XKV_ERR_TIMEOUT if a bounded wait expired.
+ */
+xkv_status xkv_prefill_attn(const xkv_dims* dims, const void* q, const void* k, const void* v,
+                            const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen, void* out,
+                            float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * xkv_score_lse -- xkv_score when the normalisers of the window rows are already known (Alg. 2 step 1 takes
+ * W_attn from the layer's attention; only Select, Merge, Pooling and the curves remain: Alg. 2 steps 2-4, Eq. 4).
+ *
+ *   a[h,r,c] = exp(scale * q_win[b,h,r,:] . k[c,g,:] - lse[h][cu_seqlens[b] + t_b - W + r])
+ * and everything after it as in xkv_score; the keys are read once. With the "nothing cached" mini-prefill of
+ * Sec. IV-A the caller has no normalisers and uses xkv_score, which forms them from the window queries alone.
+ *
+ * lse        dev fp32 [Hq][T] as xkv_prefill_attn writes it (only the last min(W, t_b) positions of every
+ *            sequence are read)
+ * other arguments, outputs and workspace: those of xkv_score.
+ * Returns XKV_ERR_UNSUPPORTED unless G*W is 32, 64, 128 or 256.
+ */
+xkv_status xkv_score_lse(const xkv_dims* dims, const void* q_win, const void* k, const int32_t* cu_seqlens,
+                         int64_t total_tokens, int32_t max_seqlen, const float* lse, float* scores, float* sorted,
+                         float* gains, float* mass, int32_t curve_len, void* workspace, size_t workspace_bytes,
+                         void* stream);
 
 /*
  * xkv_alloc_budgets -- Algorithm 1 (adaptive allocation), host only, no CUDA call.
@@ -336,6 +381,7 @@ xkv_status xkv_decode_attn_static(const xkv_dims* dims, const xkv_cache* cache, 
 /*
  * Workspace size in bytes for one call of `op` (XKV_OP_*). Unused arguments may be 0.
  *   XKV_OP_SCORE, XKV_OP_SELECT_COMPACT: dims, max_seqlen, total_tokens
+ *   XKV_OP_PREFILL_ATTN: dims
  *   XKV_OP_DECODE_ATTN: dims, n_layers (layers per call), max_cache_len (upper bound of any
  *                       seq_lens entry, e.g. max_pages_per_seq*page_size), chunk_rows as passed
  * Returns 0 for invalid arguments.

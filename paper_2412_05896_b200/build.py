@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libxkv.so")
-SOURCES = ["xkv_api.cu", "xkv_score.cu", "xkv_score_tc.cu", "xkv_score_fused.cu", "xkv_select.cu", "xkv_decode.cu"]
+SOURCES = ["xkv_api.cu", "xkv_score.cu", "xkv_score_tc.cu", "xkv_score_fused.cu", "xkv_select.cu", "xkv_decode.cu", "xkv_prefill.cu"]
 HEADERS = ["common.cuh", "ops.h", "score_params.h", "tc_common.cuh", os.path.join("..", "..", "include", "xkv.h")]
 
 

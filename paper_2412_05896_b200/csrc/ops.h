@@ -10,7 +10,15 @@ namespace xkv {
 size_t score_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens);
 xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int32_t* cu_seqlens,
                  int64_t total_tokens, int max_seqlen, float* scores, float* sorted, float* gains, float* mass,
-                 int curve_len, void* workspace, size_t workspace_bytes, cudaStream_t st);
+                 int curve_len, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                 const float* lse = nullptr);
+// 1 when the shape is one the scoring pass from given row normalisers covers
+int score_lse_supported(const xkv_dims* d, int max_seqlen);
+
+size_t prefill_workspace_bytes();
+xkv_status prefill_attn(const xkv_dims* d, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                        int64_t total_tokens, int max_seqlen, void* out, float* lse, void* workspace,
+                        cudaStream_t st);
 
 size_t select_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens);
 xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, int per_sequence,

@@ -34,6 +34,8 @@ struct ScoreParams {
 // tcgen05 variant of the two logit passes (xkv_score_tc.cu).  Returns XKV_ERR_UNSUPPORTED when the shape
 // is outside what it covers; the caller then uses the mma.sync kernels.
 xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st);
+// The column-sum pass alone, for row normalisers that are already in p.mrow (same shapes as score_tc_passes).
+xkv_status score_tc_pass2(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st);
 // Key split the tcgen05 variant uses (0 if it does not cover the shape).
 int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen);
 

@@ -104,6 +104,49 @@ xkv_status xkv_score(const xkv_dims* dims, const void* q_win, const void* k, con
                workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
+xkv_status xkv_score_lse(const xkv_dims* dims, const void* q_win, const void* k, const int32_t* cu_seqlens,
+                         int64_t total_tokens, int32_t max_seqlen, const float* lse, float* scores, float* sorted,
+                         float* gains, float* mass, int32_t curve_len, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+  xkv_status s = check_prefill_dims(dims);
+  if (s != XKV_OK) return s;
+  if (q_win == nullptr || k == nullptr || cu_seqlens == nullptr || scores == nullptr || workspace == nullptr ||
+      lse == nullptr)
+    return XKV_ERR_INVALID_ARG;
+  if (sorted != nullptr && (gains == nullptr || curve_len < 1)) return XKV_ERR_INVALID_ARG;
+  if (!aligned16(q_win) || !aligned16(k) || !aligned16(cu_seqlens) || !aligned16(scores) || !aligned16(sorted) ||
+      !aligned16(gains) || !aligned16(mass) || !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return XKV_ERR_INVALID_ARG;
+  if (total_tokens <= 0 || total_tokens >= (1ll << 31) || max_seqlen <= 0 || max_seqlen > total_tokens)
+    return XKV_ERR_INVALID_ARG;
+  if (!score_lse_supported(dims, max_seqlen)) return XKV_ERR_UNSUPPORTED;
+  const size_t need = score_workspace_bytes(dims, max_seqlen, total_tokens);
+  if (need == 0) return XKV_ERR_INVALID_ARG;
+  if (workspace_bytes < need) return XKV_ERR_WORKSPACE;
+  return score(dims, q_win, k, cu_seqlens, total_tokens, max_seqlen, scores, sorted, gains, mass, curve_len,
+               workspace, workspace_bytes, static_cast<cudaStream_t>(stream), lse);
+}
+
+xkv_status xkv_prefill_attn(const xkv_dims* dims, const void* q, const void* k, const void* v,
+                            const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen, void* out,
+                            float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  xkv_status s = check_dims(dims);
+  if (s != XKV_OK) return s;
+  if (q == nullptr || k == nullptr || v == nullptr || cu_seqlens == nullptr || out == nullptr || workspace == nullptr)
+    return XKV_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(cu_seqlens) || !aligned16(out) ||
+      !aligned16(lse) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0)
+    return XKV_ERR_INVALID_ARG;
+  if (dims->kv_stride_head < dims->head_dim || dims->kv_stride_head % 8 != 0 ||
+      dims->kv_stride_token < (int64_t)dims->n_kv_heads * dims->head_dim || dims->kv_stride_token % 8 != 0)
+    return XKV_ERR_INVALID_ARG;
+  if (total_tokens <= 0 || total_tokens >= (1ll << 31) || max_seqlen <= 0 || max_seqlen > total_tokens)
+    return XKV_ERR_INVALID_ARG;
+  if (workspace_bytes < prefill_workspace_bytes()) return XKV_ERR_WORKSPACE;
+  return prefill_attn(dims, q, k, v, cu_seqlens, total_tokens, max_seqlen, out, lse, workspace,
+                      static_cast<cudaStream_t>(stream));
+}
+
 xkv_status xkv_select_compact(const xkv_dims* dims, int32_t layer, const int32_t* budget, int32_t per_sequence,
                               const float* scores, const float* sorted, const void* k, const void* v,
                               const int32_t* cu_seqlens, int64_t total_tokens, int32_t max_seqlen,
@@ -222,6 +265,9 @@ size_t xkv_workspace_bytes(int32_t op, const xkv_dims* dims, int32_t max_seqlen,
     case XKV_OP_SELECT_COMPACT:
       if (check_prefill_dims(dims) != XKV_OK || max_seqlen <= 0 || total_tokens <= 0) return 0;
       return select_workspace_bytes(dims, max_seqlen, total_tokens);
+    case XKV_OP_PREFILL_ATTN:
+      if (check_dims(dims) != XKV_OK) return 0;
+      return prefill_workspace_bytes();
     case XKV_OP_DECODE_ATTN:
       if (check_dims(dims) != XKV_OK || n_layers <= 0 || max_cache_len < 0 || chunk_rows < 0 ||
           chunk_rows % 64 != 0)

@@ -1,0 +1,461 @@
+// xkv_prefill_attn: causal attention of the whole prompt (Eq. 1 with the weights of Eq. 2) on the 5th-generation
+// tensor cores, writing next to its output the softmax normaliser of every row.  The normalisers of the last W
+// rows are what the scoring step needs of W_attn (Alg. 2 step 1): with them xkv_score_lse forms the column
+// scores in one pass over the keys.
+//
+// One CTA per (sequence, tile of 128 query rows, query head), 224 threads:
+//   warps 0-3  softmax: thread = query row = TMEM lane.  Per key tile: row maximum out of TMEM, a reference
+//              maximum that is exact on the first tile and raised lazily afterwards (only when a logit exceeds
+//              it by 2^8, which is when the O accumulator in TMEM is rescaled: load, multiply, store),
+//              P = exp2(s*c - ref) rounded to bf16 into shared memory in the K-major 128-byte-swizzled layout
+//              the MMA reads as its A operand, row sum in fp32.  At the end O / l -> bf16 rows, lse.
+//   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles, and of the V tiles (two stages
+//              each, 128 keys a tile), so that a K tile never queues behind the V stage of an earlier tile
+//   warp 5     MMA issuer (one lane): S = Q K^T into one of two 128-column TMEM buffers, one tile ahead of the
+//              softmax; O += P V with V as an MN-major B operand straight from its [keys][d] tile
+// Every wait is bounded; an expired wait sets the status word and lets the CTA drain.
+#include <atomic>
+
+#include "tc_common.cuh"
+#include "ops.h"
+
+namespace xkv {
+namespace {
+
+using namespace tc;
+
+constexpr int kPfThreads = 224;
+constexpr int kPfRows = 128;          // query rows per CTA
+constexpr int kPfKeys = 128;          // keys per tile
+constexpr float kPfLazy = 8.f;        // log2 slack before the reference maximum is raised
+
+struct PrefillParams {
+  const int32_t* cu_seqlens;
+  __nv_bfloat16* out;     // [T][Hq][D]
+  float* lse;             // [Hq][T]
+  WorkspaceHeader* hdr;
+  int64_t total_tokens;
+  int32_t batch, n_q_heads, n_kv_heads, group, max_seqlen;
+  float scale_log2;
+  uint64_t wait_ns;
+};
+
+template <int D>
+struct PfCfg {
+  static constexpr int kHalves = D / 64;
+  static constexpr int kSteps = D / 16;                      // k-steps of S = Q K^T
+  static constexpr int kHalfBytes = 128 * 128;               // 128 rows of 128 bytes
+  static constexpr int kTileBytes = kHalves * kHalfBytes;    // Q, K or V tile
+  static constexpr int kPBytes = 2 * kHalfBytes;             // P: 128 rows x 128 keys bf16
+  static constexpr int kStages = 2;
+  static constexpr uint32_t kSCols = 128;                    // one S buffer
+  static constexpr uint32_t kOCol = 256;                     // O accumulator starts here
+  static constexpr uint32_t kTmemCols = 512;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kTileBytes * (1 + 2 * kStages) + kPBytes + 256;
+};
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+        "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+        "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])),
+        "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])),
+        "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
+        "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory descriptor of an MN-major operand tile stored as rows of 128 bytes (64 bf16 along MN) per K index
+// with the 128-byte swizzle: eight K rows form a 1024-byte group (stride byte offset), the next 64 MN elements
+// start `mn_block_bytes` further (leading byte offset).  This is what a TMA box {64, rows} of a [keys][d] tile is
+// when d is the MMA's N and the keys its K.
+__device__ __forceinline__ uint64_t umma_desc_mn128(uint32_t smem_addr, uint32_t mn_block_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)(mn_block_bytes >> 4) << 16;     // leading byte offset: next block of 64 MN elements
+  d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset: next group of eight K rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;                         // SWIZZLE_128B
+  return d;
+}
+
+// bf16 x bf16 -> fp32, A K-major, B MN-major.
+__host__ __device__ constexpr uint32_t umma_idesc_b_mn(int M, int N) { return umma_idesc(M, N) | (1u << 16); }
+
+// The (sequence, query tile) of CTA-tile index `idx`, counted from the end so that the long tiles of the last
+// sequence start first; false when idx is beyond the tiles that exist.  Computed by every warp for itself: a lane
+// takes one sequence, a warp scan gives the tiles before it.
+__device__ __forceinline__ bool pf_tile(const PrefillParams& p, int idx, int* b_out, int* q0_out, int* cu_out,
+                                        int* t_out) {
+  const int lane = threadIdx.x & 31;
+  int before = 0;                                   // tiles of the sequences already passed
+  for (int base = 0; base < p.batch; base += 32) {
+    const int b = p.batch - 1 - (base + lane);
+    int cu = 0, t = 0, n = 0;
+    if (b >= 0) {
+      cu = p.cu_seqlens[b];
+      t = min(p.cu_seqlens[b + 1] - cu, p.max_seqlen);
+      n = (t + kPfRows - 1) / kPfRows;
+    }
+    int incl = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    const unsigned hit = __ballot_sync(0xffffffffu, idx < before + incl);
+    if (hit != 0u) {
+      const int src = __ffs(hit) - 1;
+      const int first = before + __shfl_sync(0xffffffffu, incl - n, src);     // tiles before that sequence
+      const int n_src = __shfl_sync(0xffffffffu, n, src);
+      *b_out = p.batch - 1 - (base + src);
+      *q0_out = (n_src - 1 - (idx - first)) * kPfRows;
+      *cu_out = __shfl_sync(0xffffffffu, cu, src);
+      *t_out = __shfl_sync(0xffffffffu, t, src);
+      return true;
+    }
+    before += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  return false;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kPfThreads, 1)
+prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
+  using C = PfCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_s = smem;
+  uint8_t* k_s = q_s + C::kTileBytes;
+  uint8_t* v_s = k_s + (size_t)C::kStages * C::kTileBytes;
+  uint8_t* p_s = v_s + (size_t)C::kStages * C::kTileBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + C::kPBytes);
+  uint64_t* q_full = bars;             // [1]
+  uint64_t* k_full = bars + 1;         // [2]
+  uint64_t* k_empty = bars + 3;        // [2]
+  uint64_t* v_full = bars + 5;         // [2]
+  uint64_t* v_empty = bars + 7;        // [2]
+  uint64_t* s_full = bars + 9;         // [2] S buffer complete (MMA -> softmax)
+  uint64_t* s_empty = bars + 11;       // [2] S buffer read (softmax -> MMA)
+  uint64_t* p_full = bars + 13;        // [1] P written, O rescaled (softmax -> MMA)
+  uint64_t* p_empty = bars + 14;       // [1] O += P V complete (MMA -> softmax)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 15);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int b, q0, cu, t;
+  const int h = blockIdx.x % p.n_q_heads;
+  if (!pf_tile(p, blockIdx.x / p.n_q_heads, &b, &q0, &cu, &t)) return;      // uniform over the CTA
+  const int g = h / p.group;
+  const int n_kt = q0 / kPfKeys + 1;                 // key tiles up to and including the diagonal one
+
+  if (tid == 0) {
+    mbar_init(q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&k_full[i], 1);
+      mbar_init(&k_empty[i], 1);
+      mbar_init(&v_full[i], 1);
+      mbar_init(&v_empty[i], 1);
+      mbar_init(&s_full[i], 1);
+      mbar_init(&s_empty[i], 4);
+    }
+    mbar_init(p_full, 4);
+    mbar_init(p_empty, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmap_q);
+    prefetch_tmap(&tmap_k);
+    prefetch_tmap(&tmap_v);
+  }
+  if (warp == 0) {
+    tmem_alloc(s_tmem, C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ producer of Q and the K tiles
+    if (lane == 0) {
+      mbar_arrive_expect_tx(q_full, (uint32_t)C::kTileBytes);
+#pragma unroll
+      for (int hf = 0; hf < C::kHalves; ++hf) tma_load_3d(q_s + hf * C::kHalfBytes, &tmap_q, hf * 64, h, cu + q0, q_full);
+      bool ok = true;
+      for (int j = 0; ok && j < n_kt; ++j) {
+        const uint32_t s = j & 1u, ph = ((j >> 1) & 1u) ^ 1u;
+        ok = ws_wait(&k_empty[s], ph, s_abort, p.wait_ns);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&k_full[s], (uint32_t)C::kTileBytes);
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf)
+          tma_load_3d(k_s + (size_t)s * C::kTileBytes + hf * C::kHalfBytes, &tmap_k, hf * 64, g, cu + j * kPfKeys,
+                      &k_full[s]);
+      }
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ producer of the V tiles
+    if (lane == 0) {
+      bool ok = true;
+      for (int j = 0; ok && j < n_kt; ++j) {
+        const uint32_t s = j & 1u, ph = ((j >> 1) & 1u) ^ 1u;
+        ok = ws_wait(&v_empty[s], ph, s_abort, p.wait_ns);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&v_full[s], (uint32_t)C::kTileBytes);
+#pragma unroll
+        for (int hf = 0; hf < C::kHalves; ++hf)
+          tma_load_3d(v_s + (size_t)s * C::kTileBytes + hf * C::kHalfBytes, &tmap_v, hf * 64, g, cu + j * kPfKeys,
+                      &v_full[s]);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = ws_wait(q_full, 0u, s_abort, p.wait_ns);
+      const uint64_t q_desc = umma_desc_k128(smem_u32(q_s));
+      const uint64_t p_desc = umma_desc_k128(smem_u32(p_s));
+      auto issue_qk = [&](int j) -> bool {
+        const uint32_t s = j & 1u;
+        if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
+        if (!ws_wait(&s_empty[s], ((j >> 1) & 1u) ^ 1u, s_abort, p.wait_ns)) return false;
+        tc_fence_after_sync();
+        const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kTileBytes);
+#pragma unroll
+        for (int k = 0; k < C::kSteps; ++k) {
+          const uint64_t off = (uint64_t)(((k / 4) * C::kHalfBytes + (k % 4) * 32) >> 4);
+          umma_bf16(tmem_base + s * C::kSCols, q_desc + off, k_desc + off, umma_idesc(kPfRows, kPfKeys),
+                    k > 0 ? 1u : 0u);
+        }
+        umma_commit(&k_empty[s]);
+        umma_commit(&s_full[s]);
+        return true;
+      };
+      if (ok) ok = issue_qk(0);
+      for (int j = 0; ok && j < n_kt; ++j) {
+        if (j + 1 < n_kt) {
+          ok = issue_qk(j + 1);           // the next tile's logits run under this tile's softmax
+          if (!ok) break;
+        }
+        const uint32_t s = j & 1u;
+        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(&v_full[s], (j >> 1) & 1u, s_abort, p.wait_ns);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t v_base = smem_u32(v_s) + s * C::kTileBytes;
+#pragma unroll
+        for (int k = 0; k < kPfKeys / 16; ++k) {
+          // A: P[rows][keys 16k .. 16k+15], K-major; B: V[keys 16k ..][d], MN-major (16 keys = two 8-row groups)
+          const uint64_t pd = p_desc + (uint64_t)(((k / 4) * C::kHalfBytes + (k % 4) * 32) >> 4);
+          const uint64_t vd = umma_desc_mn128(v_base + k * 16 * 128, C::kHalfBytes);
+          umma_bf16(tmem_base + C::kOCol, pd, vd, umma_idesc_b_mn(kPfRows, D), (j > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(&v_empty[s]);
+        umma_commit(p_empty);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps 0..3
+    const int r = tid;                                       // query row of the tile = TMEM lane
+    const uint32_t lane_base = tmem_base + ((uint32_t)(32 * warp) << 16);
+    const int row_pos = q0 + r;                              // position in the sequence
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; ok && j < n_kt; ++j) {
+      const uint32_t s = j & 1u;
+      ok = __all_sync(0xffffffffu, ws_wait(&s_full[s], (j >> 1) & 1u, s_abort, p.wait_ns));
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t s_addr = lane_base + s * C::kSCols;
+      const bool diag = j == n_kt - 1;                       // the only tile with keys beyond some row's position
+      const int c_base = j * kPfKeys;
+      // ---- row maximum of the tile
+      float mx = -INFINITY;
+#pragma unroll
+      for (int cc = 0; cc < kPfKeys; cc += 64) {
+        float va[32], vb[32];
+        tmem_ld32(s_addr + (uint32_t)cc, va);
+        tmem_ld32(s_addr + (uint32_t)(cc + 32), vb);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float a = (diag && c_base + cc + i > row_pos) ? -INFINITY : va[i];
+          const float bb = (diag && c_base + cc + 32 + i > row_pos) ? -INFINITY : vb[i];
+          mx = fmaxf(mx, fmaxf(a, bb));
+        }
+      }
+      mx *= p.scale_log2;                                    // key 0 is always visible, so mx is finite
+      const bool grow = mx > m_ref + kPfLazy;                // also true on the first tile (m_ref = -inf)
+      float alpha = 1.f;
+      if (grow) {
+        alpha = j == 0 ? 0.f : fast_exp2(m_ref - mx);
+        m_ref = mx;
+        l *= alpha;
+      }
+      // ---- the previous tile's O += P V must be complete before P is overwritten or O rescaled
+      if (j > 0) {
+        ok = __all_sync(0xffffffffu, ws_wait(p_empty, (j - 1) & 1u, s_abort, p.wait_ns));
+        if (!ok) break;
+        tc_fence_after_sync();
+        if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+          for (int cc = 0; cc < D; cc += 32) {
+            float o[32];
+            tmem_ld32(lane_base + C::kOCol + (uint32_t)cc, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+            tmem_st32(lane_base + C::kOCol + (uint32_t)cc, o);
+          }
+          tmem_wait_st();
+        }
+      }
+      // ---- P = exp2(s*c - ref) as bf16 into shared memory, row sum in fp32
+      float sum = 0.f;
+#pragma unroll
+      for (int cc = 0; cc < kPfKeys; cc += 32) {
+        float v[32];
+        tmem_ld32(s_addr + (uint32_t)cc, v);
+        tmem_wait_ld();
+        uint32_t packed[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          float e0 = fast_exp2(fmaf(v[i], p.scale_log2, -m_ref));
+          float e1 = fast_exp2(fmaf(v[i + 1], p.scale_log2, -m_ref));
+          if (diag) {
+            if (c_base + cc + i > row_pos) e0 = 0.f;
+            if (c_base + cc + i + 1 > row_pos) e1 = 0.f;
+          }
+          sum += e0 + e1;
+          packed[i >> 1] = pack_bf16(e0, e1);
+        }
+        // 32 keys = four 16-byte pieces of the row's 128-byte line in half cc/64; piece index XOR (row & 7)
+        uint8_t* line = p_s + (cc >> 6) * C::kHalfBytes + r * 128;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int piece = ((cc & 63) >> 3) + q;
+          *reinterpret_cast<uint4*>(line + ((piece ^ (r & 7)) << 4)) =
+              make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+        }
+      }
+      l += sum;
+      // the S buffer has been read for the last time; P and O are ready for the MMA
+      tc_fence_before_sync();
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&s_empty[s]);
+        mbar_arrive(p_full);
+      }
+    }
+    // ---- epilogue: O / l -> bf16, lse
+    if (ok) ok = __all_sync(0xffffffffu, ws_wait(p_empty, (n_kt - 1) & 1u, s_abort, p.wait_ns));
+    if (ok) {
+      tc_fence_after_sync();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      const bool live = row_pos < t;
+      __nv_bfloat16* orow = p.out + ((size_t)(cu + row_pos) * p.n_q_heads + h) * D;
+#pragma unroll
+      for (int cc = 0; cc < D; cc += 32) {
+        float o[32];
+        tmem_ld32(lane_base + C::kOCol + (uint32_t)cc, o);
+        tmem_wait_ld();
+        if (live) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 w;
+            w.x = pack_bf16(o[8 * q + 0] * inv, o[8 * q + 1] * inv);
+            w.y = pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv);
+            w.z = pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv);
+            w.w = pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv);
+            *reinterpret_cast<uint4*>(orow + cc + 8 * q) = w;
+          }
+        }
+      }
+      if (live && p.lse != nullptr)
+        p.lse[(size_t)h * p.total_tokens + cu + row_pos] = (m_ref + log2f(l)) * 0.6931471805599453f;
+    }
+  }
+
+  // ---- teardown
+  __syncthreads();
+  if (*s_abort) {
+    if (tid == 0) record_status(p.hdr, XKV_ERR_TIMEOUT);
+    for (int i = 0; i < 1000; ++i) __nanosleep(1000);   // let copies and MMAs already issued finish
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, C::kTmemCols);
+}
+
+template <int D>
+xkv_status pf_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const PrefillParams& p,
+                     int grid, cudaStream_t st) {
+  static std::atomic<bool> done[64];   // idempotent set-up: two threads doing it twice is harmless
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
+  if (!done[dev].load(std::memory_order_acquire)) {
+    if (cudaFuncSetAttribute(prefill_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)PfCfg<D>::kSmemBytes) != cudaSuccess)
+      return XKV_ERR_CUDA;
+    done[dev].store(true, std::memory_order_release);
+  }
+  prefill_attn_kernel<D><<<grid, kPfThreads, PfCfg<D>::kSmemBytes, st>>>(tq, tk, tv, p);
+  count_launch();
+  return check_launch();
+}
+
+// 3-D map {d, heads, tokens} with box {64, 1, 128} over a packed [T][heads][d] bf16 tensor.
+bool pf_make_tmap(CUtensorMap* tmap, const void* base, int head_dim, int heads, int64_t tokens, int64_t stride_token,
+                  int64_t stride_head) {
+  const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)heads, (cuuint64_t)tokens};
+  const cuuint64_t strides[2] = {(cuuint64_t)stride_head * 2, (cuuint64_t)stride_token * 2};
+  const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)kPfKeys};
+  return tc_make_tmap(tmap, base, 3, dims, strides, box);
+}
+
+}  // namespace
+
+size_t prefill_workspace_bytes() { return kHeaderBytes; }
+
+xkv_status prefill_attn(const xkv_dims* d, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                        int64_t total_tokens, int max_seqlen, void* out, float* lse, void* workspace,
+                        cudaStream_t st) {
+  PrefillParams p;
+  p.cu_seqlens = cu_seqlens;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = lse;
+  p.hdr = reinterpret_cast<WorkspaceHeader*>(workspace);
+  p.total_tokens = total_tokens;
+  p.batch = d->batch;
+  p.n_q_heads = d->n_q_heads;
+  p.n_kv_heads = d->n_kv_heads;
+  p.group = d->n_q_heads / d->n_kv_heads;
+  p.max_seqlen = max_seqlen;
+  const float scale = d->scale != 0.f ? d->scale : 1.0f / sqrtf((float)d->head_dim);
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.wait_ns = wait_limit_ns();
+  CUtensorMap tq, tk, tv;
+  if (!pf_make_tmap(&tq, q, d->head_dim, d->n_q_heads, total_tokens, (int64_t)d->n_q_heads * d->head_dim, d->head_dim) ||
+      !pf_make_tmap(&tk, k, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head) ||
+      !pf_make_tmap(&tv, v, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head))
+    return XKV_ERR_CUDA;
+  // an upper bound of the query tiles that exist: every sequence adds at most one partial tile
+  const int64_t tiles = total_tokens / kPfRows + d->batch;
+  const int64_t grid = tiles * d->n_q_heads;
+  if (grid > 0x7fffffffll) return XKV_ERR_UNSUPPORTED;
+  if (d->head_dim == 128) return pf_launch<128>(tq, tk, tv, p, (int)grid, st);
+  return pf_launch<64>(tq, tk, tv, p, (int)grid, st);
+}
+
+}  // namespace xkv

@@ -662,6 +662,21 @@ __global__ void __launch_bounds__(1024) mass_kernel(const ScoreParams p) {
   }
 }
 
+// mrow[unit][row] = the given softmax normaliser (natural log of the row's sum of exponentials) of window row
+// `row` = (query head within the group) * W + r, in log2 units; +inf for rows before the start of a sequence shorter
+// than the window, so that they contribute nothing.  grid = units, block = M.
+__global__ void mrow_from_lse_kernel(const ScoreParams p, const float* lse) {
+  const int unit = blockIdx.x, row = threadIdx.x;
+  if (row >= p.M) return;
+  const int b = unit / p.n_kv_heads, g = unit % p.n_kv_heads;
+  const int cu = p.cu_seqlens[b];
+  const int t = min(p.cu_seqlens[b + 1] - cu, p.max_seqlen);
+  const int h = g * p.group + row / p.window;
+  const int pos = t - p.window + row % p.window;
+  p.mrow[(size_t)unit * p.M + row] =
+      pos >= 0 ? lse[(size_t)h * p.total_tokens + cu + pos] * 1.4426950408889634f : INFINITY;
+}
+
 struct ScoreLayout {
   size_t flags, u, tmp_sorted, stats_part, mrow, part_sum, total;
   int split_keys, n_splits, n_chunks, slice_tiles, ctas_per_sm;
@@ -746,6 +761,12 @@ xkv_status launch_passes(const ScoreParams& p, const ScoreLayout& L, cudaStream_
 
 }  // namespace
 
+int score_lse_supported(const xkv_dims* d, int max_seqlen) {
+  ScoreLayout L;
+  score_layout(d, max_seqlen, max_seqlen, &L);
+  return L.use_tc ? 1 : 0;
+}
+
 size_t score_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_tokens) {
   ScoreLayout L;
   score_layout(d, max_seqlen, total_tokens, &L);
@@ -754,7 +775,7 @@ size_t score_workspace_bytes(const xkv_dims* d, int max_seqlen, int64_t total_to
 
 xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int32_t* cu_seqlens,
                  int64_t total_tokens, int max_seqlen, float* scores, float* sorted, float* gains, float* mass,
-                 int curve_len, void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                 int curve_len, void* workspace, size_t workspace_bytes, cudaStream_t st, const float* lse) {
   ScoreLayout L;
   score_layout(d, max_seqlen, total_tokens, &L);
   if (workspace_bytes < L.total) return XKV_ERR_WORKSPACE;
@@ -803,7 +824,15 @@ xkv_status score(const xkv_dims* d, const void* q_win, const void* k, const int3
   // counters, tickets and ready flags start at zero; the status word (first four bytes) keeps an unread error
   if (cudaMemsetAsync(ws + 4, 0, L.u - 4, st) != cudaSuccess) return XKV_ERR_CUDA;
   xkv_status s;
-  if (L.use_tc && score_fused_covers(p.M, d->head_dim, units, max_seqlen)) {
+  if (lse != nullptr) {
+    // the row normalisers come from the prefill attention: only the column-sum pass runs
+    if (!L.use_tc) return XKV_ERR_UNSUPPORTED;
+    mrow_from_lse_kernel<<<units, p.M, 0, st>>>(p, lse);
+    count_launch();
+    s = check_launch();
+    if (s != XKV_OK) return s;
+    s = score_tc_pass2(p, d->head_dim, max_seqlen, st);
+  } else if (L.use_tc && score_fused_covers(p.M, d->head_dim, units, max_seqlen)) {
     s = score_fused_pass(p, d->head_dim, max_seqlen, st);      // both passes in one cluster kernel, keys read once
   } else if (L.use_tc) {
     s = score_tc_passes(p, d->head_dim, max_seqlen, st);

@@ -408,6 +408,20 @@ int score_tc_split_keys(int M, int head_dim, int units, int max_seqlen) {
 #endif
 }
 
+xkv_status score_tc_pass2(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st) {
+  const int units = p.batch * p.n_kv_heads;
+  const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen);
+  if (tiles == 0 || tiles * kTcKeyTile != p.split_keys) return XKV_ERR_UNSUPPORTED;
+  CUtensorMap tq, tk;
+  if (!tc_make_score_tmaps(p, head_dim, &tq, &tk)) return XKV_ERR_CUDA;
+#define XKV_TC_CASE(DD, MM) \
+  if (head_dim == DD && p.M == MM) return tc_launch<DD, MM, 2>(tq, tk, p, st);
+  XKV_TC_CASE(128, 32) XKV_TC_CASE(128, 64) XKV_TC_CASE(128, 128) XKV_TC_CASE(128, 256)
+  XKV_TC_CASE(64, 32) XKV_TC_CASE(64, 64) XKV_TC_CASE(64, 128) XKV_TC_CASE(64, 256)
+#undef XKV_TC_CASE
+  return XKV_ERR_UNSUPPORTED;
+}
+
 xkv_status score_tc_passes(const ScoreParams& p, int head_dim, int max_seqlen, cudaStream_t st) {
   const int units = p.batch * p.n_kv_heads;
   const int tiles = tc_tiles(p.M, head_dim, units, max_seqlen);

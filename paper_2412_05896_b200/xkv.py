@@ -18,12 +18,12 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_BUDGET = -1, -2, -3, -4
 ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = -5, -6, -7
 POOL_MAX, POOL_AVG = 0, 1
-OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN = 0, 1, 2
+OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2, 3
 BUDGET_PER_LAYER, BUDGET_PER_SEQUENCE, BUDGET_PER_HEAD = 0, 1, 2
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
-EXPORTS = ("xkv_score", "xkv_batch_curves", "xkv_head_curves", "xkv_build_block_table", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
+EXPORTS = ("xkv_score", "xkv_score_lse", "xkv_prefill_attn", "xkv_batch_curves", "xkv_head_curves", "xkv_build_block_table", "xkv_alloc_budgets", "xkv_average_budgets", "xkv_select_compact", "xkv_decode_attn", "xkv_decode_attn_static",
            "xkv_workspace_bytes",
            "xkv_read_device_status", "xkv_profile_events", "xkv_test_hooks", "xkv_launch_count", "xkv_status_string",
            "xkv_version")
@@ -64,6 +64,10 @@ def lib() -> ctypes.CDLL:
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     L.xkv_score.restype = i32
     L.xkv_score.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.xkv_score_lse.restype = i32
+    L.xkv_score_lse.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, i64, i32, vp, vp, vp, vp, vp, i32, vp, sz, vp]
+    L.xkv_prefill_attn.restype = i32
+    L.xkv_prefill_attn.argtypes = [ctypes.POINTER(Dims), vp, vp, vp, vp, i64, i32, vp, vp, vp, sz, vp]
     L.xkv_batch_curves.restype = i32
     L.xkv_batch_curves.argtypes = [vp, i32, i32, i32, i32, vp, vp]
     L.xkv_head_curves.restype = i32
@@ -158,6 +162,22 @@ def score(dims: Dims, q_win, k, cu_seqlens, total_tokens: int, max_seqlen: int, 
     _check(lib().xkv_score(ctypes.byref(dims), _ptr(q_win), _ptr(k), _ptr(cu_seqlens), total_tokens, max_seqlen,
                            _ptr(scores), _ptr(sorted_scores), _ptr(gains), _ptr(mass), curve_len,
                            _ptr(workspace), _nbytes(workspace), _stream(stream)), "xkv_score")
+
+
+def score_lse(dims: Dims, q_win, k, cu_seqlens, total_tokens: int, max_seqlen: int, lse, scores, sorted_scores,
+              gains, mass, curve_len: int, workspace, stream=None) -> None:
+    """xkv_score with the window rows' normalisers given (lse dev fp32 [Hq, T] from prefill_attn)."""
+    _check(lib().xkv_score_lse(ctypes.byref(dims), _ptr(q_win), _ptr(k), _ptr(cu_seqlens), total_tokens, max_seqlen,
+                               _ptr(lse), _ptr(scores), _ptr(sorted_scores), _ptr(gains), _ptr(mass), curve_len,
+                               _ptr(workspace), _nbytes(workspace), _stream(stream)), "xkv_score_lse")
+
+
+def prefill_attn(dims: Dims, q, k, v, cu_seqlens, total_tokens: int, max_seqlen: int, out, lse, workspace,
+                 stream=None) -> None:
+    """q dev bf16 [T, Hq, d], k/v dev bf16 [T, Hkv, d] -> out dev bf16 [T, Hq, d], lse dev fp32 [Hq, T]."""
+    _check(lib().xkv_prefill_attn(ctypes.byref(dims), _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens), total_tokens,
+                                  max_seqlen, _ptr(out), _ptr(lse), _ptr(workspace), _nbytes(workspace),
+                                  _stream(stream)), "xkv_prefill_attn")
 
 
 def batch_curves(gains, n_layers: int, batch: int, curve_len: int, divisor: int, out, stream=None) -> None:
