@@ -54,6 +54,16 @@ def measured_peak():
         return 6650.0, "fallback (earlier measurement on this pool)"
 
 
+def measured_tflops():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            j = json.load(f)
+        return float(j["bf16_tflops"]), float(j["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return 1590.0, 1400.0, "fallback (earlier measurement on this pool)"
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -228,6 +238,7 @@ class Ctx:
         replicas.barrier()
         xkv.lib()
         self.peak, self.peak_src = measured_peak()
+        self.tf_burst, self.tf_sustained, self.tf_src = measured_tflops()
         self.sms = torch.cuda.get_device_properties(self.local).multi_processor_count
 
     def sync_all(self):
@@ -404,6 +415,66 @@ def run_workload(ctx: Ctx, name: str, steps: int, warmup: int, headline: bool) -
             "achieved": n_exp / (score_ms * 1e-3) / 1e9, "frac": n_exp / (score_ms * 1e-3) / xu_peak,
             "score_ms_per_layer": score_ms,
             "note": "time is the whole scoring phase per layer (logit passes, pooling, sort, curves)"}
+
+    # ---------------------------------------------------------------- prefill attention and scoring from its normalisers
+    # The step before the path (Alg. 2 step 1 takes W_attn from the layer's own attention): causal attention of every
+    # layer's prompt, timed per layer, whose row normalisers then let the scoring read the keys once.  Outside the
+    # timed region of the headline number; the queries are random with the window queries in their last rows.
+    if world == 1 and not args.no_prefill_attn:
+        T, Hq = sess.T, w.n_q_heads
+        lse_all = torch.empty(L, Hq, T, dtype=torch.float32, device=dev)
+        q_full = torch.empty(T, Hq, d, dtype=torch.bfloat16, device=dev)
+        o_full = torch.empty_like(q_full)
+        gen = torch.Generator(device=dev)
+        pf = [(ev(), ev()) for _ in range(L)]
+        for l in range(L):
+            gen.manual_seed(w.seed * 7919 + l)
+            q_full.normal_(generator=gen)
+            for b, t in enumerate(lengths):
+                n = min(W, t)
+                lo = int(sess.cu_host[b])
+                q_full[lo + t - n: lo + t] = q_win[l][b, :, W - n:].transpose(0, 1)
+            pf[l][0].record()
+            sess.prefill_attention(q_full, k[l], v[l], out=o_full, lse=lse_all[l])
+            pf[l][1].record()
+        torch.cuda.synchronize()
+        if sess.device_status("prefill") != xkv.OK:
+            raise SystemExit(f"{name}: prefill attention reported a device error")
+        pf_ms = np.array([a.elapsed_time(b) for a, b in pf])
+        flops = 4.0 * d * Hq * sum(t * (t + 1) / 2 for t in lengths)
+        tf = flops / (float(np.median(pf_ms)) * 1e-3) / 1e12
+        rec["prefill_attn"] = {
+            "kernel": "prefill_attn_kernel (tcgen05, causal, bf16 in, fp32 accumulate)", "layers_measured": L,
+            "ms_per_layer_median": float(np.median(pf_ms)), "flops_per_layer": flops, "achieved_TFLOPs": tf,
+            "frac_of_measured_bf16_burst": tf / ctx.tf_burst, "frac_of_measured_bf16_sustained": tf / ctx.tf_sustained,
+            "peak_source": ctx.tf_src,
+            "note": "4*d*Hq*sum_b t_b(t_b+1)/2 flops; outside the timed step (the model's own attention)"}
+        lse_list = [lse_all[l] for l in range(L)]
+        reps = 3
+        sess.score_layers(q_win, k, lse=lse_list)
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            sess.score_layers(q_win, k, lse=lse_list)
+        b_.record()
+        torch.cuda.synchronize()
+        check_status("scoring from the prefill normalisers")
+        score_lse_ms = a.elapsed_time(b_) / reps
+        se_lse = (score_lse_ms + float(phase[:, 2].mean())) / L
+        se_lse_gbps = pre_bytes / L / (se_lse * 1e-3) / 1e9
+        rec["score_from_prefill_lse"] = {
+            "score_ms": score_lse_ms, "score_evict_ms_per_layer": se_lse,
+            "score_evict_roofline": {"bound": "hbm", "algorithmic_bytes_per_layer": pre_bytes / L,
+                                     "achieved_GBps": se_lse_gbps, "frac_of_measured": se_lse_gbps / peak,
+                                     "frac_of_nominal_8000": se_lse_gbps / 8000.0},
+            "note": "xkv_score_lse: the window rows' normalisers come from xkv_prefill_attn, so scoring is one pass "
+                    "over the keys; select+compact time is that of the timed steps"}
+        if M >= 128:
+            n_exp1 = sum(Hkv * M * P for P in prefix)
+            mhz = (clocks or {}).get("sm_mhz") or 1965.0
+            rec["score_from_prefill_lse"]["xu_frac"] = n_exp1 / (score_lse_ms / L * 1e-3) / (16.0 * ctx.sms * mhz * 1e6)
+        del lse_all, q_full, o_full, lse_list
+        torch.cuda.empty_cache()
 
     # ---------------------------------------------------------------- full-cache decode, for comparison only
     if world == 1 and not args.no_full_cache and (headline or name == "llama3_8b_long" or args.full_cache_all):
@@ -654,6 +725,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle legs (CPU baseline and parity)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workloads' decode steps")
+    ap.add_argument("--no-prefill-attn", action="store_true",
+                    help="skip the prefill attention and the scoring from its normalisers")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the uncompressed-cache decode comparison")
     ap.add_argument("--full-cache-all", action="store_true", help="uncompressed-cache comparison for every workload")
     ap.add_argument("--lanes", type=int, default=None, help="side streams of the scoring and eviction phases")
@@ -700,6 +773,7 @@ def main():
         "phases_ms": head["phases_ms"], "solver_host_ms": head["solver_host_ms"], "budgets": head["budgets"],
         "timed_region_ms": head["timed_region_ms"],
         "full_cache_decode": head.get("full_cache_decode"),
+        "prefill_attn": head.get("prefill_attn"), "score_from_prefill_lse": head.get("score_from_prefill_lse"),
         "roofline": head["roofline"], "cpu_baseline": extras.get("cpu_baseline"), "e2e": extras.get("e2e"),
         "parity": extras.get("parity"),
         "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],

@@ -77,6 +77,7 @@ class XkvSession:
         self.ws_select = [self._ws(xkv.workspace_bytes(xkv.OP_SELECT_COMPACT, self.dims, self.max_seqlen, self.T))
                           for _ in range(n_ws)]
         self._lanes_busy = False
+        self.ws_prefill = None
 
         # ragged paged cache: a pool large enough for any split of the global budget
         per_layer_cap = min(max_budget if max_budget else self.max_prefix, self.max_prefix)
@@ -147,16 +148,24 @@ class XkvSession:
             self._lanes_busy = False
 
     def score_layer(self, layer: int, q_win: torch.Tensor, k: torch.Tensor, want_curves: bool = True,
-                    mass: torch.Tensor | None = None) -> None:
-        stream, i = self._lane(layer, q_win, k, mass)
-        xkv.score(self.dims, q_win, k, self.cu, self.T, self.max_seqlen, self.scores[layer],
-                  self.sorted[layer] if want_curves else None, self.gains[layer] if want_curves else None,
-                  mass, self.curve_len, self.ws_score[i], stream=stream)
+                    mass: torch.Tensor | None = None, lse: torch.Tensor | None = None) -> None:
+        """lse: fp32 [Hq, T] row normalisers of the layer's prefill attention (prefill_attention's second result);
+        with them the scores take one pass over the keys instead of two."""
+        stream, i = self._lane(layer, q_win, k, mass, lse)
+        srt = self.sorted[layer] if want_curves else None
+        gains = self.gains[layer] if want_curves else None
+        if lse is None:
+            xkv.score(self.dims, q_win, k, self.cu, self.T, self.max_seqlen, self.scores[layer], srt, gains, mass,
+                      self.curve_len, self.ws_score[i], stream=stream)
+        else:
+            xkv.score_lse(self.dims, q_win, k, self.cu, self.T, self.max_seqlen, lse, self.scores[layer], srt, gains,
+                          mass, self.curve_len, self.ws_score[i], stream=stream)
         if self.head_level and want_curves:
             xkv.head_curves(self.dims, self.scores[layer], self.sorted[layer], self.cu, self.T, self.max_seqlen,
                             self.head_gains[layer], self.curve_len, stream=stream)
 
-    def score_layers(self, q_win: list[torch.Tensor], k: list[torch.Tensor]) -> None:
+    def score_layers(self, q_win: list[torch.Tensor], k: list[torch.Tensor],
+                     lse: list[torch.Tensor] | None = None) -> None:
         """score_layer for every layer, with one fork and one join of the side streams for the whole phase (the
         inputs of all layers must be ready on the caller's stream at the call)."""
         cur = torch.cuda.current_stream()
@@ -169,10 +178,16 @@ class XkvSession:
         for l in range(self.L):
             i = l % len(streams)
             ws = self.ws_score[i]
-            st = lib.xkv_score(dims, q_win[l].data_ptr(), k[l].data_ptr(), cu, self.T, self.max_seqlen,
-                               self.scores.data_ptr() + l * esz, self.sorted.data_ptr() + l * esz,
-                               self.gains.data_ptr() + l * gsz, None, self.curve_len, ws.data_ptr(), ws.numel(),
-                               streams[i].cuda_stream)
+            if lse is None:
+                st = lib.xkv_score(dims, q_win[l].data_ptr(), k[l].data_ptr(), cu, self.T, self.max_seqlen,
+                                   self.scores.data_ptr() + l * esz, self.sorted.data_ptr() + l * esz,
+                                   self.gains.data_ptr() + l * gsz, None, self.curve_len, ws.data_ptr(), ws.numel(),
+                                   streams[i].cuda_stream)
+            else:
+                st = lib.xkv_score_lse(dims, q_win[l].data_ptr(), k[l].data_ptr(), cu, self.T, self.max_seqlen,
+                                       lse[l].data_ptr(), self.scores.data_ptr() + l * esz,
+                                       self.sorted.data_ptr() + l * esz, self.gains.data_ptr() + l * gsz, None,
+                                       self.curve_len, ws.data_ptr(), ws.numel(), streams[i].cuda_stream)
             if st < 0:
                 raise xkv.XkvError(st, "xkv_score")
             if self.head_level:
@@ -180,6 +195,19 @@ class XkvSession:
                                 self.head_gains[l], self.curve_len, stream=streams[i])
         self._lanes_busy = bool(self.lanes)
         self.join()
+
+    def prefill_attention(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor | None = None,
+                          lse: torch.Tensor | None = None):
+        """Causal attention of one layer's prompt: q [T, Hq, d], k/v [T, Hkv, d] -> (out [T, Hq, d] bf16,
+        lse [Hq, T] fp32).  The lse goes to score_layer(..., lse=) of that layer."""
+        if out is None:
+            out = torch.empty_like(q)
+        if lse is None:
+            lse = torch.empty(self.Hq, self.T, dtype=torch.float32, device=self.device)
+        if self.ws_prefill is None:
+            self.ws_prefill = self._ws(xkv.workspace_bytes(xkv.OP_PREFILL_ATTN, self.dims))
+        xkv.prefill_attn(self.dims, q, k, v, self.cu, self.T, self.max_seqlen, out, lse, self.ws_prefill)
+        return out, lse
 
     def select_layers(self, budgets, k: list[torch.Tensor], v: list[torch.Tensor]) -> None:
         """select_layer for every layer under one budget per layer ([L]), or per (layer, KV head) ([L, Hkv]) with
@@ -301,7 +329,8 @@ class XkvSession:
         """First error any call of that kind recorded since the last check (the status words are sticky and
         reading resets them), XKV_OK otherwise."""
         self.join()
-        ws = {"decode": [self.ws_decode], "score": self.ws_score, "select": self.ws_select}[which]
+        ws = {"decode": [self.ws_decode], "score": self.ws_score, "select": self.ws_select,
+              "prefill": [] if self.ws_prefill is None else [self.ws_prefill]}[which]
         first = xkv.OK
         for w in ws:
             st = xkv.read_device_status(w)
