@@ -105,7 +105,8 @@ __device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_
 constexpr int kWsThreads = 320;
 constexpr int kEpiThreads = 128;     // threads of one epilogue group
 constexpr int kWsStages = 4;       // shared-memory ring of key tiles
-constexpr int kAccBufs = 2;        // TMEM accumulator buffers
+constexpr int kAccBufs = 4;        // TMEM accumulator buffers of 128 columns
+constexpr int kEpiGroups = 2;      // epilogue groups (each takes every other tile)
 constexpr int kMrowSlots = 4;      // pass 2: ring of row-normaliser vectors (one per item in flight)
 
 template <int D, int M>
@@ -119,47 +120,53 @@ struct TcCfg {
   static constexpr int kQBufs = M == 256 ? 1 : 2;
   static constexpr int kKHalfBytes = kTcKeyTile * 128;
   static constexpr int kKTileBytes = kHalves * kKHalfBytes;
-  static constexpr uint32_t kBufCols = M == 256 ? 256 : 128;     // TMEM columns of one accumulator buffer
+  static constexpr uint32_t kBufCols = 128;                      // TMEM columns of one accumulator buffer
   static constexpr uint32_t kTmemCols = kAccBufs * kBufCols;
+  static constexpr int kJobs = M == 256 ? 2 : 1;                 // accumulator jobs per key tile
+  static constexpr int kJobRows = M == 256 ? 128 : M;            // pass 2: query rows (MMA N) of one job
   static constexpr int kColsPerThread = M < 128 ? M : 128;       // pass-1 key columns a thread reduces per tile
   static constexpr uint32_t kQTxBytes = (uint32_t)(kRep * kHalves * (M < 128 ? M : kQRows) * 128);
   static constexpr size_t kSmemBytes = 1024 + (size_t)kQBufs * kQBytes + (size_t)kWsStages * kKTileBytes +
                                        kMrowSlots * 256 * 4 /*row normalisers*/ + 256 /*barriers*/;
 };
 
-// Online-softmax update of one query row with 32 more logits v (raw dot products; scale > 0 folds 1/sqrt(d) and
+// Online-softmax update of one query row with 32*N more logits v (raw dot products; scale > 0 folds 1/sqrt(d) and
 // log2 e).  Tiles that reach into the observation window mask the keys the row must not see; all other tiles
 // skip that work (masked is the same for every thread of a tile).  Maximum and sum run as four independent
-// chains so that neither is one long dependent sequence.
-__device__ __forceinline__ void p1_update(const float (&v)[32], bool masked, int c0, int limit, float scale,
-                                          float& m, float& l) {
-  float x[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) x[i] = v[i];
+// chains so that neither is one long dependent sequence, and the running sum is rescaled once per call.
+template <int N>
+__device__ __forceinline__ void p1_update(float (&x)[N][32], bool masked, int c0, int limit, float scale, float& m,
+                                          float& l) {
   if (masked) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i)
-      if (c0 + i > limit) x[i] = -INFINITY;
-  }
-  float mx[4] = {x[0], x[1], x[2], x[3]};
+    for (int j = 0; j < N; ++j)
 #pragma unroll
-  for (int i = 4; i < 32; i += 4) {
-    mx[0] = fmaxf(mx[0], x[i]);
-    mx[1] = fmaxf(mx[1], x[i + 1]);
-    mx[2] = fmaxf(mx[2], x[i + 2]);
-    mx[3] = fmaxf(mx[3], x[i + 3]);
+      for (int i = 0; i < 32; ++i)
+        if (c0 + 32 * j + i > limit) x[j][i] = -INFINITY;
   }
+  float mx[4] = {x[0][0], x[0][1], x[0][2], x[0][3]};
+#pragma unroll
+  for (int j = 0; j < N; ++j)
+#pragma unroll
+    for (int i = (j == 0 ? 4 : 0); i < 32; i += 4) {
+      mx[0] = fmaxf(mx[0], x[j][i]);
+      mx[1] = fmaxf(mx[1], x[j][i + 1]);
+      mx[2] = fmaxf(mx[2], x[j][i + 2]);
+      mx[3] = fmaxf(mx[3], x[j][i + 3]);
+    }
   const float vmax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   const float m_new = fmaxf(m, vmax * scale);
   const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
   float sm[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int i = 0; i < 32; i += 4) {
-    sm[0] += fast_exp2(fmaf(x[i], scale, -m_ref));
-    sm[1] += fast_exp2(fmaf(x[i + 1], scale, -m_ref));
-    sm[2] += fast_exp2(fmaf(x[i + 2], scale, -m_ref));
-    sm[3] += fast_exp2(fmaf(x[i + 3], scale, -m_ref));
-  }
+  for (int j = 0; j < N; ++j)
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+      sm[0] += fast_exp2(fmaf(x[j][i], scale, -m_ref));
+      sm[1] += fast_exp2(fmaf(x[j][i + 1], scale, -m_ref));
+      sm[2] += fast_exp2(fmaf(x[j][i + 2], scale, -m_ref));
+      sm[3] += fast_exp2(fmaf(x[j][i + 3], scale, -m_ref));
+    }
   l = l * fast_exp2(m - m_ref) + ((sm[0] + sm[1]) + (sm[2] + sm[3]));
   m = m_new;
 }
