@@ -240,12 +240,20 @@ class XkvSession:
         self.join()
 
     def solve_budgets(self, total: int | None = None, r_target: float = 0.0, n_min: int = 0, n_max: int = 0,
-                      per_sequence: bool = False):
+                      per_sequence: bool = False, head_shards: int = 1, exchange=None):
         """Curves device -> host (the one crossing of the prefill), then Algorithm 1 on the host.  For one list per
-        batch the curves are averaged over the sequences on the device first, so L x curve_len numbers cross."""
+        batch the curves are averaged over the sequences on the device first, so L x curve_len numbers cross.
+
+        head_shards > 1: this session holds one of that many equal shares of the model's KV heads (one rank of a
+        KV-head-sharded run).  The layers' curves are then combined over the shards before the solver -- summed
+        (every shard contributes its heads' share of the layer mean), or with head-level budgets gathered, since
+        each (layer, KV head) unit lives on one shard -- and every shard solves the same problem; `total` counts
+        the whole model.  exchange(tensor) -> tensor does the combining: by default the torch.distributed
+        collectives of `replicas`; a test on one GPU passes a function that stands in for the other shards.
+        Returns this shard's budgets ([L], or [L, Hkv_local] with head-level budgets)."""
         self.join()
-        if per_sequence and self.head_level:
-            raise ValueError("per-sequence lists are not combined with head-level budgets in this session")
+        if per_sequence and (self.head_level or head_shards > 1):
+            raise ValueError("per-sequence lists are not combined with head-level budgets or head shards here")
         if per_sequence:
             if self.gains_host is None:
                 self.gains_host = torch.empty(self.L, self.B, self.curve_len, dtype=torch.float32, pin_memory=True)
@@ -253,11 +261,27 @@ class XkvSession:
             torch.cuda.current_stream().synchronize()
             gains, prefix = self.gains_host.numpy(), np.asarray(self.prefix, dtype=np.int32)
         else:
+            from . import replicas
             src = self.head_gains if self.head_level else self.gains        # [units, B, curve_len] either way
-            xkv.batch_curves(src, self.n_solver_units, self.B, self.curve_len, self.B, self.layer_gains)
-            self.layer_gains_host.copy_(self.layer_gains, non_blocking=True)
+            # layer curves: a shard's mean over its heads is 1/head_shards of the layer's mean over all heads
+            divisor = self.B * (1 if self.head_level else head_shards)
+            xkv.batch_curves(src, self.n_solver_units, self.B, self.curve_len, divisor, self.layer_gains)
+            curves = self.layer_gains
+            if head_shards > 1:
+                if self.head_level:
+                    local = curves.view(self.L, self.Hkv, self.curve_len)
+                    curves = (exchange or replicas.gather_unit_curves)(local).reshape(-1, self.curve_len)
+                else:
+                    curves = (exchange or replicas.sum_curves_over_ranks)(curves)
+            n_units = curves.shape[0]
+            if n_units == self.n_solver_units:
+                self.layer_gains_host.copy_(curves, non_blocking=True)
+                host = self.layer_gains_host
+            else:
+                host = torch.empty(n_units, self.curve_len, dtype=torch.float32, pin_memory=True)
+                host.copy_(curves, non_blocking=True)
             torch.cuda.current_stream().synchronize()
-            gains = self.layer_gains_host.numpy().reshape(self.n_solver_units, 1, self.curve_len)
+            gains = host.numpy().reshape(n_units, 1, self.curve_len)
             prefix = np.asarray([self.max_prefix], dtype=np.int32)
         t0 = time.perf_counter()
         budgets, r_avg = xkv.alloc_budgets(gains, prefix, per_sequence=per_sequence,
@@ -265,7 +289,11 @@ class XkvSession:
                                            r_target=r_target, n_min=n_min, n_max=n_max)
         self.last_solver_ms = 1e3 * (time.perf_counter() - t0)
         if self.head_level:
-            budgets = budgets.reshape(self.L, self.Hkv)          # one count per (layer, KV head)
+            budgets = budgets.reshape(self.L, -1)                # one count per (layer, KV head of the whole model)
+            if head_shards > 1:
+                from . import replicas
+                rank = replicas.env_ranks()[0] if exchange is None else getattr(exchange, "rank", 0)
+                budgets = np.ascontiguousarray(budgets[:, rank * self.Hkv: (rank + 1) * self.Hkv])
         self.budgets, self.r_avg = budgets, r_avg
         return budgets, r_avg
 

@@ -1,7 +1,13 @@
-"""Host-side plumbing of the multi-GPU mode: N replicas, one process per GPU, each with its own batch.
+"""Host-side plumbing of the multi-GPU modes, one process per GPU.
 
-The path shards by independent units (sequence x KV head x layer), so no tensor of the method crosses GPUs and
-there is no collective on the data path; what the ranks exchange is a barrier and the reductions of the timing.
+Replicas: every rank has its own batch.  The path shards by independent units (sequence x KV head x layer), so no
+tensor of the method crosses GPUs and there is no collective on the data path; what the ranks exchange is a barrier
+and the reductions of the timing.
+
+KV-head shards: every rank holds an equal share of the KV heads (with their query heads) of every layer and
+sequence, as a tensor-parallel model does.  K, V, scores and caches stay on their GPU; the one exchange is the
+layers' curves before the solver (head_shard, sum_curves_over_ranks, gather_unit_curves).
+
 The functions work on any torch.distributed backend (nccl on GPUs, gloo in the CPU tests).
 """
 from __future__ import annotations
@@ -84,3 +90,24 @@ def sum_curves_over_ranks(local_curves: torch.Tensor) -> torch.Tensor:
     if dist.is_initialized() and dist.get_world_size() > 1:
         dist.all_reduce(local_curves, op=dist.ReduceOp.SUM)
     return local_curves
+
+
+def head_shard(n_q_heads: int, n_kv_heads: int, rank: int, world: int) -> tuple[slice, slice]:
+    """(KV heads, query heads) of one of `world` equal shards: consecutive KV heads with the query heads of their
+    groups, so that a shard is a smaller model of the same group size."""
+    if n_kv_heads % world != 0:
+        raise ValueError("the KV heads do not divide evenly over the ranks")
+    per = n_kv_heads // world
+    group = n_q_heads // n_kv_heads
+    return slice(rank * per, (rank + 1) * per), slice(rank * per * group, (rank + 1) * per * group)
+
+
+def gather_unit_curves(local_curves: torch.Tensor) -> torch.Tensor:
+    """Head-level budgets over KV-head shards: the solver's units are (layer, KV head) pairs and every rank holds
+    the curves of its own heads.  local_curves [L, Hkv_local, curve_len] -> [L, Hkv, curve_len] with the heads in
+    rank order (all-gather); every rank then solves for all units and keeps the budgets of its heads."""
+    if not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_curves
+    parts = [torch.empty_like(local_curves) for _ in range(dist.get_world_size())]
+    dist.all_gather(parts, local_curves.contiguous())
+    return torch.cat(parts, dim=1)

@@ -103,6 +103,60 @@ def test_budget_list_shared_by_all_ranks_equals_the_list_of_the_whole_batch():
         assert budgets == whole and sum(budgets) == 60 and err < 1e-6
 
 
+def _head_shard_worker(rank: int, world: int, port: int, out):
+    import numpy as np
+    from oracle import xkv_oracle as O
+    from paper_2412_05896_b200 import xkv
+    os.environ.update(RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank), MASTER_ADDR="127.0.0.1",
+                      MASTER_PORT=str(port))
+    replicas.init("gloo")
+    L, Hq, Hkv, n = 4, 8, 4, 30
+    rng = np.random.default_rng(91)
+    w_heads = [[rng.random(n) ** (2 + l + g) for g in range(Hkv)] for l in range(L)]          # one sequence
+    kv, qh = replicas.head_shard(Hq, Hkv, rank, world)
+    assert (kv, qh) == (slice(2 * rank, 2 * rank + 2), slice(4 * rank, 4 * rank + 4))
+    # layer budgets: this shard's mean over its heads, divided by the number of shards, summed over the ranks
+    mine = np.stack([O.layer_gains(w_heads[l][kv], n) for l in range(L)]) / world
+    layer = replicas.sum_curves_over_ranks(torch.from_numpy(mine.astype(np.float32).astype(np.float64))).numpy()
+    whole = np.stack([O.layer_gains(w_heads[l], n) for l in range(L)])
+    b_layer, _ = xkv.alloc_budgets(layer[:, None, :].astype(np.float32), [n], total=40)
+    b_whole, _ = xkv.alloc_budgets(whole[:, None, :].astype(np.float32), [n], total=40)
+    # head-level budgets: the units' curves are gathered in rank order
+    local_units = torch.from_numpy(np.stack([[O.head_gains(w) for w in w_heads[l][kv]] for l in range(L)])
+                                   .astype(np.float32))                                        # [L, 2, n]
+    units = replicas.gather_unit_curves(local_units).numpy()                                   # [L, 4, n]
+    ref_units = np.stack([[O.head_gains(w) for w in w_heads[l]] for l in range(L)]).astype(np.float32)
+    b_units, _ = xkv.alloc_budgets(units.reshape(L * Hkv, 1, n), [n], total=160)
+    n_ref, _ = O.head_level_allocation(w_heads, N=160)
+    out.put((rank, float(np.abs(layer - whole).max()), b_layer.tolist(), b_whole.tolist(),
+             bool(np.array_equal(units, ref_units)), b_units.reshape(L, Hkv).tolist(), n_ref))
+    dist.destroy_process_group()
+
+
+def test_kv_head_shards_exchange_curves_before_the_solver():
+    """A KV-head-sharded run: the layer curve is the sum over the ranks of each rank's share, the per-head curves
+    are gathered in rank order, and both give the budgets of the unsharded problem."""
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_head_shard_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert results[0][2] == results[1][2] and results[0][5] == results[1][5], "every rank derives the same lists"
+    for rank, err, b_layer, b_whole, same_units, b_units, n_ref in results:
+        assert err < 1e-7 and b_layer == b_whole and sum(b_layer) == 40
+        assert same_units and b_units == n_ref
+    try:
+        replicas.head_shard(8, 4, 0, 3)
+        raise AssertionError("uneven shards must be refused")
+    except ValueError:
+        pass
+
+
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
