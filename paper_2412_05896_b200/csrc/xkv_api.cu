@@ -73,6 +73,10 @@ xkv_status check_cache(const xkv_cache* c, const xkv_dims* d) {
   if (c->n_layers <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return XKV_ERR_INVALID_ARG;
   if (c->page_size <= 0 || c->page_size % 16 != 0 || c->page_size > 256) return XKV_ERR_INVALID_ARG;
   if ((int64_t)c->max_pages_per_seq * c->page_size > (1 << 30)) return XKV_ERR_INVALID_ARG;
+  if (c->kv_format != XKV_KV_BF16 && c->kv_format != XKV_KV_FP8_E4M3) return XKV_ERR_INVALID_ARG;
+  if (c->kv_format == XKV_KV_FP8_E4M3 &&
+      (c->k_scales == nullptr || c->v_scales == nullptr || !aligned16(c->k_scales) || !aligned16(c->v_scales)))
+    return XKV_ERR_INVALID_ARG;
   (void)d;
   return XKV_OK;
 }
@@ -251,6 +255,7 @@ xkv_status xkv_decode_attn_static(const xkv_dims* dims, const xkv_cache* cache, 
   if (layer_begin < 0 || layer_end <= layer_begin || layer_end > cache->n_layers) return XKV_ERR_INVALID_ARG;
   if (chunk_rows < 0 || chunk_rows % 64 != 0) return XKV_ERR_INVALID_ARG;
   if (dims->n_q_heads / dims->n_kv_heads > 8) return XKV_ERR_UNSUPPORTED;
+  if (cache->kv_format != XKV_KV_BF16) return XKV_ERR_UNSUPPORTED;
   return decode_attn_static(dims, cache, layer_begin, layer_end, q, k_new, v_new, out, lse, chunk_rows,
                             status_out, static_cast<cudaStream_t>(stream));
 }

@@ -64,8 +64,10 @@ struct DecodeParams {
   const __nv_bfloat16* v_new;
   __nv_bfloat16* out;
   float* lse;
-  __nv_bfloat16* k_pages;
+  __nv_bfloat16* k_pages;   // uint8 codes when the cache is stored in 8 bits
   __nv_bfloat16* v_pages;
+  float* k_scales;          // 8-bit caches: one fp32 scale per cached row, [n_pages][Hkv][page_size]
+  float* v_scales;
   const int32_t* block_table;
   int32_t* seq_lens;
   int32_t layer_begin, n_layers, batch, n_q_heads, n_kv_heads, group;
@@ -84,17 +86,43 @@ struct DecodeParams {
   float* part_ml;     // [max_items][G][2]
 };
 
-template <int D>
+// Q8: the cache holds 8-bit codes and per-row scales.  A stage of the ring is then the raw tile as it lies in the
+// pages (K codes, V codes, K scales, V scales); the warp expands K and V into two 16-bit tiles of its own, in the same
+// swizzled layout a 16-bit TMA box has, and the rest of the tile's work reads those.
+template <int D, bool Q8>
 struct Cfg {
   static constexpr int kHalves = D / 64;                       // 128-byte swizzled column halves
-  static constexpr int kBoxBytes = kTileRows * 128;            // one half of a K or V tile (one TMA box)
+  static constexpr int kBoxBytes = kTileRows * 128;            // one half of a 16-bit K or V tile (one TMA box)
   static constexpr int kTileBytes = kHalves * kBoxBytes;
-  static constexpr int kStageBytes = 2 * kTileBytes;           // K tile + V tile
-  static constexpr int kStages = (D == 128) ? 3 : 6;
-  static constexpr int kRingBytes = kStages * kStageBytes;     // per warp
+  static constexpr int kRawTileBytes = kTileRows * D;          // Q8: one tile of codes
+  static constexpr int kScaleBytes = kTileRows * 4;            // Q8: the scales of a tile's rows
+  static constexpr int kStageBytes = Q8 ? 2 * kRawTileBytes + 2 * kScaleBytes : 2 * kTileBytes;   // K tile + V tile
+  static constexpr int kStages = Q8 ? ((D == 128) ? 4 : 8) : ((D == 128) ? 3 : 6);
+  static constexpr int kExpandBytes = Q8 ? 2 * kTileBytes : 0; // Q8: the expanded K tile and V tile
+  static constexpr int kRingBytes = kStages * kStageBytes + kExpandBytes;     // per warp
   static constexpr int kSmemBytes = 1024 + kAttnWarps * kRingBytes + kAttnWarps * kStages * 8 +
                                     kAttnWarps * kFifo * 20 + (kMaxPlanUnits + 1) * 4 + kMaxPlanUnits * 2 + 64;
 };
+
+// fp16 tensor-core tile for the 8-bit caches (the codes are exact in fp16).
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// Plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
 
 // ---------------------------------------------------------------------------------------------
 // Append (optional) and plan.  grid = n_layers*batch CTAs when appending, else 1.
@@ -110,7 +138,7 @@ __device__ __forceinline__ int choose_chunk(long long total, int forced) {
 }
 
 // Stores the new K/V row of every KV head of unit e = (layer, sequence) in slot seq_lens and advances seq_lens.
-__device__ __forceinline__ void append_unit(const DecodeParams& p, int D, int e, int* s_page) {
+__device__ __forceinline__ void append_unit(const DecodeParams& p, int D, int e, int* s_page, bool q8) {
   const int tid = threadIdx.x;
   const int l_rel = e / p.batch, b = e % p.batch;
   const int le = (p.layer_begin + l_rel) * p.batch + b;
@@ -132,10 +160,28 @@ __device__ __forceinline__ void append_unit(const DecodeParams& p, int D, int e,
     const int chunks = D / 8;
     for (int idx = tid; idx < p.n_kv_heads * chunks; idx += blockDim.x) {
       const int h = idx / chunks, c = idx % chunks;
-      const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size) * D + c * 8;
+      const size_t slot = ((size_t)page * p.n_kv_heads + h) * p.page_size + n % p.page_size;
+      const size_t dst = slot * D + c * 8;
       const size_t src = ((size_t)e * p.n_kv_heads + h) * D + c * 8;
-      *reinterpret_cast<uint4*>(p.k_pages + dst) = *reinterpret_cast<const uint4*>(p.k_new + src);
-      *reinterpret_cast<uint4*>(p.v_pages + dst) = *reinterpret_cast<const uint4*>(p.v_new + src);
+      const uint4 kv = *reinterpret_cast<const uint4*>(p.k_new + src);
+      const uint4 vv = *reinterpret_cast<const uint4*>(p.v_new + src);
+      if (q8) {
+        // a row's pieces sit on consecutive threads (D/8 of them, whole rows per warp)
+        float x[8], ks, vs;
+        bf16x8_to_f32(kv, x);
+        const uint2 kc = quantize_row_piece(x, chunks, &ks);
+        bf16x8_to_f32(vv, x);
+        const uint2 vc = quantize_row_piece(x, chunks, &vs);
+        *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.k_pages) + dst) = kc;
+        *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.v_pages) + dst) = vc;
+        if (c == 0) {
+          p.k_scales[slot] = ks;
+          p.v_scales[slot] = vs;
+        }
+      } else {
+        *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
+        *reinterpret_cast<uint4*>(p.v_pages + dst) = vv;
+      }
     }
     if (tid == 0) p.seq_lens[le] = n + 1;
   }
@@ -228,11 +274,11 @@ __device__ void plan_items(const DecodeParams& p) {
   }
 }
 
-__global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodeParams p, int D, int do_append) {
+__global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodeParams p, int D, int do_append, int q8) {
   __shared__ int s_page;
   __shared__ int s_last;
   const int tid = threadIdx.x;
-  if (do_append) append_unit(p, D, blockIdx.x, &s_page);
+  if (do_append) append_unit(p, D, blockIdx.x, &s_page, q8 != 0);
   // the last CTA to get here sees every sequence length already advanced and writes the plan
   __threadfence();
   __syncthreads();
@@ -247,15 +293,17 @@ __global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodePara
 }
 
 // ---------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool Q8>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const DecodeParams p) {
-  using C = Cfg<D>;
+  using C = Cfg<D, Q8>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint8_t* ring = smem + (size_t)warp * C::kRingBytes;
+  uint8_t* k_exp = ring + (size_t)C::kStages * C::kStageBytes;   // Q8: this warp's expanded K tile, then its V tile
+  uint8_t* v_exp = k_exp + C::kTileBytes;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes) + warp * C::kStages;
   uint8_t* fifo_base = smem + (size_t)kAttnWarps * C::kRingBytes + kAttnWarps * C::kStages * 8;
   int4* fifo = reinterpret_cast<int4*>(fifo_base) + warp * kFifo;                        // item descriptors
@@ -441,12 +489,21 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const int grow = (page * p.n_kv_heads + p_desc.y) * p.page_size + p_row % p.page_size;
         const int s = issued % C::kStages;
         uint8_t* ks = ring + (size_t)s * C::kStageBytes;
-        uint8_t* vs = ks + C::kTileBytes;
         mbar_arrive_expect_tx(&full_bar[s], kTxBytes);
+        if constexpr (Q8) {
+          // raw codes of the 16 rows (one box of D bytes per row) and their scales (16 consecutive floats)
+          uint8_t* vs = ks + C::kRawTileBytes;
+          tma_load_2d(ks, &tmap_k, 0, grow, &full_bar[s]);
+          tma_load_2d(vs, &tmap_v, 0, grow, &full_bar[s]);
+          bulk_copy_g2s(vs + C::kRawTileBytes, p.k_scales + grow, C::kScaleBytes, &full_bar[s]);
+          bulk_copy_g2s(vs + C::kRawTileBytes + C::kScaleBytes, p.v_scales + grow, C::kScaleBytes, &full_bar[s]);
+        } else {
+          uint8_t* vs = ks + C::kTileBytes;
 #pragma unroll
-        for (int hf = 0; hf < C::kHalves; ++hf) {
-          tma_load_2d(ks + hf * C::kBoxBytes, &tmap_k, hf * 64, grow, &full_bar[s]);
-          tma_load_2d(vs + hf * C::kBoxBytes, &tmap_v, hf * 64, grow, &full_bar[s]);
+          for (int hf = 0; hf < C::kHalves; ++hf) {
+            tma_load_2d(ks + hf * C::kBoxBytes, &tmap_k, hf * 64, grow, &full_bar[s]);
+            tma_load_2d(vs + hf * C::kBoxBytes, &tmap_v, hf * 64, grow, &full_bar[s]);
+          }
         }
       }
       ++issued;
@@ -503,6 +560,10 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const __nv_bfloat16* qp = p.q + (q_row0 + gid) * D + 16 * ks + 2 * tig;
         qb[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
         qb[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
+        if constexpr (Q8) {           // the 8-bit path multiplies in fp16
+          qb[ks][0] = pack_f16(bf16_lo(qb[ks][0]), bf16_hi(qb[ks][0]));
+          qb[ks][1] = pack_f16(bf16_lo(qb[ks][1]), bf16_hi(qb[ks][1]));
+        }
       }
     }
     float o[D / 16][4];               // O^T: [mt] = columns 16*mt + gid (regs 0,1) and + 8 (regs 2,3); heads 2*tig, +1
@@ -512,18 +573,56 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     float l_part[2] = {0.f, 0.f};
 
     // S^T of one 16-row tile: rows gid (regs 0,1) and gid + 8 (regs 2,3), heads 2*tig, 2*tig + 1
+    // Q8: expands a tile of codes (16 rows of D bytes, rows contiguous) into the warp's 16-bit tile: rows of 128 bytes
+    // per 64 columns, 16-byte pieces at their swizzled places, exactly what a 16-bit TMA box would have written.
+    auto expand_tile = [&](const uint8_t* raw, uint8_t* dst) {
+      constexpr int kPieces = kTileRows * D / 16;               // 16-code pieces of the tile
+#pragma unroll
+      for (int i = 0; i < kPieces / 32; ++i) {
+        const int q = lane + 32 * i;
+        const int r = q / (D / 16), c16 = q % (D / 16);         // row, 16-code piece of the row
+        const uint4 w = *reinterpret_cast<const uint4*>(raw + q * 16);
+        uint4 lo, hi;
+        lo.x = e4m3x2_to_f16x2((uint16_t)(w.x & 0xffffu)); lo.y = e4m3x2_to_f16x2((uint16_t)(w.x >> 16));
+        lo.z = e4m3x2_to_f16x2((uint16_t)(w.y & 0xffffu)); lo.w = e4m3x2_to_f16x2((uint16_t)(w.y >> 16));
+        hi.x = e4m3x2_to_f16x2((uint16_t)(w.z & 0xffffu)); hi.y = e4m3x2_to_f16x2((uint16_t)(w.z >> 16));
+        hi.z = e4m3x2_to_f16x2((uint16_t)(w.w & 0xffffu)); hi.w = e4m3x2_to_f16x2((uint16_t)(w.w >> 16));
+        const int c = (2 * c16) & 7;                            // first of the two 8-element pieces, within its half
+        uint8_t* row = dst + ((2 * c16) >> 3) * C::kBoxBytes + r * 128;
+        *reinterpret_cast<uint4*>(row + ((c ^ (r & 7)) << 4)) = lo;
+        *reinterpret_cast<uint4*>(row + (((c + 1) ^ (r & 7)) << 4)) = hi;
+      }
+      __syncwarp();
+    };
     auto qk_tile = [&](uint32_t idx, float (&acc)[4]) {
-      const uint32_t ks_base = smem_u32(ring + (size_t)(idx % C::kStages) * C::kStageBytes);
+      uint8_t* stage = ring + (size_t)(idx % C::kStages) * C::kStageBytes;
+      uint32_t ks_base = smem_u32(stage);
+      if constexpr (Q8) {
+        expand_tile(stage, k_exp);
+        ks_base = smem_u32(k_exp);
+      }
       float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) {
         uint32_t af[4];
         ldmatrix_x4(af, ks_base + (ks >> 2) * C::kBoxBytes + (k_lane_off ^ (uint32_t)(((2 * ks) & 7) << 4)));
-        if (ks & 1) mma_bf16_16816(a1, af, qb[ks][0], qb[ks][1]);
-        else        mma_bf16_16816(a0, af, qb[ks][0], qb[ks][1]);
+        if constexpr (Q8) {
+          if (ks & 1) mma_f16_16816(a1, af, qb[ks][0], qb[ks][1]);
+          else        mma_f16_16816(a0, af, qb[ks][0], qb[ks][1]);
+        } else {
+          if (ks & 1) mma_bf16_16816(a1, af, qb[ks][0], qb[ks][1]);
+          else        mma_bf16_16816(a0, af, qb[ks][0], qb[ks][1]);
+        }
       }
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[i] = a0[i] + a1[i];
+      if constexpr (Q8) {
+        // the rows' scales: keys gid (registers 0, 1) and gid + 8 (registers 2, 3)
+        const float* kscale = reinterpret_cast<const float*>(stage + 2 * C::kRawTileBytes);
+        const float s0 = kscale[gid], s1 = kscale[gid + 8];
+        acc[0] *= s0; acc[1] *= s0; acc[2] *= s1; acc[3] *= s1;
+        __syncwarp();                 // every lane is done with the expanded K tile before the next one overwrites it
+      }
     };
 
     const int n_tiles = (I.w - I.z + kTileRows - 1) / kTileRows;
@@ -545,6 +644,29 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       const int page = p.block_table[(size_t)le * p.max_pages_per_seq + new_slot / p.page_size];
       const bool page_ok = page >= 0 && page < p.n_pages;
       if (!page_ok && lane == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
+      if constexpr (Q8) {
+        // The new row is quantised here (its D/8 pieces on consecutive lanes: K on the first D/8 lanes, V on the next
+        // ones), its codes and scales go into the raw tile, where the expansion picks them up, and into the page.
+        static_assert(2 * kPieces <= 32, "one warp holds the K and V pieces of a row");
+        if (lane < 2 * kPieces) {
+          const int is_v = lane / kPieces, c = lane % kPieces;
+          float x[8], sc;
+          bf16x8_to_f32(*reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8), x);
+          const uint2 codes = quantize_row_piece(x, kPieces, &sc);
+          uint8_t* raw = ks + is_v * C::kRawTileBytes;
+          *reinterpret_cast<uint2*>(raw + r * D + c * 8) = codes;
+          float* tile_scales = reinterpret_cast<float*>(ks + 2 * C::kRawTileBytes + is_v * C::kScaleBytes);
+          if (c == 0) tile_scales[r] = sc;
+          if (page_ok) {
+            const size_t slot = ((size_t)page * p.n_kv_heads + h) * p.page_size + new_slot % p.page_size;
+            *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(is_v ? p.v_pages : p.k_pages) + slot * D + c * 8) = codes;
+            if (c == 0) (is_v ? p.v_scales : p.k_scales)[slot] = sc;
+          }
+        }
+        fence_proxy_async_smem();     // the stage is written again by a later copy
+        __syncwarp();
+        return;
+      }
       for (int i = lane; i < 2 * kPieces; i += 32) {
         const int is_v = i / kPieces, c = i % kPieces;
         const uint4 val = *reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8);
@@ -576,13 +698,21 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (!aborted) qk_tile(consumed + 1, s_next);
       }
       if (!aborted) {
-        const uint32_t vs_base = smem_u32(ring + (size_t)s * C::kStageBytes) + C::kTileBytes;
+        uint8_t* stage = ring + (size_t)s * C::kStageBytes;
+        float vs0 = 1.f, vs1 = 1.f;                    // Q8: scales of the V rows gid and gid + 8
+        if constexpr (Q8) {
+          expand_tile(stage + C::kRawTileBytes, v_exp);
+          const float* vscale = reinterpret_cast<const float*>(stage + 2 * C::kRawTileBytes + C::kScaleBytes);
+          vs0 = gid < wrows ? vscale[gid] : 0.f;       // rows past the end of the cache carry no weight at all
+          vs1 = gid + 8 < wrows ? vscale[gid + 8] : 0.f;
+        }
+        const uint32_t vs_base = Q8 ? smem_u32(v_exp) : smem_u32(stage) + C::kTileBytes;
         if (wrows < kTileRows) {
           // rows past the end of the cache hold whatever the page held: mask their scores and clear V so
           // that 0 * x stays 0
           if (gid >= wrows) sv[0] = sv[1] = -INFINITY;
           if (gid + 8 >= wrows) sv[2] = sv[3] = -INFINITY;
-          uint8_t* vs = ring + (size_t)s * C::kStageBytes + C::kTileBytes;
+          uint8_t* vs = Q8 ? v_exp : stage + C::kTileBytes;
           const int n_bad = kTileRows - wrows;
           for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
             const int row = wrows + idx / (D / 8);
@@ -620,13 +750,14 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         l_part[0] += p0 + p2;
         l_part[1] += p1 + p3;
         // P^T as the B operand of O^T += V^T.P^T: transpose the two 8x8 blocks of the accumulator layout
-        const uint32_t b0 = movmatrix_trans(pack_bf16(p0, p1));
-        const uint32_t b1 = movmatrix_trans(pack_bf16(p2, p3));
+        const uint32_t b0 = movmatrix_trans(Q8 ? pack_f16(p0 * vs0, p1 * vs0) : pack_bf16(p0, p1));
+        const uint32_t b1 = movmatrix_trans(Q8 ? pack_f16(p2 * vs1, p3 * vs1) : pack_bf16(p2, p3));
 #pragma unroll
         for (int mt = 0; mt < D / 16; ++mt) {
           uint32_t af[4];
           ldmatrix_x4_trans(af, vs_base + (mt >> 2) * C::kBoxBytes + (v_lane_off ^ (uint32_t)(((2 * mt) & 7) << 4)));
-          mma_bf16_16816(o[mt], af, b0, b1);
+          if constexpr (Q8) mma_f16_16816(o[mt], af, b0, b1);
+          else              mma_bf16_16816(o[mt], af, b0, b1);
         }
       }
       __syncwarp();
@@ -816,13 +947,21 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows) {
+bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows, bool q8) {
   EncodeTiledFn enc = encode_tiled_fn();
   if (enc == nullptr) return false;
   const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+  const cuuint32_t estr[2] = {1u, 1u};
+  if (q8) {
+    // one byte per element: a box is 16 whole rows of D bytes, stored as they are (no swizzle)
+    const cuuint64_t gstride[1] = {(cuuint64_t)D};
+    const cuuint32_t box[2] = {(cuuint32_t)D, (cuuint32_t)kTileRows};
+    return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  }
   const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
   const cuuint32_t box[2] = {64u, (cuuint32_t)kTileRows};
-  const cuuint32_t estr[2] = {1u, 1u};
   return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -861,7 +1000,7 @@ bool decode_layout(const xkv_dims* d, int n_layers, int max_cache_len, int chunk
 
 cudaEvent_t g_ev_start = nullptr, g_ev_stop = nullptr;
 
-template <int D>
+template <int D, bool Q8>
 xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const DecodeParams& p, cudaStream_t st) {
   cudaError_t attr_err = cudaSuccess;
   // opt in to the large dynamic shared-memory carve-out once per process and device in use
@@ -870,13 +1009,13 @@ xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const Decod
   static std::atomic<bool> done[64];   // idempotent set-up: two threads doing it twice is harmless
   if (dev < 0 || dev >= 64) return XKV_ERR_CUDA;
   if (!done[dev].load(std::memory_order_acquire)) {
-    attr_err = cudaFuncSetAttribute(decode_attn_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    Cfg<D>::kSmemBytes);
+    attr_err = cudaFuncSetAttribute(decode_attn_kernel<D, Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    Cfg<D, Q8>::kSmemBytes);
     if (attr_err != cudaSuccess) return XKV_ERR_CUDA;
     done[dev].store(true, std::memory_order_release);
   }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_start, st);
-  decode_attn_kernel<D><<<sm_count(), kAttnThreads, Cfg<D>::kSmemBytes, st>>>(tk, tv, p);
+  decode_attn_kernel<D, Q8><<<sm_count(), kAttnThreads, Cfg<D, Q8>::kSmemBytes, st>>>(tk, tv, p);
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_stop, st);
   count_launch();
   return check_launch();
@@ -909,9 +1048,10 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   const uint64_t page_rows = (uint64_t)c->n_pages * d->n_kv_heads * c->page_size;
   if (page_rows >= (1ull << 31)) return XKV_ERR_UNSUPPORTED;
 
+  const bool q8 = c->kv_format == XKV_KV_FP8_E4M3;
   CUtensorMap tk, tv;
-  if (!make_page_tmap(&tk, c->k_pages, d->head_dim, page_rows) ||
-      !make_page_tmap(&tv, c->v_pages, d->head_dim, page_rows))
+  if (!make_page_tmap(&tk, c->k_pages, d->head_dim, page_rows, q8) ||
+      !make_page_tmap(&tv, c->v_pages, d->head_dim, page_rows, q8))
     return XKV_ERR_CUDA;
 
   uint8_t* ws = static_cast<uint8_t*>(workspace);
@@ -923,6 +1063,8 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   p.lse = lse;
   p.k_pages = static_cast<__nv_bfloat16*>(c->k_pages);
   p.v_pages = static_cast<__nv_bfloat16*>(c->v_pages);
+  p.k_scales = c->k_scales;
+  p.v_scales = c->v_scales;
   p.block_table = c->block_table;
   p.seq_lens = c->seq_lens;
   p.layer_begin = layer_begin;
@@ -959,13 +1101,13 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   const size_t keep = clear_status ? 0 : sizeof(int32_t);
   if (cudaMemsetAsync(ws + keep, 0, L.unit_info - keep, st) != cudaSuccess) return XKV_ERR_CUDA;
   if (!p.fused_plan) {
-    decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append);
+    decode_prepare_kernel<<<do_append ? n_units : 1, kPrepThreads, 0, st>>>(p, d->head_dim, do_append, q8 ? 1 : 0);
     count_launch();
     xkv_status s = check_launch();
     if (s != XKV_OK) return s;
   }
-  if (d->head_dim == 128) return launch_attn<128>(tk, tv, p, st);
-  return launch_attn<64>(tk, tv, p, st);
+  if (q8) return d->head_dim == 128 ? launch_attn<128, true>(tk, tv, p, st) : launch_attn<64, true>(tk, tv, p, st);
+  return d->head_dim == 128 ? launch_attn<128, false>(tk, tv, p, st) : launch_attn<64, false>(tk, tv, p, st);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -38,6 +38,9 @@ struct SelectParams {
   const __nv_bfloat16* v;
   __nv_bfloat16* k_pages;
   __nv_bfloat16* v_pages;
+  float* k_scales;             // 8-bit caches only: one scale per cached row
+  float* v_scales;
+  int32_t kv_format;
   int64_t total_tokens, stride_token, stride_head;
   int32_t batch, n_kv_heads, head_dim, window, page_size, max_pages_per_seq, n_pages;
   int2* counts;                // [units][n_chunks] scores above / equal to the threshold per chunk (chunked path)
@@ -280,11 +283,27 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
       continue;
     }
     const size_t src = (size_t)(cu + pos) * p.stride_token + (size_t)g * p.stride_head + lc * 8;
-    const size_t dst = (((size_t)page * page_heads + page_head) * p.page_size + r % p.page_size) * p.head_dim + lc * 8;
+    const size_t slot = ((size_t)page * page_heads + page_head) * p.page_size + r % p.page_size;
+    const size_t dst = slot * p.head_dim + lc * 8;
     const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k + src));
     const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v + src));
-    *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
-    *reinterpret_cast<uint4*>(p.v_pages + dst) = vv;
+    if (p.kv_format == XKV_KV_FP8_E4M3) {
+      // the row's lanes (consecutive lanes of the warp) agree on its scale; a lane stores its eight codes
+      float x[8], ks, vs;
+      bf16x8_to_f32(kv, x);
+      const uint2 kc = quantize_row_piece(x, lanes_per_row, &ks);
+      bf16x8_to_f32(vv, x);
+      const uint2 vc = quantize_row_piece(x, lanes_per_row, &vs);
+      *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.k_pages) + dst) = kc;
+      *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(p.v_pages) + dst) = vc;
+      if (lc == 0) {
+        p.k_scales[slot] = ks;
+        p.v_scales[slot] = vs;
+      }
+    } else {
+      *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
+      *reinterpret_cast<uint4*>(p.v_pages + dst) = vv;
+    }
   }
 }
 
@@ -416,6 +435,9 @@ xkv_status select_compact(const xkv_dims* d, int layer, const int32_t* budget, i
   p.v = static_cast<const __nv_bfloat16*>(v);
   p.k_pages = static_cast<__nv_bfloat16*>(c->k_pages);
   p.v_pages = static_cast<__nv_bfloat16*>(c->v_pages);
+  p.k_scales = c->k_scales;
+  p.v_scales = c->v_scales;
+  p.kv_format = c->kv_format;
   p.total_tokens = total_tokens;
   p.stride_token = d->kv_stride_token;
   p.stride_head = d->kv_stride_head;

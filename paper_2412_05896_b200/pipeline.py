@@ -22,12 +22,14 @@ class XkvSession:
                  pool_kernel: int, lengths: list[int], pool_mode: int = xkv.POOL_MAX, page_size: int = 16,
                  max_new_tokens: int = 0, max_budget: int | None = None, total_budget: int | None = None,
                  curve_len: int | None = None, device="cuda:0", scale: float = 0.0,
-                 decode_chunk_rows: int = 0, n_lanes: int = 3, head_level: bool = False):
+                 decode_chunk_rows: int = 0, n_lanes: int = 3, head_level: bool = False,
+                 kv_format: int = xkv.KV_BF16):
         """head_level: budgets, cache lengths and page lists per (layer, sequence, KV head) instead of per (layer,
         sequence); total_budget and the solver's total then count prefix tokens over all heads of all layers, and
         max_budget bounds one head."""
         self.L, self.Hq, self.Hkv, self.d, self.W = n_layers, n_q_heads, n_kv_heads, head_dim, window
         self.head_level = bool(head_level)
+        self.kv_format = kv_format                 # xkv.KV_FP8_E4M3: the reduced caches hold 8-bit codes and row scales
         self.G = n_q_heads // n_kv_heads
         self.B = len(lengths)
         self.lengths = list(lengths)
@@ -96,8 +98,13 @@ class XkvSession:
             n_pages += math.ceil(rows / page_size)
         self.n_pages = max(n_pages, 1)
         bf16 = dict(dtype=torch.bfloat16, device=self.device)
-        self.k_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, **bf16)
-        self.v_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, **bf16)
+        page_dtype = torch.uint8 if kv_format == xkv.KV_FP8_E4M3 else torch.bfloat16
+        self.k_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, dtype=page_dtype, device=self.device)
+        self.v_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, dtype=page_dtype, device=self.device)
+        self.k_scales = self.v_scales = None
+        if kv_format == xkv.KV_FP8_E4M3:
+            self.k_scales = torch.zeros(self.n_pages, page_heads, page_size, **f32)
+            self.v_scales = torch.zeros(self.n_pages, page_heads, page_size, **f32)
         self.block_table = torch.zeros(n_layers, self.n_caches, self.max_pages_per_seq, dtype=torch.int32,
                                        device=self.device)
         # page runs of every (layer, cache): [0] first page, [1] number of pages; expanded on the device
@@ -108,7 +115,8 @@ class XkvSession:
         self.seq_lens = torch.zeros(n_layers, self.n_caches, dtype=torch.int32, device=self.device)
         self.cache = xkv.Cache(self.k_pages.data_ptr(), self.v_pages.data_ptr(), self.block_table.data_ptr(),
                                self.seq_lens.data_ptr(), n_layers, page_size, self.max_pages_per_seq,
-                               self.n_pages)
+                               self.n_pages, None if self.k_scales is None else self.k_scales.data_ptr(),
+                               None if self.v_scales is None else self.v_scales.data_ptr(), kv_format, 0)
         # decode sees the head-level caches as B*Hkv sequences of one KV head with G query heads each
         self.dec_dims = self.dims if not self.head_level else xkv.Dims(
             self.n_caches, self.G, 1, head_dim, window, pool_kernel, pool_mode, scale, head_dim, head_dim)

@@ -20,6 +20,7 @@ ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = -5, -6, -7
 POOL_MAX, POOL_AVG = 0, 1
 OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2, 3
 BUDGET_PER_LAYER, BUDGET_PER_SEQUENCE, BUDGET_PER_HEAD = 0, 1, 2
+KV_BF16, KV_FP8_E4M3 = 0, 1
 
 STATIC_SCRATCH_BYTES = 16 << 20
 
@@ -46,7 +47,9 @@ class Cache(ctypes.Structure):
     _fields_ = [("k_pages", ctypes.c_void_p), ("v_pages", ctypes.c_void_p),
                 ("block_table", ctypes.c_void_p), ("seq_lens", ctypes.c_void_p),
                 ("n_layers", ctypes.c_int32), ("page_size", ctypes.c_int32),
-                ("max_pages_per_seq", ctypes.c_int32), ("n_pages", ctypes.c_int32)]
+                ("max_pages_per_seq", ctypes.c_int32), ("n_pages", ctypes.c_int32),
+                ("k_scales", ctypes.c_void_p), ("v_scales", ctypes.c_void_p),
+                ("kv_format", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 _lib = None
