@@ -351,55 +351,26 @@ def decode_attention(q: np.ndarray, K_c: np.ndarray, V_c: np.ndarray,
 # A reduced cache stored with few bits (Sec. II-B: quantisation is compatible with eviction)
 # ----------------------------------------------------------------------------------------------
 # The paper names no format.  Reading taken here: every cached row (one token of one KV head, K and V separately)
-# is stored as 8-bit floating-point codes of the E4M3 kind (1 sign, 4 exponent bits with bias 7, 3 mantissa bits,
-# subnormals, no infinities, the all-ones pattern is NaN, largest finite value 448) times one fp32 scale per row,
-# scale = max|x| / 448 (1 for an all-zero row), code = nearest representable value of x / scale, ties to the even
-# mantissa.  Where floating point decides the code, the decision is taken in fp32 (the division by 448, the division
-# by the scale), which is the precision of the CUDA path.
-E4M3_MAX = 448.0
+# is stored as 8-bit integers times one fp32 scale per row: scale = max|x| / 127 (1 for an all-zero row),
+# q = x / scale rounded to the nearest integer, ties to even, kept within [-127, 127]; the stored byte is q + 128.
+# Where floating point decides the integer, the decision is taken in fp32 (the division by 127, the division by the
+# scale), which is the precision of the CUDA path.
+INT8_MAX = 127
 
 
-def e4m3_values() -> np.ndarray:
-    """Value of each of the 256 codes (NaN for the two all-ones patterns), from the format's definition."""
-    out = np.empty(256, dtype=np.float64)
-    for code in range(256):
-        sign = -1.0 if code & 0x80 else 1.0
-        e, m = (code >> 3) & 0xF, code & 0x7
-        if e == 0xF and m == 0x7:
-            out[code] = np.nan
-        elif e == 0:
-            out[code] = sign * (m / 8.0) * 2.0 ** -6            # subnormal
-        else:
-            out[code] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
-    return out
-
-
-def e4m3_encode(y: np.ndarray) -> np.ndarray:
-    """Nearest E4M3 code of every entry of y, ties to the even mantissa, magnitudes beyond 448 saturate."""
-    y = np.asarray(y, dtype=np.float64)
-    mags = e4m3_values()[:0x7F]                                 # codes 0x00..0x7E: the non-negative finite values, ascending
-    a = np.minimum(np.abs(y), E4M3_MAX)
-    hi = np.searchsorted(mags, a, side="left")                  # first code whose value is >= a
-    hi = np.minimum(hi, 0x7E)
-    lo = np.maximum(hi - 1, 0)
-    d_lo, d_hi = a - mags[lo], mags[hi] - a
-    pick_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))  # a tie goes to the code with an even last mantissa bit
-    code = np.where(pick_hi, hi, lo).astype(np.uint8)
-    return np.where(np.signbit(y), code | 0x80, code).astype(np.uint8)
-
-
-def quantize_rows_e4m3(X: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
-    """Rows of X [n, d] -> (codes uint8 [n, d], scales float32 [n])."""
+def quantize_rows_int8(X: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
+    """Rows of X [n, d] -> (stored bytes uint8 [n, d] = q + 128, scales float32 [n])."""
     X32 = np.asarray(X, dtype=np.float32)
     amax = np.max(np.abs(X32), axis=1) if X32.shape[0] else np.zeros(0, dtype=np.float32)
-    scales = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    scales = np.where(amax > 0, amax / np.float32(INT8_MAX), np.float32(1.0)).astype(np.float32)
     y = (X32 / scales[:, None]).astype(np.float32)              # fp32 division, as on the GPU
-    return e4m3_encode(y.astype(np.float64)), scales
+    q = np.clip(np.rint(y.astype(np.float64)), -INT8_MAX, INT8_MAX).astype(np.int64)   # rint: ties to even
+    return (q + 128).astype(np.uint8), scales
 
 
-def dequantize_rows_e4m3(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
-    """What the computation recovers from a stored row: value of the code times the row's scale (float64)."""
-    return e4m3_values()[np.asarray(codes, dtype=np.uint8)] * np.asarray(scales, dtype=np.float64)[:, None]
+def dequantize_rows_int8(stored: np.ndarray, scales: np.ndarray) -> np.ndarray:
+    """What the computation recovers from a stored row: (byte - 128) times the row's scale (float64)."""
+    return (np.asarray(stored, dtype=np.int64) - 128).astype(np.float64) * np.asarray(scales, dtype=np.float64)[:, None]
 
 
 # ----------------------------------------------------------------------------------------------

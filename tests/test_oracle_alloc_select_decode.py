@@ -242,53 +242,48 @@ def test_decode_split_and_lse_merge_is_invariant(splits):
 
 
 # ------------------------------------------------------------------ 8-bit rows of a reduced cache (Sec. II-B)
-def test_e4m3_codes_by_hand_and_format_properties():
-    v = O.e4m3_values()
-    by_hand = {0x00: 0.0, 0x01: 2.0 ** -9, 0x07: 7 * 2.0 ** -9, 0x08: 2.0 ** -6, 0x0F: 1.875 * 2.0 ** -6, 0x38: 1.0,
-               0x39: 1.125, 0x3C: 1.5, 0x40: 2.0, 0x77: 1.875 * 128, 0x78: 256.0, 0x7E: 448.0, 0xB8: -1.0, 0xFE: -448.0}
-    for code, val in by_hand.items():
-        assert v[code] == val, hex(code)
-    assert np.isnan(v[0x7F]) and np.isnan(v[0xFF]) and np.signbit(v[0x80]) and v[0x80] == 0.0
-    pos = v[:0x7F]
-    assert np.all(np.diff(pos) > 0) and np.all(v[0x80:0xFF] == -pos)                 # ascending, sign-symmetric
-    # every representable value encodes to itself; midpoints go to the even mantissa; beyond 448 saturates
-    assert np.array_equal(O.e4m3_encode(pos), np.arange(0x7F, dtype=np.uint8))
-    assert np.array_equal(O.e4m3_encode(-pos[1:]), np.arange(1, 0x7F, dtype=np.uint8) | 0x80)
-    mid = (pos[:-1] + pos[1:]) / 2
-    want = np.where(np.arange(0x7E) % 2 == 0, np.arange(0x7E), np.arange(0x7E) + 1)
-    assert np.array_equal(O.e4m3_encode(mid), want.astype(np.uint8))
-    assert O.e4m3_encode(np.array([1.0625, 1.1875, 1.07, 500.0, -1e9, 2.0 ** -10, 2.0 ** -10 * 1.01])).tolist() == \
-        [0x38, 0x3A, 0x39, 0x7E, 0xFE, 0x00, 0x01]
+def test_int8_rows_by_hand():
+    # one row whose largest entry is 127 so that the scale is exactly 1: the integers are the rounded entries,
+    # halves go to the even neighbour, the stored byte is the integer plus 128
+    x = np.array([[127.0, -127.0, 0.0, 0.5, 1.5, 2.5, -0.5, -1.5, 3.49, 3.51, -126.5, 100.25]])
+    stored, scales = O.quantize_rows_int8(x)
+    assert scales.tolist() == [1.0]
+    assert (stored.astype(int) - 128).tolist() == [[127, -127, 0, 0, 2, 2, 0, -2, 3, 4, -126, 100]]
+    assert np.array_equal(O.dequantize_rows_int8(stored, scales), (stored.astype(np.float64) - 128))
+    # scale = max|x| / 127 in fp32; the largest entry maps to +-127 exactly; an all-zero row keeps scale 1
+    y = np.array([[0.25, -2.0, 1.0], [0.0, 0.0, 0.0], [3.0, 0.0, -0.01]])
+    st, sc = O.quantize_rows_int8(y)
+    assert sc.dtype == np.float32 and st.dtype == np.uint8
+    assert sc[0] == np.float32(2.0) / np.float32(127) and sc[1] == 1.0 and sc[2] == np.float32(3.0) / np.float32(127)
+    assert (st.astype(int) - 128)[:, :2].tolist() == [[16, -127], [0, 0], [127, 0]]        # 0.25 * 63.5 = 15.875 -> 16
+    assert (st.astype(int) - 128)[1:, 2].tolist() == [0, 0]
 
 
 def test_quantized_rows_scale_round_trip_and_error_bound():
     rng = np.random.default_rng(50)
     X = torch.from_numpy(rng.standard_normal((40, 128)) * rng.uniform(0.01, 30, (40, 1))).to(torch.bfloat16)
     X = X.float().numpy().astype(np.float64)
-    X[3] = 0.0                                                  # an all-zero row keeps scale 1 and codes 0
+    X[3] = 0.0
     X[5, :] = 0.0
-    X[5, 17] = -3.0                                             # a one-hot row: its entry becomes -448 * scale exactly
-    codes, scales = O.quantize_rows_e4m3(X)
-    assert codes.dtype == np.uint8 and scales.dtype == np.float32
-    assert scales[3] == 1.0 and np.all(codes[3] == 0)
-    assert codes[5, 17] == 0xFE and np.all(np.delete(codes[5], 17) == 0)
-    back = O.dequantize_rows_e4m3(codes, scales)
-    assert back[5, 17] == -448.0 * float(scales[5]) and abs(back[5, 17] + 3.0) < 1e-6
+    X[5, 17] = -3.0                                             # a one-hot row: its entry becomes -127 * scale
+    stored, scales = O.quantize_rows_int8(X)
+    assert scales[3] == 1.0 and np.all(stored[3] == 128)
+    assert stored[5, 17] == 1 and np.all(np.delete(stored[5], 17) == 128)
+    back = O.dequantize_rows_int8(stored, scales)
+    assert abs(back[5, 17] + 3.0) < 1e-6
     amax = np.abs(X).max(axis=1)
     nz = amax > 0
-    assert np.allclose(scales[nz], amax[nz] / 448.0, rtol=1e-7)
-    # the largest entry of every row takes the largest code; the error is half a step of a 3-bit mantissa for normal
-    # codes (relative 2^-4) and half a subnormal step (2^-10 of the scale) below them; one more fp32 rounding on top
-    assert np.all(np.max(codes & 0x7F, axis=1)[nz] == 0x7E)
-    err = np.abs(back - X)
-    bound = np.maximum(np.abs(X) * 2.0 ** -4, scales[:, None].astype(np.float64) * 2.0 ** -10) * (1 + 1e-6)
-    assert np.all(err <= bound)
-    # stored rows are a fixed point: quantising what was recovered gives the same codes and scales
-    codes2, scales2 = O.quantize_rows_e4m3(back)
-    assert np.array_equal(codes2, codes) and np.array_equal(scales2, scales)
-    # attention over the recovered rows moves with the quantisation error only: a coarse sanity bound
-    q = rng.standard_normal(128)
-    V = rng.standard_normal((40, 128))
-    z_ref, _ = O.decode_attention(q, X, V)
-    z_q, _ = O.decode_attention(q, back, V)
-    assert np.max(np.abs(z_ref - z_q)) < 0.5
+    assert np.allclose(scales[nz], amax[nz] / 127.0, rtol=1e-7)
+    assert np.all(np.abs(stored.astype(int) - 128).max(axis=1)[nz] == 127) and stored.min() >= 1
+    # the error is half a step of the row's grid (plus the fp32 roundings of scale and quotient)
+    assert np.all(np.abs(back - X) <= 0.5 * scales[:, None].astype(np.float64) * (1 + 1e-5))
+    # stored rows are a fixed point: quantising what was recovered gives the same bytes and scales
+    stored2, scales2 = O.quantize_rows_int8(back)
+    assert np.array_equal(stored2, stored) and np.array_equal(scales2, scales)
+    # brute force on a small row: the nearest grid point, ties to the even integer
+    row = X[7:8, :16]
+    st, sc = O.quantize_rows_int8(row)
+    for j in range(16):
+        y = float(np.float32(row[0, j]) / sc[0])
+        cands = sorted(range(-127, 128), key=lambda n: (abs(n - y), n % 2))
+        assert int(st[0, j]) - 128 == cands[0]
