@@ -476,6 +476,45 @@ def run_workload(ctx: Ctx, name: str, steps: int, warmup: int, headline: bool) -
         del lse_all, q_full, o_full, lse_list
         torch.cuda.empty_cache()
 
+    # ---------------------------------------------------------------- decode over caches stored in 8 bits
+    # The same budgets, the kept rows stored as 8-bit integers with a scale per row (Sec. II-B: quantisation is compatible
+    # with eviction): the second bandwidth lever.  Outside the timed region of the headline number.
+    if world == 1 and not args.no_q8:
+        q8 = ctx.XkvSession(L, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
+                            max_new_tokens=n_dec, max_budget=w.n_max or None, total_budget=N_total,
+                            curve_len=w.n_max or None, device=dev, decode_chunk_rows=args.chunk_rows,
+                            kv_format=xkv.KV_INT8)
+        q8.scores, q8.sorted = sess.scores, sess.sorted            # the scores of the last scoring pass
+        q8._layer_stride = sess._layer_stride
+        q8.assign_pages(budgets)
+        q8.select_layers(budgets, k, v)
+        n_q8 = min(n_dec, 48)
+        qs = [ev() for _ in range(n_q8)]
+        qe = [ev() for _ in range(n_q8)]
+        for e in qs + qe:
+            e.record()
+        for s_ in range(n_q8):
+            q, kn, vn = dec[s_ % n_distinct]
+            xkv.profile_events(qs[s_], qe[s_])
+            q8.decode(q, kn, vn)
+        xkv.profile_events(None, None)
+        torch.cuda.synchronize()
+        for which in ("select", "decode"):
+            if q8.device_status(which) != xkv.OK:
+                raise SystemExit(f"{name}: 8-bit cache {which} reported a device error")
+        q8_ms = float(np.mean([a.elapsed_time(b) for a, b in zip(qs, qe)][2:]))
+        rows = float(np.mean(dbytes[2:n_q8])) / (2 * d * 2)           # cached rows (all layers, sequences, KV heads) per step
+        q8_bytes = rows * (2 * d + 8)                                   # K and V bytes plus two fp32 scales per row
+        bf16_ms = float(kern_ms[:, 2:n_q8].mean())
+        rec["quantized_cache_decode"] = {
+            "format": "8-bit integers with one fp32 scale per cached row, K and V",
+            "steps_measured": n_q8 - 2, "avg_launch_ms": q8_ms, "stored_bytes_per_launch": q8_bytes,
+            "achieved_GBps_of_stored_bytes": q8_bytes / (q8_ms * 1e-3) / 1e9,
+            "frac_of_measured_hbm": q8_bytes / (q8_ms * 1e-3) / 1e9 / peak,
+            "bf16_launch_ms_same_steps": bf16_ms, "speedup_over_bf16_cache": bf16_ms / q8_ms}
+        del q8
+        torch.cuda.empty_cache()
+
     # ---------------------------------------------------------------- full-cache decode, for comparison only
     if world == 1 and not args.no_full_cache and (headline or name == "llama3_8b_long" or args.full_cache_all):
         per_layer = sum(-(-(t + n_dec + sess.page_size) // sess.page_size) * sess.page_size for t in lengths) \
@@ -727,6 +766,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workloads' decode steps")
     ap.add_argument("--no-prefill-attn", action="store_true",
                     help="skip the prefill attention and the scoring from its normalisers")
+    ap.add_argument("--no-q8", action="store_true", help="skip the decode over caches stored in 8 bits")
     ap.add_argument("--no-full-cache", action="store_true", help="skip the uncompressed-cache decode comparison")
     ap.add_argument("--full-cache-all", action="store_true", help="uncompressed-cache comparison for every workload")
     ap.add_argument("--lanes", type=int, default=None, help="side streams of the scoring and eviction phases")
@@ -774,6 +814,7 @@ def main():
         "timed_region_ms": head["timed_region_ms"],
         "full_cache_decode": head.get("full_cache_decode"),
         "prefill_attn": head.get("prefill_attn"), "score_from_prefill_lse": head.get("score_from_prefill_lse"),
+        "quantized_cache_decode": head.get("quantized_cache_decode"),
         "roofline": head["roofline"], "cpu_baseline": extras.get("cpu_baseline"), "e2e": extras.get("e2e"),
         "parity": extras.get("parity"),
         "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],

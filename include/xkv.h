@@ -68,8 +68,8 @@ typedef int32_t xkv_status;
 #define XKV_BUDGET_PER_SEQUENCE 1 /* [B]: one count per sequence (the paper's offline mode, one list per task) */
 #define XKV_BUDGET_PER_HEAD     2 /* [B][Hkv]: head-level budgets inside the layer (Sec. II-C)                 */
 
-#define XKV_KV_BF16     0
-#define XKV_KV_FP8_E4M3 1
+#define XKV_KV_BF16 0
+#define XKV_KV_INT8 1
 
 #define XKV_OP_SCORE          0
 #define XKV_OP_SELECT_COMPACT 1
@@ -101,15 +101,14 @@ typedef struct xkv_dims {
  * page_size is a multiple of 16 (at most 256).
  *
  * A cache stored with few bits (Sec. II-B: quantisation is compatible with eviction; the paper names no format, this
- * one is the library's): with kv_format = XKV_KV_FP8_E4M3 the pages hold one byte per element,
- *   k_pages / v_pages : dev uint8 [n_pages][Hkv][page_size][d], 8-bit floating-point codes (1 sign bit, 4 exponent
- *                       bits with bias 7, 3 mantissa bits, subnormals, no infinities, largest finite value 448)
+ * one is the library's): with kv_format = XKV_KV_INT8 the pages hold one byte per element,
+ *   k_pages / v_pages : dev uint8 [n_pages][Hkv][page_size][d], the byte is q + 128 with q an integer in [-127, 127]
  *   k_scales / v_scales : dev fp32 [n_pages][Hkv][page_size]
- * and a cached row stands for code value * scale with scale = max|x| / 448 over the row (1 for an all-zero row) and
- * code = the representable value nearest to x / scale (ties to the even mantissa), both divisions in fp32.
+ * and a cached row stands for q * scale with scale = max|x| / 127 over the row (1 for an all-zero row) and
+ * q = x / scale rounded to the nearest integer (ties to even), both divisions in fp32.
  * xkv_select_compact and the append of xkv_decode_attn store rows that way; xkv_decode_attn multiplies the scales back
- * in (K: on the logits, V: on the weights) and computes in fp16 x fp16 -> fp32: query and weight magnitudes must stay
- * below 65504 (for the weights: max|v| of a row below about 1e5). head_dim 64 and 128.
+ * in (K: on the logits, V: on the weights) and computes in fp16 x fp16 -> fp32: query magnitudes must stay below
+ * 65504, and so must 256 * max|v| / 127 of a row. head_dim 64 and 128.
  *
  * Head-level budgets (XKV_BUDGET_PER_HEAD) give every KV head of a sequence a cache of its own length. The same
  * structure then describes B*Hkv caches of one KV head each per layer:
@@ -129,9 +128,9 @@ typedef struct xkv_cache {
   int32_t  page_size;
   int32_t  max_pages_per_seq;
   int32_t  n_pages;
-  float*   k_scales;   /* XKV_KV_FP8_E4M3 only: dev fp32 [n_pages][Hkv][page_size], one scale per cached row */
+  float*   k_scales;   /* XKV_KV_INT8 only: dev fp32 [n_pages][Hkv][page_size], one scale per cached row */
   float*   v_scales;
-  int32_t  kv_format;  /* XKV_KV_BF16 (0) or XKV_KV_FP8_E4M3 */
+  int32_t  kv_format;  /* XKV_KV_BF16 (0) or XKV_KV_INT8 */
   int32_t  reserved;   /* 0 */
 } xkv_cache;
 

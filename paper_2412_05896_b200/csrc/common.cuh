@@ -67,25 +67,18 @@ __device__ __forceinline__ float fast_exp2(float x) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Cache rows stored as 8-bit floating-point codes (1-4-3, bias 7, largest finite value 448) with one fp32 scale
-// per row: scale = max|x| / 448 (1 for an all-zero row), code = nearest value to x / scale, ties to even; both
-// divisions are IEEE fp32 divisions, so that the codes are the same wherever they are computed.
+// Cache rows stored as 8-bit integers with one fp32 scale per row: scale = max|x| / 127 (1 for an all-zero row),
+// q = x / scale rounded to nearest, ties to even, within [-127, 127]; the stored byte is q + 128.  Both divisions are
+// IEEE fp32 divisions, so that the bytes are the same wherever they are computed.
 // ---------------------------------------------------------------------------------------------
-// Two fp32 -> two codes; `lo` lands in the low byte.
-__device__ __forceinline__ uint16_t f32x2_to_e4m3x2(float lo, float hi) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-// Two codes -> two fp16 (exact); the low byte lands in the low half.
-__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
-  uint32_t r;
-  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
-  return r;
+__device__ __forceinline__ uint32_t int8_stored_byte(float x, float scale) {
+  int q = __float2int_rn(__fdiv_rn(x, scale));
+  q = max(-127, min(127, q));
+  return (uint32_t)(q + 128);
 }
 // Quantises one row spread over consecutive lanes of a warp, eight consecutive elements per lane (x = this lane's
 // elements as fp32, group = D / 8 lanes per row, a power of two, rows aligned to multiples of `group` lanes; every lane
-// of the row must be here).  Returns the lane's eight codes; *scale is the row's scale in every lane of the row.
+// of the row must be here).  Returns the lane's eight stored bytes; *scale is the row's scale in every lane of the row.
 __device__ __forceinline__ uint2 quantize_row_piece(const float (&x)[8], int group, float* scale) {
   const unsigned lane = threadIdx.x & 31u;
   const unsigned mask = (group >= 32 ? 0xffffffffu : ((1u << group) - 1u)) << (lane & ~(unsigned)(group - 1));
@@ -93,14 +86,27 @@ __device__ __forceinline__ uint2 quantize_row_piece(const float (&x)[8], int gro
 #pragma unroll
   for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(x[i]));
   for (int o = 1; o < group; o <<= 1) amax = fmaxf(amax, __shfl_xor_sync(mask, amax, o));
-  const float s = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+  const float s = amax > 0.f ? __fdiv_rn(amax, 127.f) : 1.f;
   *scale = s;
   uint2 out;
-  out.x = (uint32_t)f32x2_to_e4m3x2(__fdiv_rn(x[0], s), __fdiv_rn(x[1], s)) |
-          ((uint32_t)f32x2_to_e4m3x2(__fdiv_rn(x[2], s), __fdiv_rn(x[3], s)) << 16);
-  out.y = (uint32_t)f32x2_to_e4m3x2(__fdiv_rn(x[4], s), __fdiv_rn(x[5], s)) |
-          ((uint32_t)f32x2_to_e4m3x2(__fdiv_rn(x[6], s), __fdiv_rn(x[7], s)) << 16);
+  out.x = int8_stored_byte(x[0], s) | (int8_stored_byte(x[1], s) << 8) | (int8_stored_byte(x[2], s) << 16) |
+          (int8_stored_byte(x[3], s) << 24);
+  out.y = int8_stored_byte(x[4], s) | (int8_stored_byte(x[5], s) << 8) | (int8_stored_byte(x[6], s) << 16) |
+          (int8_stored_byte(x[7], s) << 24);
   return out;
+}
+// Two stored bytes of a 32-bit word -> two fp16 integers (exact).  kSelector picks the bytes (a prmt selector whose
+// odd result bytes take the constant 0x64): 0x64nn read as fp16 is 1024 + nn, and 1024 + 128 is subtracted.
+template <uint32_t kSelector>
+__device__ __forceinline__ uint32_t int8x2_to_f16x2(uint32_t word) {
+  uint32_t r;
+  asm("{\n\t.reg .b32 t, c;\n\t"
+      "prmt.b32 t, %1, 0x64646464, %2;\n\t"
+      "mov.b32 c, 0x64806480;\n\t"
+      "sub.f16x2 %0, t, c;\n\t}"
+      : "=r"(r)
+      : "r"(word), "n"(kSelector));
+  return r;
 }
 // The eight bf16 of a 16-byte piece as fp32.
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&x)[8]) {

@@ -73,8 +73,8 @@ xkv_status check_cache(const xkv_cache* c, const xkv_dims* d) {
   if (c->n_layers <= 0 || c->max_pages_per_seq <= 0 || c->n_pages <= 0) return XKV_ERR_INVALID_ARG;
   if (c->page_size <= 0 || c->page_size % 16 != 0 || c->page_size > 256) return XKV_ERR_INVALID_ARG;
   if ((int64_t)c->max_pages_per_seq * c->page_size > (1 << 30)) return XKV_ERR_INVALID_ARG;
-  if (c->kv_format != XKV_KV_BF16 && c->kv_format != XKV_KV_FP8_E4M3) return XKV_ERR_INVALID_ARG;
-  if (c->kv_format == XKV_KV_FP8_E4M3 &&
+  if (c->kv_format != XKV_KV_BF16 && c->kv_format != XKV_KV_INT8) return XKV_ERR_INVALID_ARG;
+  if (c->kv_format == XKV_KV_INT8 &&
       (c->k_scales == nullptr || c->v_scales == nullptr || !aligned16(c->k_scales) || !aligned16(c->v_scales)))
     return XKV_ERR_INVALID_ARG;
   (void)d;

@@ -50,7 +50,6 @@ namespace {
 constexpr int kTileRows = 16;        // cache rows per pipeline stage = one TMA box; page_size is a multiple
 constexpr int kChunkAlign = 64;      // chunk_rows granularity
 constexpr int kAttnWarps = 8;
-constexpr int kAttnThreads = kAttnWarps * 32;
 constexpr int kTargetItems = 12 * 148 * kAttnWarps;  // auto chunking aims at about this many extra work items (a dozen per warp keeps the tail short)
 constexpr int kMinChunkRows = 256;
 constexpr int kMaxGroup = 8;
@@ -86,22 +85,28 @@ struct DecodeParams {
   float* part_ml;     // [max_items][G][2]
 };
 
-// Q8: the cache holds 8-bit codes and per-row scales.  A stage of the ring is then the raw tile as it lies in the
-// pages (K codes, V codes, K scales, V scales); the warp expands K and V into two 16-bit tiles of its own, in the same
-// swizzled layout a 16-bit TMA box has, and the rest of the tile's work reads those.
+// Q8: the cache holds 8-bit integers and per-row scales.  The ring then holds the raw tiles as they lie in the pages:
+// all K tiles first (each 1024-byte aligned, 128-byte swizzled when a row is 128 bytes), then the V tiles, then the
+// scales of the K rows and of the V rows; the tensor-core fragments are formed from the bytes in registers.
 template <int D, bool Q8>
 struct Cfg {
   static constexpr int kHalves = D / 64;                       // 128-byte swizzled column halves
   static constexpr int kBoxBytes = kTileRows * 128;            // one half of a 16-bit K or V tile (one TMA box)
   static constexpr int kTileBytes = kHalves * kBoxBytes;
-  static constexpr int kRawTileBytes = kTileRows * D;          // Q8: one tile of codes
+  static constexpr int kRawTileBytes = kTileRows * D;          // Q8: one tile of stored bytes
   static constexpr int kScaleBytes = kTileRows * 4;            // Q8: the scales of a tile's rows
   static constexpr int kStageBytes = Q8 ? 2 * kRawTileBytes + 2 * kScaleBytes : 2 * kTileBytes;   // K tile + V tile
-  static constexpr int kStages = Q8 ? ((D == 128) ? 4 : 8) : ((D == 128) ? 3 : 6);
-  static constexpr int kExpandBytes = Q8 ? 2 * kTileBytes : 0; // Q8: the expanded K tile and V tile
-  static constexpr int kRingBytes = kStages * kStageBytes + kExpandBytes;     // per warp
-  static constexpr int kSmemBytes = 1024 + kAttnWarps * kRingBytes + kAttnWarps * kStages * 8 +
-                                    kAttnWarps * kFifo * 20 + (kMaxPlanUnits + 1) * 4 + kMaxPlanUnits * 2 + 64;
+  // The 8-bit path has twice the work per byte (the fragments are formed in registers) and half the bytes per
+  // tile: sixteen warps with rings of as many tiles keep as many bytes in flight and hide twice the instruction latency.
+  static constexpr int kWarps = Q8 ? 2 * kAttnWarps : kAttnWarps;
+  static constexpr int kThreads = kWarps * 32;
+  static constexpr int kStages = (D == 128) ? 3 : 6;
+  static constexpr int kRingBytes = (kStages * kStageBytes + 1023) / 1024 * 1024;     // per warp
+  static constexpr int kSmemBytes = 1024 + kWarps * kRingBytes + kWarps * kStages * 8 +
+                                    kWarps * kFifo * 20 + (kMaxPlanUnits + 1) * 4 + kMaxPlanUnits * 2 + 64;
+  // Q8 ring layout
+  static constexpr int kRawVOff = kStages * kRawTileBytes;
+  static constexpr int kScaleOff = 2 * kStages * kRawTileBytes;
 };
 
 // fp16 tensor-core tile for the 8-bit caches (the codes are exact in fp16).
@@ -294,7 +299,7 @@ __global__ void __launch_bounds__(kPrepThreads) decode_prepare_kernel(DecodePara
 
 // ---------------------------------------------------------------------------------------------
 template <int D, bool Q8>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __launch_bounds__((Cfg<D, Q8>::kThreads), 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                    const DecodeParams p) {
   using C = Cfg<D, Q8>;
@@ -302,21 +307,25 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint8_t* ring = smem + (size_t)warp * C::kRingBytes;
-  uint8_t* k_exp = ring + (size_t)C::kStages * C::kStageBytes;   // Q8: this warp's expanded K tile, then its V tile
-  uint8_t* v_exp = k_exp + C::kTileBytes;
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes) + warp * C::kStages;
-  uint8_t* fifo_base = smem + (size_t)kAttnWarps * C::kRingBytes + kAttnWarps * C::kStages * 8;
+  // Q8: where stage s keeps its K bytes, V bytes and the two scale vectors
+  auto raw_k = [&](uint32_t s) -> uint8_t* { return ring + (size_t)s * C::kRawTileBytes; };
+  auto raw_v = [&](uint32_t s) -> uint8_t* { return ring + C::kRawVOff + (size_t)s * C::kRawTileBytes; };
+  auto raw_scales = [&](uint32_t s) -> float* {       // [0..15] K rows, [16..31] V rows
+    return reinterpret_cast<float*>(ring + C::kScaleOff + (size_t)s * 2 * C::kScaleBytes);
+  };
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + (size_t)C::kWarps * C::kRingBytes) + warp * C::kStages;
+  uint8_t* fifo_base = smem + (size_t)C::kWarps * C::kRingBytes + C::kWarps * C::kStages * 8;
   int4* fifo = reinterpret_cast<int4*>(fifo_base) + warp * kFifo;                        // item descriptors
-  int* fifo_idx = reinterpret_cast<int*>(fifo_base + kAttnWarps * kFifo * 16) + warp * kFifo;   // and their indices
-  int* s_excl = reinterpret_cast<int*>(fifo_base + kAttnWarps * kFifo * 20);   // [units + 1] chunks before each unit
+  int* fifo_idx = reinterpret_cast<int*>(fifo_base + C::kWarps * kFifo * 16) + warp * kFifo;   // and their indices
+  int* s_excl = reinterpret_cast<int*>(fifo_base + C::kWarps * kFifo * 20);   // [units + 1] chunks before each unit
   uint16_t* s_multi = reinterpret_cast<uint16_t*>(s_excl + kMaxPlanUnits + 1);  // units cut into several chunks
   __shared__ int s_plan[4];                                                     // chunk rows, split units, page scratch
-  __shared__ int s_scan[2 * kAttnWarps];
-  __shared__ long long s_rows[kAttnWarps];
+  __shared__ int s_scan[2 * C::kWarps];
+  __shared__ long long s_rows[C::kWarps];
 
   if (tid == 0) {
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnWarps * C::kRingBytes);
-    for (int s = 0; s < kAttnWarps * C::kStages; ++s) mbar_init(&bars[s], 1);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)C::kWarps * C::kRingBytes);
+    for (int s = 0; s < C::kWarps * C::kStages; ++s) mbar_init(&bars[s], 1);
     fence_mbar_init();
     prefetch_tmap(&tmap_k);
     prefetch_tmap(&tmap_v);
@@ -338,7 +347,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     // ---- prologue of the self-planning launch
     // the plan, computed by every CTA for itself: chunk size from the total length, then the number of chunks
     // before each unit (and the list of units with more than one)
-    constexpr int kPer = kMaxPlanUnits / kAttnThreads;
+    constexpr int kPer = kMaxPlanUnits / C::kThreads;
     int nloc[kPer];
     long long rows = 0;
 #pragma unroll
@@ -353,7 +362,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     __syncthreads();
     long long total = 0;
 #pragma unroll
-    for (int w8 = 0; w8 < kAttnWarps; ++w8) total += s_rows[w8];
+    for (int w8 = 0; w8 < C::kWarps; ++w8) total += s_rows[w8];
     const int chunk = choose_chunk(total * p.n_kv_heads, p.chunk_rows_forced);
     int cnt = 0, mcnt = 0;
 #pragma unroll
@@ -375,18 +384,18 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     }
     if (lane == 31) {
       s_scan[warp] = icnt;
-      s_scan[kAttnWarps + warp] = imcnt;
+      s_scan[C::kWarps + warp] = imcnt;
     }
     __syncthreads();
     int base = icnt - cnt, mbase = imcnt - mcnt, all = 0, mall = 0;
 #pragma unroll
-    for (int w8 = 0; w8 < kAttnWarps; ++w8) {
+    for (int w8 = 0; w8 < C::kWarps; ++w8) {
       if (w8 < warp) {
         base += s_scan[w8];
-        mbase += s_scan[kAttnWarps + w8];
+        mbase += s_scan[C::kWarps + w8];
       }
       all += s_scan[w8];
-      mall += s_scan[kAttnWarps + w8];
+      mall += s_scan[C::kWarps + w8];
     }
 #pragma unroll
     for (int i = 0; i < kPer; ++i) {
@@ -491,12 +500,11 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         uint8_t* ks = ring + (size_t)s * C::kStageBytes;
         mbar_arrive_expect_tx(&full_bar[s], kTxBytes);
         if constexpr (Q8) {
-          // raw codes of the 16 rows (one box of D bytes per row) and their scales (16 consecutive floats)
-          uint8_t* vs = ks + C::kRawTileBytes;
-          tma_load_2d(ks, &tmap_k, 0, grow, &full_bar[s]);
-          tma_load_2d(vs, &tmap_v, 0, grow, &full_bar[s]);
-          bulk_copy_g2s(vs + C::kRawTileBytes, p.k_scales + grow, C::kScaleBytes, &full_bar[s]);
-          bulk_copy_g2s(vs + C::kRawTileBytes + C::kScaleBytes, p.v_scales + grow, C::kScaleBytes, &full_bar[s]);
+          // stored bytes of the 16 rows (one box of D bytes per row) and their scales (16 consecutive floats)
+          tma_load_2d(raw_k(s), &tmap_k, 0, grow, &full_bar[s]);
+          tma_load_2d(raw_v(s), &tmap_v, 0, grow, &full_bar[s]);
+          bulk_copy_g2s(raw_scales(s), p.k_scales + grow, C::kScaleBytes, &full_bar[s]);
+          bulk_copy_g2s(raw_scales(s) + kTileRows, p.v_scales + grow, C::kScaleBytes, &full_bar[s]);
         } else {
           uint8_t* vs = ks + C::kTileBytes;
 #pragma unroll
@@ -560,9 +568,12 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const __nv_bfloat16* qp = p.q + (q_row0 + gid) * D + 16 * ks + 2 * tig;
         qb[ks][0] = *reinterpret_cast<const uint32_t*>(qp);
         qb[ks][1] = *reinterpret_cast<const uint32_t*>(qp + 8);
-        if constexpr (Q8) {           // the 8-bit path multiplies in fp16
-          qb[ks][0] = pack_f16(bf16_lo(qb[ks][0]), bf16_hi(qb[ks][0]));
-          qb[ks][1] = pack_f16(bf16_lo(qb[ks][1]), bf16_hi(qb[ks][1]));
+        if constexpr (Q8) {
+          // The 8-bit path multiplies in fp16, and a lane's K fragment of this k-step holds the four consecutive
+          // columns 16*ks + 4*tig .. + 3 (two registers of two): the query columns follow that order.
+          const uint2 four = *reinterpret_cast<const uint2*>(p.q + (q_row0 + gid) * D + 16 * ks + 4 * tig);
+          qb[ks][0] = pack_f16(bf16_lo(four.x), bf16_hi(four.x));
+          qb[ks][1] = pack_f16(bf16_lo(four.y), bf16_hi(four.y));
         }
       }
     }
@@ -573,43 +584,38 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     float l_part[2] = {0.f, 0.f};
 
     // S^T of one 16-row tile: rows gid (regs 0,1) and gid + 8 (regs 2,3), heads 2*tig, 2*tig + 1
-    // Q8: expands a tile of codes (16 rows of D bytes, rows contiguous) into the warp's 16-bit tile: rows of 128 bytes
-    // per 64 columns, 16-byte pieces at their swizzled places, exactly what a 16-bit TMA box would have written.
-    auto expand_tile = [&](const uint8_t* raw, uint8_t* dst) {
-      constexpr int kPieces = kTileRows * D / 16;               // 16-code pieces of the tile
-#pragma unroll
-      for (int i = 0; i < kPieces / 32; ++i) {
-        const int q = lane + 32 * i;
-        const int r = q / (D / 16), c16 = q % (D / 16);         // row, 16-code piece of the row
-        const uint4 w = *reinterpret_cast<const uint4*>(raw + q * 16);
-        uint4 lo, hi;
-        lo.x = e4m3x2_to_f16x2((uint16_t)(w.x & 0xffffu)); lo.y = e4m3x2_to_f16x2((uint16_t)(w.x >> 16));
-        lo.z = e4m3x2_to_f16x2((uint16_t)(w.y & 0xffffu)); lo.w = e4m3x2_to_f16x2((uint16_t)(w.y >> 16));
-        hi.x = e4m3x2_to_f16x2((uint16_t)(w.z & 0xffffu)); hi.y = e4m3x2_to_f16x2((uint16_t)(w.z >> 16));
-        hi.z = e4m3x2_to_f16x2((uint16_t)(w.w & 0xffffu)); hi.w = e4m3x2_to_f16x2((uint16_t)(w.w >> 16));
-        const int c = (2 * c16) & 7;                            // first of the two 8-element pieces, within its half
-        uint8_t* row = dst + ((2 * c16) >> 3) * C::kBoxBytes + r * 128;
-        *reinterpret_cast<uint4*>(row + ((c ^ (r & 7)) << 4)) = lo;
-        *reinterpret_cast<uint4*>(row + (((c + 1) ^ (r & 7)) << 4)) = hi;
-      }
-      __syncwarp();
+    // Q8: address this lane hands to ldmatrix for row `row` (0..15) and 16-byte piece `piece` of a raw tile (rows of D
+    // bytes; pieces at their swizzled places when a row is the 128 bytes of the swizzle span)
+    auto raw_piece = [&](uint32_t tile_base, int row, int piece) -> uint32_t {
+      return D == 128 ? tile_base + row * 128 + ((piece ^ (row & 7)) << 4) : tile_base + row * D + (piece << 4);
     };
     auto qk_tile = [&](uint32_t idx, float (&acc)[4]) {
-      uint8_t* stage = ring + (size_t)(idx % C::kStages) * C::kStageBytes;
-      uint32_t ks_base = smem_u32(stage);
-      if constexpr (Q8) {
-        expand_tile(stage, k_exp);
-        ks_base = smem_u32(k_exp);
-      }
+      const uint32_t s = idx % C::kStages;
       float a0[4] = {0.f, 0.f, 0.f, 0.f}, a1[4] = {0.f, 0.f, 0.f, 0.f};
+      if constexpr (Q8) {
+        // One ldmatrix.x4 covers two k-steps: matrices (rows 0-7 | 8-15) x (piece 2j | 2j+1); a lane then holds, per
+        // matrix, the four consecutive bytes 4*tig .. of row gid: columns 0, 1 feed the fragment's first k pair and
+        // columns 2, 3 its second one (the query fragment is loaded in the same column order).
+        const uint32_t kt = smem_u32(raw_k(s));
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        uint32_t af[4];
-        ldmatrix_x4(af, ks_base + (ks >> 2) * C::kBoxBytes + (k_lane_off ^ (uint32_t)(((2 * ks) & 7) << 4)));
-        if constexpr (Q8) {
-          if (ks & 1) mma_f16_16816(a1, af, qb[ks][0], qb[ks][1]);
-          else        mma_f16_16816(a0, af, qb[ks][0], qb[ks][1]);
-        } else {
+        for (int j = 0; j < D / 32; ++j) {
+          uint32_t r[4];
+          ldmatrix_x4(r, raw_piece(kt, (mat & 1) * 8 + mrow, 2 * j + (mat >> 1)));
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int ks = 2 * j + half;
+            const uint32_t af[4] = {int8x2_to_f16x2<0x5140>(r[2 * half]), int8x2_to_f16x2<0x5140>(r[2 * half + 1]),
+                                    int8x2_to_f16x2<0x5342>(r[2 * half]), int8x2_to_f16x2<0x5342>(r[2 * half + 1])};
+            if (half) mma_f16_16816(a1, af, qb[ks][0], qb[ks][1]);
+            else      mma_f16_16816(a0, af, qb[ks][0], qb[ks][1]);
+          }
+        }
+      } else {
+        const uint32_t ks_base = smem_u32(ring + (size_t)s * C::kStageBytes);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          uint32_t af[4];
+          ldmatrix_x4(af, ks_base + (ks >> 2) * C::kBoxBytes + (k_lane_off ^ (uint32_t)(((2 * ks) & 7) << 4)));
           if (ks & 1) mma_bf16_16816(a1, af, qb[ks][0], qb[ks][1]);
           else        mma_bf16_16816(a0, af, qb[ks][0], qb[ks][1]);
         }
@@ -618,10 +624,9 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       for (int i = 0; i < 4; ++i) acc[i] = a0[i] + a1[i];
       if constexpr (Q8) {
         // the rows' scales: keys gid (registers 0, 1) and gid + 8 (registers 2, 3)
-        const float* kscale = reinterpret_cast<const float*>(stage + 2 * C::kRawTileBytes);
+        const float* kscale = raw_scales(s);
         const float s0 = kscale[gid], s1 = kscale[gid + 8];
         acc[0] *= s0; acc[1] *= s0; acc[2] *= s1; acc[3] *= s1;
-        __syncwarp();                 // every lane is done with the expanded K tile before the next one overwrites it
       }
     };
 
@@ -638,7 +643,6 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     auto patch_new_row = [&](uint32_t idx) {
       constexpr int kPieces = D / 8;                     // 16-byte pieces of one row
       const int r = (new_slot - I.z) % kTileRows;
-      uint8_t* ks = ring + (size_t)(idx % C::kStages) * C::kStageBytes;
       const size_t src = ((size_t)e * p.n_kv_heads + h) * D;
       const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
       const int page = p.block_table[(size_t)le * p.max_pages_per_seq + new_slot / p.page_size];
@@ -646,35 +650,35 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       if (!page_ok && lane == 0) record_status(p.hdr, XKV_ERR_CAPACITY);
       if constexpr (Q8) {
         // The new row is quantised here (its D/8 pieces on consecutive lanes: K on the first D/8 lanes, V on the next
-        // ones), its codes and scales go into the raw tile, where the expansion picks them up, and into the page.
+        // ones); its bytes and scales go into the landed raw tile and into the page.
         static_assert(2 * kPieces <= 32, "one warp holds the K and V pieces of a row");
+        const uint32_t st = idx % C::kStages;
         if (lane < 2 * kPieces) {
           const int is_v = lane / kPieces, c = lane % kPieces;
           float x[8], sc;
           bf16x8_to_f32(*reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8), x);
-          const uint2 codes = quantize_row_piece(x, kPieces, &sc);
-          uint8_t* raw = ks + is_v * C::kRawTileBytes;
-          *reinterpret_cast<uint2*>(raw + r * D + c * 8) = codes;
-          float* tile_scales = reinterpret_cast<float*>(ks + 2 * C::kRawTileBytes + is_v * C::kScaleBytes);
-          if (c == 0) tile_scales[r] = sc;
+          const uint2 bytes = quantize_row_piece(x, kPieces, &sc);
+          uint8_t* raw = is_v ? raw_v(st) : raw_k(st);
+          const int off = D == 128 ? r * 128 + (((c >> 1) ^ (r & 7)) << 4) + (c & 1) * 8 : r * D + c * 8;
+          *reinterpret_cast<uint2*>(raw + off) = bytes;
+          if (c == 0) raw_scales(st)[is_v * kTileRows + r] = sc;
           if (page_ok) {
             const size_t slot = ((size_t)page * p.n_kv_heads + h) * p.page_size + new_slot % p.page_size;
-            *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(is_v ? p.v_pages : p.k_pages) + slot * D + c * 8) = codes;
+            *reinterpret_cast<uint2*>(reinterpret_cast<uint8_t*>(is_v ? p.v_pages : p.k_pages) + slot * D + c * 8) = bytes;
             if (c == 0) (is_v ? p.v_scales : p.k_scales)[slot] = sc;
           }
         }
-        fence_proxy_async_smem();     // the stage is written again by a later copy
-        __syncwarp();
-        return;
-      }
-      for (int i = lane; i < 2 * kPieces; i += 32) {
-        const int is_v = i / kPieces, c = i % kPieces;
-        const uint4 val = *reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8);
-        *reinterpret_cast<uint4*>(ks + is_v * C::kTileBytes + (c >> 3) * C::kBoxBytes + r * 128 +
-                                  (((c & 7) ^ (r & 7)) << 4)) = val;
-        if (page_ok) {
-          const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + new_slot % p.page_size) * D + c * 8;
-          *reinterpret_cast<uint4*>((is_v ? p.v_pages : p.k_pages) + dst) = val;
+      } else {
+        uint8_t* ks = ring + (size_t)(idx % C::kStages) * C::kStageBytes;
+        for (int i = lane; i < 2 * kPieces; i += 32) {
+          const int is_v = i / kPieces, c = i % kPieces;
+          const uint4 val = *reinterpret_cast<const uint4*>((is_v ? p.v_new : p.k_new) + src + c * 8);
+          *reinterpret_cast<uint4*>(ks + is_v * C::kTileBytes + (c >> 3) * C::kBoxBytes + r * 128 +
+                                    (((c & 7) ^ (r & 7)) << 4)) = val;
+          if (page_ok) {
+            const size_t dst = (((size_t)page * p.n_kv_heads + h) * p.page_size + new_slot % p.page_size) * D + c * 8;
+            *reinterpret_cast<uint4*>((is_v ? p.v_pages : p.k_pages) + dst) = val;
+          }
         }
       }
       fence_proxy_async_smem();       // the stage is written again by a later copy
@@ -698,30 +702,30 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         if (!aborted) qk_tile(consumed + 1, s_next);
       }
       if (!aborted) {
-        uint8_t* stage = ring + (size_t)s * C::kStageBytes;
         float vs0 = 1.f, vs1 = 1.f;                    // Q8: scales of the V rows gid and gid + 8
         if constexpr (Q8) {
-          expand_tile(stage + C::kRawTileBytes, v_exp);
-          const float* vscale = reinterpret_cast<const float*>(stage + 2 * C::kRawTileBytes + C::kScaleBytes);
+          const float* vscale = raw_scales(s) + kTileRows;
           vs0 = gid < wrows ? vscale[gid] : 0.f;       // rows past the end of the cache carry no weight at all
           vs1 = gid + 8 < wrows ? vscale[gid + 8] : 0.f;
         }
-        const uint32_t vs_base = Q8 ? smem_u32(v_exp) : smem_u32(stage) + C::kTileBytes;
+        const uint32_t vs_base = smem_u32(ring + (size_t)s * C::kStageBytes) + C::kTileBytes;
         if (wrows < kTileRows) {
-          // rows past the end of the cache hold whatever the page held: mask their scores and clear V so
-          // that 0 * x stays 0
+          // rows past the end of the cache hold whatever the page held: mask their scores and (16-bit tiles, where the
+          // leftovers may be NaN) clear V so that 0 * x stays 0; stored bytes are always finite integers
           if (gid >= wrows) sv[0] = sv[1] = -INFINITY;
           if (gid + 8 >= wrows) sv[2] = sv[3] = -INFINITY;
-          uint8_t* vs = Q8 ? v_exp : stage + C::kTileBytes;
-          const int n_bad = kTileRows - wrows;
-          for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
-            const int row = wrows + idx / (D / 8);
-            const int c = idx % (D / 8);
-            *reinterpret_cast<uint4*>(vs + (c >> 3) * C::kBoxBytes + row * 128 + (c & 7) * 16) =
-                make_uint4(0u, 0u, 0u, 0u);
+          if constexpr (!Q8) {
+            uint8_t* vs = ring + (size_t)s * C::kStageBytes + C::kTileBytes;
+            const int n_bad = kTileRows - wrows;
+            for (int idx = lane; idx < n_bad * (D / 8); idx += 32) {
+              const int row = wrows + idx / (D / 8);
+              const int c = idx % (D / 8);
+              *reinterpret_cast<uint4*>(vs + (c >> 3) * C::kBoxBytes + row * 128 + (c & 7) * 16) =
+                  make_uint4(0u, 0u, 0u, 0u);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
           }
-          fence_proxy_async_smem();
-          __syncwarp();
         }
         float mx0 = fmaxf(sv[0], sv[2]), mx1 = fmaxf(sv[1], sv[3]);
         const bool grow = (mx0 > m_ref[0] + kLazy) || (mx1 > m_ref[1] + kLazy);
@@ -752,12 +756,30 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // P^T as the B operand of O^T += V^T.P^T: transpose the two 8x8 blocks of the accumulator layout
         const uint32_t b0 = movmatrix_trans(Q8 ? pack_f16(p0 * vs0, p1 * vs0) : pack_bf16(p0, p1));
         const uint32_t b1 = movmatrix_trans(Q8 ? pack_f16(p2 * vs1, p3 * vs1) : pack_bf16(p2, p3));
+        if constexpr (Q8) {
+          // V^T fragments out of the raw [keys][D] tile: a transposing ldmatrix over 16-bit units hands a lane, per
+          // matrix (keys 0-7 | 8-15) x (16 columns), the bytes (key 2*tig, cols 2*gid, 2*gid+1) and (key 2*tig+1, same
+          // cols).  Bytes 0 and 2 are the two keys of column 2*gid, bytes 1 and 3 those of column 2*gid+1: the
+          // accumulator rows gid and gid+8 of a 16-column block therefore stand for columns 2*gid and 2*gid+1.
+          const uint32_t vt = smem_u32(raw_v(s));
 #pragma unroll
-        for (int mt = 0; mt < D / 16; ++mt) {
-          uint32_t af[4];
-          ldmatrix_x4_trans(af, vs_base + (mt >> 2) * C::kBoxBytes + (v_lane_off ^ (uint32_t)(((2 * mt) & 7) << 4)));
-          if constexpr (Q8) mma_f16_16816(o[mt], af, b0, b1);
-          else              mma_bf16_16816(o[mt], af, b0, b1);
+          for (int j = 0; j < D / 32; ++j) {
+            uint32_t r[4];
+            ldmatrix_x4_trans(r, raw_piece(vt, (mat & 1) * 8 + mrow, 2 * j + (mat >> 1)));
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              const uint32_t af[4] = {int8x2_to_f16x2<0x5240>(r[2 * half]), int8x2_to_f16x2<0x5341>(r[2 * half]),
+                                      int8x2_to_f16x2<0x5240>(r[2 * half + 1]), int8x2_to_f16x2<0x5341>(r[2 * half + 1])};
+              mma_f16_16816(o[2 * j + half], af, b0, b1);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int mt = 0; mt < D / 16; ++mt) {
+            uint32_t af[4];
+            ldmatrix_x4_trans(af, vs_base + (mt >> 2) * C::kBoxBytes + (v_lane_off ^ (uint32_t)(((2 * mt) & 7) << 4)));
+            mma_bf16_16816(o[mt], af, b0, b1);
+          }
         }
       }
       __syncwarp();
@@ -782,8 +804,17 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         const uint32_t u0 = movmatrix_trans(pack_bf16(acc[mt][0] * inv0, acc[mt][1] * inv1));
         const uint32_t u1 = movmatrix_trans(pack_bf16(acc[mt][2] * inv0, acc[mt][3] * inv1));
         if (gid < G) {
-          *reinterpret_cast<uint32_t*>(orow + 16 * mt + 2 * tig) = u0;
-          *reinterpret_cast<uint32_t*>(orow + 16 * mt + 8 + 2 * tig) = u1;
+          if constexpr (Q8) {
+            // accumulator rows r < 8 stand for columns 2r, rows 8 + r for columns 2r + 1: u0 holds columns 4*tig and
+            // 4*tig + 2, u1 columns 4*tig + 1 and 4*tig + 3
+            uint2 w;
+            asm("prmt.b32 %0, %1, %2, 0x5410;" : "=r"(w.x) : "r"(u0), "r"(u1));
+            asm("prmt.b32 %0, %1, %2, 0x7632;" : "=r"(w.y) : "r"(u0), "r"(u1));
+            *reinterpret_cast<uint2*>(orow + 16 * mt + 4 * tig) = w;
+          } else {
+            *reinterpret_cast<uint32_t*>(orow + 16 * mt + 2 * tig) = u0;
+            *reinterpret_cast<uint32_t*>(orow + 16 * mt + 8 + 2 * tig) = u1;
+          }
         }
       }
       if (gid == 0 && p.lse != nullptr) {
@@ -804,7 +835,8 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int head = 2 * tig + (i & 1);
-          if (head < G) p.part_o[((size_t)item * G + head) * D + 16 * mt + gid + 8 * (i >> 1)] = o[mt][i];
+          const int col = Q8 ? 2 * gid + (i >> 1) : gid + 8 * (i >> 1);     // see store_out for the 8-bit order
+          if (head < G) p.part_o[((size_t)item * G + head) * D + 16 * mt + col] = o[mt][i];
         }
       if (gid == 0) {
 #pragma unroll
@@ -913,7 +945,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     if (tid == 0) s_plan[3] = (atomicAdd(&p.hdr->grid_arrivals, 1) == (int)gridDim.x - 1) ? 1 : 0;
     __syncthreads();
     if (s_plan[3]) {
-      for (int e = tid; e < n_units; e += kAttnThreads) {
+      for (int e = tid; e < n_units; e += C::kThreads) {
         const int le = (p.layer_begin + e / p.batch) * p.batch + e % p.batch;
         const int n_old = max(p.seq_lens[le], 0);
         if (n_old < cap_rows) {
@@ -953,11 +985,12 @@ bool make_page_tmap(CUtensorMap* tmap, void* base, int D, uint64_t rows, bool q8
   const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
   const cuuint32_t estr[2] = {1u, 1u};
   if (q8) {
-    // one byte per element: a box is 16 whole rows of D bytes, stored as they are (no swizzle)
+    // one byte per element: a box is 16 whole rows of D bytes; rows of 128 bytes are swizzled like the 16-bit tiles
+    // (conflict-free ldmatrix), rows of 64 bytes are stored as they are
     const cuuint64_t gstride[1] = {(cuuint64_t)D};
     const cuuint32_t box[2] = {(cuuint32_t)D, (cuuint32_t)kTileRows};
     return enc(tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               D == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
   }
   const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
@@ -1015,7 +1048,7 @@ xkv_status launch_attn(const CUtensorMap& tk, const CUtensorMap& tv, const Decod
     done[dev].store(true, std::memory_order_release);
   }
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_start, st);
-  decode_attn_kernel<D, Q8><<<sm_count(), kAttnThreads, Cfg<D, Q8>::kSmemBytes, st>>>(tk, tv, p);
+  decode_attn_kernel<D, Q8><<<sm_count(), Cfg<D, Q8>::kThreads, Cfg<D, Q8>::kSmemBytes, st>>>(tk, tv, p);
   if (g_ev_start != nullptr && g_ev_stop != nullptr) cudaEventRecord(g_ev_stop, st);
   count_launch();
   return check_launch();
@@ -1048,7 +1081,7 @@ xkv_status decode_attn(const xkv_dims* d, const xkv_cache* c, int layer_begin, i
   const uint64_t page_rows = (uint64_t)c->n_pages * d->n_kv_heads * c->page_size;
   if (page_rows >= (1ull << 31)) return XKV_ERR_UNSUPPORTED;
 
-  const bool q8 = c->kv_format == XKV_KV_FP8_E4M3;
+  const bool q8 = c->kv_format == XKV_KV_INT8;
   CUtensorMap tk, tv;
   if (!make_page_tmap(&tk, c->k_pages, d->head_dim, page_rows, q8) ||
       !make_page_tmap(&tv, c->v_pages, d->head_dim, page_rows, q8))

@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(kGatherThreads) gather_kernel(SelectParams p) 
     const size_t dst = slot * p.head_dim + lc * 8;
     const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k + src));
     const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v + src));
-    if (p.kv_format == XKV_KV_FP8_E4M3) {
+    if (p.kv_format == XKV_KV_INT8) {
       // the row's lanes (consecutive lanes of the warp) agree on its scale; a lane stores its eight codes
       float x[8], ks, vs;
       bf16x8_to_f32(kv, x);

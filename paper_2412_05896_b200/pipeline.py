@@ -29,7 +29,7 @@ class XkvSession:
         max_budget bounds one head."""
         self.L, self.Hq, self.Hkv, self.d, self.W = n_layers, n_q_heads, n_kv_heads, head_dim, window
         self.head_level = bool(head_level)
-        self.kv_format = kv_format                 # xkv.KV_FP8_E4M3: the reduced caches hold 8-bit codes and row scales
+        self.kv_format = kv_format                 # xkv.KV_INT8: the reduced caches hold 8-bit codes and row scales
         self.G = n_q_heads // n_kv_heads
         self.B = len(lengths)
         self.lengths = list(lengths)
@@ -98,11 +98,11 @@ class XkvSession:
             n_pages += math.ceil(rows / page_size)
         self.n_pages = max(n_pages, 1)
         bf16 = dict(dtype=torch.bfloat16, device=self.device)
-        page_dtype = torch.uint8 if kv_format == xkv.KV_FP8_E4M3 else torch.bfloat16
+        page_dtype = torch.uint8 if kv_format == xkv.KV_INT8 else torch.bfloat16
         self.k_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, dtype=page_dtype, device=self.device)
         self.v_pages = torch.zeros(self.n_pages, page_heads, page_size, head_dim, dtype=page_dtype, device=self.device)
         self.k_scales = self.v_scales = None
-        if kv_format == xkv.KV_FP8_E4M3:
+        if kv_format == xkv.KV_INT8:
             self.k_scales = torch.zeros(self.n_pages, page_heads, page_size, **f32)
             self.v_scales = torch.zeros(self.n_pages, page_heads, page_size, **f32)
         self.block_table = torch.zeros(n_layers, self.n_caches, self.max_pages_per_seq, dtype=torch.int32,

@@ -20,7 +20,7 @@ ERR_CUDA, ERR_TIMEOUT, ERR_CAPACITY = -5, -6, -7
 POOL_MAX, POOL_AVG = 0, 1
 OP_SCORE, OP_SELECT_COMPACT, OP_DECODE_ATTN, OP_PREFILL_ATTN = 0, 1, 2, 3
 BUDGET_PER_LAYER, BUDGET_PER_SEQUENCE, BUDGET_PER_HEAD = 0, 1, 2
-KV_BF16, KV_FP8_E4M3 = 0, 1
+KV_BF16, KV_INT8 = 0, 1
 
 STATIC_SCRATCH_BYTES = 16 << 20
 

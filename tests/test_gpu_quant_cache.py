@@ -53,7 +53,7 @@ def test_quantized_cache_rows_and_decode(name, head_level):
     N = L * w.avg_budget * (Hkv if head_level else 1)
     sess = XkvSession(L, Hq, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode, max_new_tokens=steps,
                       max_budget=n_max or None, total_budget=N, curve_len=n_max or None, device=DEV,
-                      head_level=head_level, kv_format=xkv.KV_FP8_E4M3)
+                      head_level=head_level, kv_format=xkv.KV_INT8)
     sess.score_layers([t[0] for t in tens], [t[1] for t in tens])
     budgets, _ = sess.solve_budgets(total=N, n_min=w.n_min, n_max=n_max)
     sess.assign_pages(budgets)
@@ -75,10 +75,10 @@ def test_quantized_cache_rows_and_decode(name, head_level):
                 kc, ks, vc, vs = _cache_rows(sess, l, cache_idx, hp, n)
                 for rows, codes, scales, store in ((tens[l][1], kc, ks, Kq), (tens[l][2], vc, vs, Vq)):
                     x = O.evict_by_index(f64(rows[lo: lo + t, g]), kept)
-                    ref_codes, ref_scales = O.quantize_rows_e4m3(x)
+                    ref_codes, ref_scales = O.quantize_rows_int8(x)
                     assert np.array_equal(scales, ref_scales), (name, l, b, g)
                     assert np.array_equal(codes, ref_codes), (name, l, b, g, int((codes != ref_codes).sum()))
-                    store[(l, b, g)] = O.dequantize_rows_e4m3(ref_codes, ref_scales)
+                    store[(l, b, g)] = O.dequantize_rows_int8(ref_codes, ref_scales)
 
     for step in range(steps):
         q, kn, vn = WL.decode_tensors(w, step, DEV, stress=True)
@@ -91,10 +91,10 @@ def test_quantized_cache_rows_and_decode(name, head_level):
             for b in range(B):
                 for g in range(Hkv):
                     # the appended row is stored the same way: codes and scale of the new K/V row
-                    kcode, kscale = O.quantize_rows_e4m3(f64(kn[l, b, g])[None])
-                    vcode, vscale = O.quantize_rows_e4m3(f64(vn[l, b, g])[None])
-                    Kq[(l, b, g)] = np.concatenate([Kq[(l, b, g)], O.dequantize_rows_e4m3(kcode, kscale)], 0)
-                    Vq[(l, b, g)] = np.concatenate([Vq[(l, b, g)], O.dequantize_rows_e4m3(vcode, vscale)], 0)
+                    kcode, kscale = O.quantize_rows_int8(f64(kn[l, b, g])[None])
+                    vcode, vscale = O.quantize_rows_int8(f64(vn[l, b, g])[None])
+                    Kq[(l, b, g)] = np.concatenate([Kq[(l, b, g)], O.dequantize_rows_int8(kcode, kscale)], 0)
+                    Vq[(l, b, g)] = np.concatenate([Vq[(l, b, g)], O.dequantize_rows_int8(vcode, vscale)], 0)
                     cache_idx, hp = (b * Hkv + g, 0) if head_level else (b, g)
                     n = int(lens[l, cache_idx])
                     assert n == Kq[(l, b, g)].shape[0]
@@ -111,11 +111,11 @@ def test_quantized_cache_rejections():
     w = replace(WL.CONFIGS["tiny"], n_layers=1, batch=1, prompt=200)
     lengths = WL.prompt_lengths(w)
     sess = XkvSession(1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.window, w.pool_kernel, lengths, max_new_tokens=1,
-                      device=DEV, kv_format=xkv.KV_FP8_E4M3)
+                      device=DEV, kv_format=xkv.KV_INT8)
     q, kn, vn = WL.decode_tensors(w, 0, DEV)
     no_scales = xkv.Cache(sess.k_pages.data_ptr(), sess.v_pages.data_ptr(), sess.block_table.data_ptr(),
                           sess.seq_lens.data_ptr(), 1, sess.page_size, sess.max_pages_per_seq, sess.n_pages, None, None,
-                          xkv.KV_FP8_E4M3, 0)
+                          xkv.KV_INT8, 0)
     with pytest.raises(xkv.XkvError) as e:
         xkv.decode_attn(sess.dims, no_scales, 0, 1, q, kn, vn, sess.out, None, 0, sess.ws_decode)
     assert e.value.status == xkv.ERR_INVALID_ARG
