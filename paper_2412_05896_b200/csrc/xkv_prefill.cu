@@ -3,15 +3,16 @@
 // rows are what the scoring step needs of W_attn (Alg. 2 step 1): with them xkv_score_lse forms the column
 // scores in one pass over the keys.
 //
-// One CTA per (sequence, tile of 128 query rows, query head), 224 threads:
+// One CTA per (sequence, tile of 128 query rows, query head), 224 threads, key tiles of 64; two CTAs share an SM
+// (half of its shared memory and of its tensor memory each), so that one CTA's softmax runs under the other's MMAs:
 //   warps 0-3  softmax: thread = query row = TMEM lane.  Per key tile: row maximum out of TMEM, a reference
 //              maximum that is exact on the first tile and raised lazily afterwards (only when a logit exceeds
 //              it by 2^8, which is when the O accumulator in TMEM is rescaled: load, multiply, store),
 //              P = exp2(s*c - ref) rounded to bf16 into shared memory in the K-major 128-byte-swizzled layout
 //              the MMA reads as its A operand, row sum in fp32.  At the end O / l -> bf16 rows, lse.
-//   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles, and of the V tiles (two stages
-//              each, 128 keys a tile), so that a K tile never queues behind the V stage of an earlier tile
-//   warp 5     MMA issuer (one lane): S = Q K^T into one of two 128-column TMEM buffers, one tile ahead of the
+//   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles (two stages), and of the V tiles
+//              (one stage), so that a K tile never queues behind the V stage of an earlier tile
+//   warp 5     MMA issuer (one lane): S = Q K^T into one of two 64-column TMEM buffers, one tile ahead of the
 //              softmax; O += P V with V as an MN-major B operand straight from its [keys][d] tile
 // Every wait is bounded; an expired wait sets the status word and lets the CTA drain.
 #include <atomic>
@@ -26,7 +27,7 @@ using namespace tc;
 
 constexpr int kPfThreads = 224;
 constexpr int kPfRows = 128;          // query rows per CTA
-constexpr int kPfKeys = 128;          // keys per tile
+constexpr int kPfKeys = 64;           // keys per tile
 constexpr float kPfLazy = 8.f;        // log2 slack before the reference maximum is raised
 
 struct PrefillParams {
@@ -44,14 +45,19 @@ template <int D>
 struct PfCfg {
   static constexpr int kHalves = D / 64;
   static constexpr int kSteps = D / 16;                      // k-steps of S = Q K^T
-  static constexpr int kHalfBytes = 128 * 128;               // 128 rows of 128 bytes
-  static constexpr int kTileBytes = kHalves * kHalfBytes;    // Q, K or V tile
-  static constexpr int kPBytes = 2 * kHalfBytes;             // P: 128 rows x 128 keys bf16
-  static constexpr int kStages = 2;
-  static constexpr uint32_t kSCols = 128;                    // one S buffer
-  static constexpr uint32_t kOCol = 256;                     // O accumulator starts here
-  static constexpr uint32_t kTmemCols = 512;
-  static constexpr size_t kSmemBytes = 1024 + (size_t)kTileBytes * (1 + 2 * kStages) + kPBytes + 256;
+  static constexpr int kQHalfBytes = kPfRows * 128;          // 64 columns of the query tile: rows of 128 bytes
+  static constexpr int kQTileBytes = kHalves * kQHalfBytes;
+  static constexpr int kKvHalfBytes = kPfKeys * 128;         // 64 columns of a K or V tile
+  static constexpr int kKvTileBytes = kHalves * kKvHalfBytes;
+  static constexpr int kPHalfBytes = kPfRows * 128;          // 64 keys of P: rows of 128 bytes
+  static constexpr int kPBytes = (kPfKeys / 64) * kPHalfBytes;   // P: 128 rows x kPfKeys keys, bf16
+  static constexpr int kKStages = 2;                         // S runs one tile ahead of the softmax
+  static constexpr int kVStages = 1;
+  static constexpr uint32_t kSCols = kPfKeys;                // one S buffer
+  static constexpr uint32_t kOCol = 2 * kPfKeys;             // O accumulator starts here
+  static constexpr uint32_t kTmemCols = 256;                 // two CTAs share an SM's 512 columns
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kQTileBytes + (size_t)kKvTileBytes * (kKStages + kVStages) +
+                                       kPBytes + 256;
 };
 
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
@@ -129,16 +135,16 @@ __device__ __forceinline__ bool pf_tile(const PrefillParams& p, int idx, int* b_
 }
 
 template <int D>
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const PrefillParams p) {
   using C = PfCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem;
-  uint8_t* k_s = q_s + C::kTileBytes;
-  uint8_t* v_s = k_s + (size_t)C::kStages * C::kTileBytes;
-  uint8_t* p_s = v_s + (size_t)C::kStages * C::kTileBytes;
+  uint8_t* k_s = q_s + C::kQTileBytes;
+  uint8_t* v_s = k_s + (size_t)C::kKStages * C::kKvTileBytes;
+  uint8_t* p_s = v_s + (size_t)C::kVStages * C::kKvTileBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + C::kPBytes);
   uint64_t* q_full = bars;             // [1]
   uint64_t* k_full = bars + 1;         // [2]
@@ -157,18 +163,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   const int h = blockIdx.x % p.n_q_heads;
   if (!pf_tile(p, blockIdx.x / p.n_q_heads, &b, &q0, &cu, &t)) return;      // uniform over the CTA
   const int g = h / p.group;
-  const int n_kt = q0 / kPfKeys + 1;                 // key tiles up to and including the diagonal one
+  const int n_kt = (q0 + kPfRows) / kPfKeys;         // key tiles up to and including the last one a row of the tile sees
 
   if (tid == 0) {
     mbar_init(q_full, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
-      mbar_init(&v_full[i], 1);
-      mbar_init(&v_empty[i], 1);
       mbar_init(&s_full[i], 1);
       mbar_init(&s_empty[i], 4);
     }
+    mbar_init(v_full, 1);
+    mbar_init(v_empty, 1);
     mbar_init(p_full, 4);
     mbar_init(p_empty, 1);
     *s_abort = 0;
@@ -189,34 +195,32 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   if (warp == 4) {
     // ------------------------------------------------------------------ producer of Q and the K tiles
     if (lane == 0) {
-      mbar_arrive_expect_tx(q_full, (uint32_t)C::kTileBytes);
+      mbar_arrive_expect_tx(q_full, (uint32_t)C::kQTileBytes);
 #pragma unroll
-      for (int hf = 0; hf < C::kHalves; ++hf) tma_load_3d(q_s + hf * C::kHalfBytes, &tmap_q, hf * 64, h, cu + q0, q_full);
+      for (int hf = 0; hf < C::kHalves; ++hf) tma_load_3d(q_s + hf * C::kQHalfBytes, &tmap_q, hf * 64, h, cu + q0, q_full);
       bool ok = true;
       for (int j = 0; ok && j < n_kt; ++j) {
         const uint32_t s = j & 1u, ph = ((j >> 1) & 1u) ^ 1u;
         ok = ws_wait(&k_empty[s], ph, s_abort, p.wait_ns);
         if (!ok) break;
-        mbar_arrive_expect_tx(&k_full[s], (uint32_t)C::kTileBytes);
+        mbar_arrive_expect_tx(&k_full[s], (uint32_t)C::kKvTileBytes);
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_3d(k_s + (size_t)s * C::kTileBytes + hf * C::kHalfBytes, &tmap_k, hf * 64, g, cu + j * kPfKeys,
+          tma_load_3d(k_s + (size_t)s * C::kKvTileBytes + hf * C::kKvHalfBytes, &tmap_k, hf * 64, g, cu + j * kPfKeys,
                       &k_full[s]);
       }
     }
   } else if (warp == 6) {
-    // ------------------------------------------------------------------ producer of the V tiles
+    // ------------------------------------------------------------------ producer of the V tiles (one stage)
     if (lane == 0) {
       bool ok = true;
       for (int j = 0; ok && j < n_kt; ++j) {
-        const uint32_t s = j & 1u, ph = ((j >> 1) & 1u) ^ 1u;
-        ok = ws_wait(&v_empty[s], ph, s_abort, p.wait_ns);
+        ok = ws_wait(v_empty, (j & 1u) ^ 1u, s_abort, p.wait_ns);
         if (!ok) break;
-        mbar_arrive_expect_tx(&v_full[s], (uint32_t)C::kTileBytes);
+        mbar_arrive_expect_tx(v_full, (uint32_t)C::kKvTileBytes);
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_3d(v_s + (size_t)s * C::kTileBytes + hf * C::kHalfBytes, &tmap_v, hf * 64, g, cu + j * kPfKeys,
-                      &v_full[s]);
+          tma_load_3d(v_s + hf * C::kKvHalfBytes, &tmap_v, hf * 64, g, cu + j * kPfKeys, v_full);
       }
     }
   } else if (warp == 5) {
@@ -230,11 +234,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
         if (!ws_wait(&s_empty[s], ((j >> 1) & 1u) ^ 1u, s_abort, p.wait_ns)) return false;
         tc_fence_after_sync();
-        const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kTileBytes);
+        const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kKvTileBytes);
 #pragma unroll
         for (int k = 0; k < C::kSteps; ++k) {
-          const uint64_t off = (uint64_t)(((k / 4) * C::kHalfBytes + (k % 4) * 32) >> 4);
-          umma_bf16(tmem_base + s * C::kSCols, q_desc + off, k_desc + off, umma_idesc(kPfRows, kPfKeys),
+          const uint64_t q_off = (uint64_t)(((k / 4) * C::kQHalfBytes + (k % 4) * 32) >> 4);
+          const uint64_t k_off = (uint64_t)(((k / 4) * C::kKvHalfBytes + (k % 4) * 32) >> 4);
+          umma_bf16(tmem_base + s * C::kSCols, q_desc + q_off, k_desc + k_off, umma_idesc(kPfRows, kPfKeys),
                     k > 0 ? 1u : 0u);
         }
         umma_commit(&k_empty[s]);
@@ -248,18 +253,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           if (!ok) break;
         }
         const uint32_t s = j & 1u;
-        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(&v_full[s], (j >> 1) & 1u, s_abort, p.wait_ns);
+        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(v_full, j & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t v_base = smem_u32(v_s) + s * C::kTileBytes;
+        const uint32_t v_base = smem_u32(v_s);
 #pragma unroll
         for (int k = 0; k < kPfKeys / 16; ++k) {
           // A: P[rows][keys 16k .. 16k+15], K-major; B: V[keys 16k ..][d], MN-major (16 keys = two 8-row groups)
-          const uint64_t pd = p_desc + (uint64_t)(((k / 4) * C::kHalfBytes + (k % 4) * 32) >> 4);
-          const uint64_t vd = umma_desc_mn128(v_base + k * 16 * 128, C::kHalfBytes);
+          const uint64_t pd = p_desc + (uint64_t)(((k / 4) * C::kPHalfBytes + (k % 4) * 32) >> 4);
+          const uint64_t vd = umma_desc_mn128(v_base + k * 16 * 128, C::kKvHalfBytes);
           umma_bf16(tmem_base + C::kOCol, pd, vd, umma_idesc_b_mn(kPfRows, D), (j > 0 || k > 0) ? 1u : 0u);
         }
-        umma_commit(&v_empty[s]);
+        umma_commit(v_empty);
         umma_commit(p_empty);
       }
     }
@@ -276,7 +281,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t s_addr = lane_base + s * C::kSCols;
-      const bool diag = j == n_kt - 1;                       // the only tile with keys beyond some row's position
+      const bool diag = (j + 1) * kPfKeys - 1 > q0;          // the tile holds keys beyond some row's position
       const int c_base = j * kPfKeys;
       // ---- row maximum of the tile
       float mx = -INFINITY;
@@ -339,7 +344,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           packed[i >> 1] = pack_bf16(e0, e1);
         }
         // 32 keys = four 16-byte pieces of the row's 128-byte line in half cc/64; piece index XOR (row & 7)
-        uint8_t* line = p_s + (cc >> 6) * C::kHalfBytes + r * 128;
+        uint8_t* line = p_s + (cc >> 6) * C::kPHalfBytes + r * 128;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int piece = ((cc & 63) >> 3) + q;
@@ -415,12 +420,12 @@ xkv_status pf_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
   return check_launch();
 }
 
-// 3-D map {d, heads, tokens} with box {64, 1, 128} over a packed [T][heads][d] bf16 tensor.
+// 3-D map {d, heads, tokens} with box {64, 1, box_rows} over a packed [T][heads][d] bf16 tensor.
 bool pf_make_tmap(CUtensorMap* tmap, const void* base, int head_dim, int heads, int64_t tokens, int64_t stride_token,
-                  int64_t stride_head) {
+                  int64_t stride_head, int box_rows) {
   const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)heads, (cuuint64_t)tokens};
   const cuuint64_t strides[2] = {(cuuint64_t)stride_head * 2, (cuuint64_t)stride_token * 2};
-  const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)kPfKeys};
+  const cuuint32_t box[3] = {64u, 1u, (cuuint32_t)box_rows};
   return tc_make_tmap(tmap, base, 3, dims, strides, box);
 }
 
@@ -446,9 +451,10 @@ xkv_status prefill_attn(const xkv_dims* d, const void* q, const void* k, const v
   p.scale_log2 = scale * 1.4426950408889634f;
   p.wait_ns = wait_limit_ns();
   CUtensorMap tq, tk, tv;
-  if (!pf_make_tmap(&tq, q, d->head_dim, d->n_q_heads, total_tokens, (int64_t)d->n_q_heads * d->head_dim, d->head_dim) ||
-      !pf_make_tmap(&tk, k, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head) ||
-      !pf_make_tmap(&tv, v, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head))
+  if (!pf_make_tmap(&tq, q, d->head_dim, d->n_q_heads, total_tokens, (int64_t)d->n_q_heads * d->head_dim, d->head_dim,
+                    kPfRows) ||
+      !pf_make_tmap(&tk, k, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head, kPfKeys) ||
+      !pf_make_tmap(&tv, v, d->head_dim, d->n_kv_heads, total_tokens, d->kv_stride_token, d->kv_stride_head, kPfKeys))
     return XKV_ERR_CUDA;
   // an upper bound of the query tiles that exist: every sequence adds at most one partial tile
   const int64_t tiles = total_tokens / kPfRows + d->batch;
