@@ -42,7 +42,7 @@ DEC_DISTINCT = 64          # distinct sets of decode-step inputs held in memory;
 # (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one decode_attn_kernel launch, taken from
 # an ncu capture of a smaller case of the same kernel; traffic grows in proportion to the retained rows, so a full
 # launch's traffic is this ratio times its algorithmic bytes.  None whenever the kernel has changed since the capture.
-NCU_TRAFFIC_RATIO = 1.031
+NCU_TRAFFIC_RATIO = 1.033
 
 
 def measured_peak():
@@ -450,8 +450,9 @@ def run_workload(ctx: Ctx, name: str, steps: int, warmup: int, headline: bool) -
             "peak_source": ctx.tf_src,
             "note": "4*d*Hq*sum_b t_b(t_b+1)/2 flops; outside the timed step (the model's own attention)"}
         lse_list = [lse_all[l] for l in range(L)]
-        reps = 3
-        sess.score_layers(q_win, k, lse=lse_list)
+        reps = 6
+        for _ in range(2):
+            sess.score_layers(q_win, k, lse=lse_list)
         a, b_ = ev(), ev()
         a.record()
         for _ in range(reps):
