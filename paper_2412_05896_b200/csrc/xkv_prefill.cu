@@ -252,7 +252,6 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           ok = issue_qk(j + 1);           // the next tile's logits run under this tile's softmax
           if (!ok) break;
         }
-        const uint32_t s = j & 1u;
         ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(v_full, j & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         tc_fence_after_sync();
