@@ -22,7 +22,7 @@ class XkvSession:
                  pool_kernel: int, lengths: list[int], pool_mode: int = xkv.POOL_MAX, page_size: int = 16,
                  max_new_tokens: int = 0, max_budget: int | None = None, total_budget: int | None = None,
                  curve_len: int | None = None, device="cuda:0", scale: float = 0.0,
-                 decode_chunk_rows: int = 0, n_lanes: int = 3, head_level: bool = False,
+                 decode_chunk_rows: int = 0, n_lanes: int = 6, head_level: bool = False,
                  kv_format: int = xkv.KV_BF16):
         """head_level: budgets, cache lengths and page lists per (layer, sequence, KV head) instead of per (layer,
         sequence); total_budget and the solver's total then count prefix tokens over all heads of all layers, and
