@@ -337,6 +337,26 @@ struct WaitEntry {
   }
 };
 
+// A curve as the solver reads it: the caller's floats as they are (every float is a double, so nothing is copied or
+// converted up front), or doubles computed here (a batch mean).
+struct Curve {
+  const float* f = nullptr;
+  const double* d = nullptr;
+  int64_t n = 0;
+  double operator[](int64_t j) const { return f != nullptr ? (double)f[j] : d[j]; }
+  int64_t size() const { return n; }
+  // true if no value over [a, b) is larger than its predecessor (a plain reduction, so that it vectorises)
+  bool non_increasing(int64_t a, int64_t b) const {
+    int bad = 0;
+    if (f != nullptr) {
+      for (int64_t j = a; j < b; ++j) bad |= f[j] > f[j - 1];
+    } else {
+      for (int64_t j = a; j < b; ++j) bad |= d[j] > d[j - 1];
+    }
+    return bad == 0;
+  }
+};
+
 // Order-preserving map of a double onto an unsigned integer (larger value -> larger key).
 inline uint64_t ordered_key(double v) {
   uint64_t u;
@@ -349,7 +369,7 @@ inline uint64_t ordered_key(double v) {
 // position ascending), so its result is "every position above the R-th largest value, and positions equal
 // to it from the lowest layers first".  The R-th largest value is found by bisecting the value's bit pattern,
 // counting per layer with a binary search: the same budgets as the heap below, without its R pops.
-bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std::vector<int64_t>& cap, int64_t total,
+bool solve_sorted_total(const std::vector<Curve>& curve, const std::vector<int64_t>& cap, int64_t total,
                         int n_min, int32_t* budgets, double* r_avg, xkv_status* status) {
   const int L = (int)curve.size();
   std::vector<int64_t> lo(L), hi(L);           // open positions of layer l: [lo, hi); beyond the curve the gain is 0
@@ -360,8 +380,7 @@ bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std
     used += lo[l];
     open += hi[l] - lo[l];
     const int64_t n = (int64_t)curve[l].size();
-    for (int64_t j = lo[l] + 1; j < hi[l] && j < n; ++j)
-      if (curve[l][j] > curve[l][j - 1]) return false;
+    if (!curve[l].non_increasing(lo[l] + 1, hi[l] < n ? hi[l] : n)) return false;
     if (hi[l] > n && n > lo[l] && curve[l][n - 1] < 0.0) return false;       // the implicit zeros would rise again
   }
   if (total < used || total - used > open) {
@@ -370,9 +389,11 @@ bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std
   }
   const int64_t R = total - used;
   auto value_at = [&](int l, int64_t j) -> double { return j < (int64_t)curve[l].size() ? curve[l][j] : 0.0; };
-  // open positions of layer l whose key is >= key (the curve is non-increasing, so they form a prefix)
-  auto count_ge = [&](int l, uint64_t key) -> int64_t {
-    int64_t a = lo[l], b = hi[l];
+  // Open positions of layer l whose key is >= key (the curve is non-increasing, so they form a prefix), given that
+  // the answer lies in [a, b].
+  auto count_ge = [&](int l, uint64_t key, int64_t a, int64_t b) -> int64_t {
+    a += lo[l];
+    b += lo[l];
     while (a < b) {
       const int64_t mid = (a + b) >> 1;
       if (ordered_key(value_at(l, mid)) >= key) a = mid + 1;
@@ -382,22 +403,35 @@ bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std
   };
   std::vector<int64_t> alloc(lo);
   if (R > 0) {
-    uint64_t klo = 0, khi = ~0ull;               // largest key with count(key) >= R
+    // Largest key with count(key) >= R, by bisection of the key.  The counts are monotone in the key, so every layer
+    // keeps a bracket [below[l], above[l]] = [count at khi + 1, count at klo] that each step narrows: the 64 steps
+    // together cost one binary search per layer plus a few probes a step.
+    uint64_t klo = 0, khi = ~0ull;
+    std::vector<int64_t> below(L, 0), above(L), at_mid(L);
+    for (int l = 0; l < L; ++l) above[l] = hi[l] - lo[l];
     while (klo < khi) {
       const uint64_t mid = klo + ((khi - klo) >> 1) + 1;
       int64_t c = 0;
-      for (int l = 0; l < L; ++l) c += count_ge(l, mid);
-      if (c >= R) klo = mid;
-      else khi = mid - 1;
+      for (int l = 0; l < L; ++l) {
+        at_mid[l] = count_ge(l, mid, below[l], above[l]);
+        c += at_mid[l];
+      }
+      if (c >= R) {
+        klo = mid;
+        above.swap(at_mid);
+      } else {
+        khi = mid - 1;
+        below.swap(at_mid);
+      }
     }
     int64_t left = R;
     for (int l = 0; l < L; ++l) {                // everything strictly above the threshold value
-      const int64_t above = klo == ~0ull ? 0 : count_ge(l, klo + 1);
-      alloc[l] += above;
-      left -= above;
+      const int64_t n_above = klo == ~0ull ? 0 : count_ge(l, klo + 1, 0, hi[l] - lo[l]);
+      alloc[l] += n_above;
+      left -= n_above;
     }
     for (int l = 0; l < L && left > 0; ++l) {    // ties at the threshold: lowest layers first
-      const int64_t ties = count_ge(l, klo) - (alloc[l] - lo[l]);
+      const int64_t ties = count_ge(l, klo, 0, hi[l] - lo[l]) - (alloc[l] - lo[l]);
       const int64_t take = ties < left ? ties : left;
       alloc[l] += take;
       left -= take;
@@ -413,7 +447,7 @@ bool solve_sorted_total(const std::vector<std::vector<double>>& curve, const std
   return true;
 }
 
-xkv_status solve_one(const std::vector<std::vector<double>>& curve, const std::vector<int64_t>& cap,
+xkv_status solve_one(const std::vector<Curve>& curve, const std::vector<int64_t>& cap,
                      int64_t total, double r_target, int n_min, int32_t* budgets, double* r_avg) {
   const int L = (int)curve.size();
   if (total >= 0) {
@@ -472,31 +506,45 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
     if (prefix_len[b] > max_prefix) max_prefix = prefix_len[b];
   }
   const size_t lstride = (size_t)batch * curve_len;
+  std::vector<Curve> curve(n_layers);
   if (!per_sequence) {
-    std::vector<std::vector<double>> curve(n_layers, std::vector<double>(curve_len, 0.0));
-    auto mean_layers = [&](int l0, int l1) {
-      for (int l = l0; l < l1; ++l) {
-        double* c = curve[l].data();
-        for (int b = 0; b < batch; ++b) {
-          const float* g = gains + l * lstride + (size_t)b * curve_len;
-          for (int j = 0; j < curve_len; ++j) c[j] += (double)g[j];
-        }
-        for (int j = 0; j < curve_len; ++j) c[j] /= batch;
+    std::vector<std::vector<double>> mean;
+    if (batch == 1) {
+      // one curve per layer already (the session averages over the batch on the device): read it in place
+      for (int l = 0; l < n_layers; ++l) {
+        curve[l].f = gains + l * lstride;
+        curve[l].n = curve_len;
       }
-    };
-    // the batch mean reads every curve once: spread the layers over a few threads when that is megabytes
-    int n_threads = (int)std::min<size_t>(8, (size_t)n_layers * lstride / (4u << 20));
-    const int hw = (int)std::thread::hardware_concurrency();
-    if (hw > 0 && n_threads > hw) n_threads = hw;
-    if (n_threads > n_layers) n_threads = n_layers;
-    if (n_threads <= 1) {
-      mean_layers(0, n_layers);
     } else {
-      std::vector<std::thread> pool;
-      for (int i = 0; i < n_threads; ++i)
-        pool.emplace_back(mean_layers, (int)((int64_t)n_layers * i / n_threads),
-                          (int)((int64_t)n_layers * (i + 1) / n_threads));
-      for (auto& th : pool) th.join();
+      mean.assign(n_layers, std::vector<double>(curve_len, 0.0));
+      auto mean_layers = [&](int l0, int l1) {
+        for (int l = l0; l < l1; ++l) {
+          double* c = mean[l].data();
+          for (int b = 0; b < batch; ++b) {
+            const float* g = gains + l * lstride + (size_t)b * curve_len;
+            for (int j = 0; j < curve_len; ++j) c[j] += (double)g[j];
+          }
+          for (int j = 0; j < curve_len; ++j) c[j] /= batch;
+        }
+      };
+      // the batch mean reads every curve once: spread the layers over a few threads when that is megabytes
+      int n_threads = (int)std::min<size_t>(8, (size_t)n_layers * lstride / (4u << 20));
+      const int hw = (int)std::thread::hardware_concurrency();
+      if (hw > 0 && n_threads > hw) n_threads = hw;
+      if (n_threads > n_layers) n_threads = n_layers;
+      if (n_threads <= 1) {
+        mean_layers(0, n_layers);
+      } else {
+        std::vector<std::thread> pool;
+        for (int i = 0; i < n_threads; ++i)
+          pool.emplace_back(mean_layers, (int)((int64_t)n_layers * i / n_threads),
+                            (int)((int64_t)n_layers * (i + 1) / n_threads));
+        for (auto& th : pool) th.join();
+      }
+      for (int l = 0; l < n_layers; ++l) {
+        curve[l].d = mean[l].data();
+        curve[l].n = curve_len;
+      }
     }
     int64_t c = max_prefix;
     if (n_max > 0 && n_max < c) c = n_max;
@@ -504,10 +552,9 @@ xkv_status xkv_alloc_budgets(const float* gains, int32_t n_layers, int32_t batch
     return solve_one(curve, cap, total, r_target, n_min, budgets, r_avg);
   }
   for (int b = 0; b < batch; ++b) {
-    std::vector<std::vector<double>> curve(n_layers, std::vector<double>(curve_len));
     for (int l = 0; l < n_layers; ++l) {
-      const float* g = gains + l * lstride + (size_t)b * curve_len;
-      for (int j = 0; j < curve_len; ++j) curve[l][j] = (double)g[j];
+      curve[l].f = gains + l * lstride + (size_t)b * curve_len;
+      curve[l].n = curve_len;
     }
     int64_t c = prefix_len[b];
     if (n_max > 0 && n_max < c) c = n_max;
