@@ -290,12 +290,22 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         tmem_ld32(s_addr + (uint32_t)cc, va);
         tmem_ld32(s_addr + (uint32_t)(cc + 32), vb);
         tmem_wait_ld();
+        if (diag) {                                          // only tiles on the diagonal hold keys a row must not see
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float a = (diag && c_base + cc + i > row_pos) ? -INFINITY : va[i];
-          const float bb = (diag && c_base + cc + 32 + i > row_pos) ? -INFINITY : vb[i];
-          mx = fmaxf(mx, fmaxf(a, bb));
+          for (int i = 0; i < 32; ++i) {
+            if (c_base + cc + i > row_pos) va[i] = -INFINITY;
+            if (c_base + cc + 32 + i > row_pos) vb[i] = -INFINITY;
+          }
         }
+        float m4[4] = {mx, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one dependent sequence
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          m4[0] = fmaxf(m4[0], fmaxf(va[i], vb[i]));
+          m4[1] = fmaxf(m4[1], fmaxf(va[i + 1], vb[i + 1]));
+          m4[2] = fmaxf(m4[2], fmaxf(va[i + 2], vb[i + 2]));
+          m4[3] = fmaxf(m4[3], fmaxf(va[i + 3], vb[i + 3]));
+        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
       mx *= p.scale_log2;                                    // key 0 is always visible, so mx is finite
       const bool grow = mx > m_ref + kPfLazy;                // also true on the first tile (m_ref = -inf)
