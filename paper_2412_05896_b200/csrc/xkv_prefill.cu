@@ -334,23 +334,34 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
       }
       // ---- P = exp2(s*c - ref) as bf16 into shared memory, row sum in fp32
-      float sum = 0.f;
+      float sm[4] = {0.f, 0.f, 0.f, 0.f};
+      static_assert(kPfKeys == 64, "both halves of the tile's logits are loaded before one wait");
+      float v[2][32];
+      tmem_ld32(s_addr, v[0]);
+      tmem_ld32(s_addr + 32u, v[1]);
+      tmem_wait_ld();
+      if (diag) {                                            // masked logits become -inf: their exponential is exactly 0
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (c_base + i > row_pos) v[0][i] = -INFINITY;
+          if (c_base + 32 + i > row_pos) v[1][i] = -INFINITY;
+        }
+      }
 #pragma unroll
       for (int cc = 0; cc < kPfKeys; cc += 32) {
-        float v[32];
-        tmem_ld32(s_addr + (uint32_t)cc, v);
-        tmem_wait_ld();
         uint32_t packed[16];
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float e0 = fast_exp2(fmaf(v[i], p.scale_log2, -m_ref));
-          float e1 = fast_exp2(fmaf(v[i + 1], p.scale_log2, -m_ref));
-          if (diag) {
-            if (c_base + cc + i > row_pos) e0 = 0.f;
-            if (c_base + cc + i + 1 > row_pos) e1 = 0.f;
-          }
-          sum += e0 + e1;
+        for (int i = 0; i < 32; i += 4) {
+          const float e0 = fast_exp2(fmaf(v[cc >> 5][i], p.scale_log2, -m_ref));
+          const float e1 = fast_exp2(fmaf(v[cc >> 5][i + 1], p.scale_log2, -m_ref));
+          const float e2 = fast_exp2(fmaf(v[cc >> 5][i + 2], p.scale_log2, -m_ref));
+          const float e3 = fast_exp2(fmaf(v[cc >> 5][i + 3], p.scale_log2, -m_ref));
+          sm[0] += e0;
+          sm[1] += e1;
+          sm[2] += e2;
+          sm[3] += e3;
           packed[i >> 1] = pack_bf16(e0, e1);
+          packed[(i >> 1) + 1] = pack_bf16(e2, e3);
         }
         // 32 keys = four 16-byte pieces of the row's 128-byte line in half cc/64; piece index XOR (row & 7)
         uint8_t* line = p_s + (cc >> 6) * C::kPHalfBytes + r * 128;
@@ -361,6 +372,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
         }
       }
+      const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
       l += sum;
       // the S buffer has been read for the last time; P and O are ready for the MMA
       tc_fence_before_sync();
