@@ -60,25 +60,34 @@ struct PfCfg {
                                        kPBytes + 256;
 };
 
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 16 consecutive fp32 columns of this thread's TMEM lane (the rescale of O works in these smaller pieces so that the
+// tile's logits can stay in registers beside it).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
       ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
         "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
         "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
         "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
         "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
-        "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])),
-        "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])),
-        "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
-        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
-        "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
-        "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        "r"(__float_as_uint(v[15]))
       : "memory");
 }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory descriptor of an MN-major operand tile stored as rows of 128 bytes (64 bf16 along MN) per K index
 // with the 128-byte swizzle: eight K rows form a 1024-byte group (stride byte offset), the next 64 MN elements
@@ -282,31 +291,29 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const uint32_t s_addr = lane_base + s * C::kSCols;
       const bool diag = (j + 1) * kPfKeys - 1 > q0;          // the tile holds keys beyond some row's position
       const int c_base = j * kPfKeys;
-      // ---- row maximum of the tile
-      float mx = -INFINITY;
+      // ---- the tile's 64 logits of this row leave TMEM once; keys beyond the row's position (only tiles on the diagonal
+      //      hold any) become -inf here, so neither the maximum nor the exponentials below mask again
+      static_assert(kPfKeys == 64, "the softmax keeps one tile of 64 logits per row in registers");
+      float v[2][32];
+      tmem_ld32(s_addr, v[0]);
+      tmem_ld32(s_addr + 32u, v[1]);
+      tmem_wait_ld();
+      if (diag) {
 #pragma unroll
-      for (int cc = 0; cc < kPfKeys; cc += 64) {
-        float va[32], vb[32];
-        tmem_ld32(s_addr + (uint32_t)cc, va);
-        tmem_ld32(s_addr + (uint32_t)(cc + 32), vb);
-        tmem_wait_ld();
-        if (diag) {                                          // only tiles on the diagonal hold keys a row must not see
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            if (c_base + cc + i > row_pos) va[i] = -INFINITY;
-            if (c_base + cc + 32 + i > row_pos) vb[i] = -INFINITY;
-          }
+        for (int i = 0; i < 32; ++i) {
+          if (c_base + i > row_pos) v[0][i] = -INFINITY;
+          if (c_base + 32 + i > row_pos) v[1][i] = -INFINITY;
         }
-        float m4[4] = {mx, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one dependent sequence
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          m4[0] = fmaxf(m4[0], fmaxf(va[i], vb[i]));
-          m4[1] = fmaxf(m4[1], fmaxf(va[i + 1], vb[i + 1]));
-          m4[2] = fmaxf(m4[2], fmaxf(va[i + 2], vb[i + 2]));
-          m4[3] = fmaxf(m4[3], fmaxf(va[i + 3], vb[i + 3]));
-        }
-        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one dependent sequence
+#pragma unroll
+      for (int i = 0; i < 32; i += 4) {
+        m4[0] = fmaxf(m4[0], fmaxf(v[0][i], v[1][i]));
+        m4[1] = fmaxf(m4[1], fmaxf(v[0][i + 1], v[1][i + 1]));
+        m4[2] = fmaxf(m4[2], fmaxf(v[0][i + 2], v[1][i + 2]));
+        m4[3] = fmaxf(m4[3], fmaxf(v[0][i + 3], v[1][i + 3]));
+      }
+      float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       mx *= p.scale_log2;                                    // key 0 is always visible, so mx is finite
       const bool grow = mx > m_ref + kPfLazy;                // also true on the first tile (m_ref = -inf)
       float alpha = 1.f;
@@ -322,31 +329,19 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         tc_fence_after_sync();
         if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll
-          for (int cc = 0; cc < D; cc += 32) {
-            float o[32];
-            tmem_ld32(lane_base + C::kOCol + (uint32_t)cc, o);
+          for (int cc = 0; cc < D; cc += 16) {
+            float o[16];
+            tmem_ld16(lane_base + C::kOCol + (uint32_t)cc, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] *= alpha;
-            tmem_st32(lane_base + C::kOCol + (uint32_t)cc, o);
+            for (int i = 0; i < 16; ++i) o[i] *= alpha;
+            tmem_st16(lane_base + C::kOCol + (uint32_t)cc, o);
           }
           tmem_wait_st();
         }
       }
       // ---- P = exp2(s*c - ref) as bf16 into shared memory, row sum in fp32
       float sm[4] = {0.f, 0.f, 0.f, 0.f};
-      static_assert(kPfKeys == 64, "both halves of the tile's logits are loaded before one wait");
-      float v[2][32];
-      tmem_ld32(s_addr, v[0]);
-      tmem_ld32(s_addr + 32u, v[1]);
-      tmem_wait_ld();
-      if (diag) {                                            // masked logits become -inf: their exponential is exactly 0
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (c_base + i > row_pos) v[0][i] = -INFINITY;
-          if (c_base + 32 + i > row_pos) v[1][i] = -INFINITY;
-        }
-      }
 #pragma unroll
       for (int cc = 0; cc < kPfKeys; cc += 32) {
         uint32_t packed[16];
