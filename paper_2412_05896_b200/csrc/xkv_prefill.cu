@@ -49,18 +49,43 @@ struct PfCfg {
   static constexpr int kQTileBytes = kHalves * kQHalfBytes;
   static constexpr int kKvHalfBytes = kPfKeys * 128;         // 64 columns of a K or V tile
   static constexpr int kKvTileBytes = kHalves * kKvHalfBytes;
-  static constexpr int kPHalfBytes = kPfRows * 128;          // 64 keys of P: rows of 128 bytes
-  static constexpr int kPBytes = (kPfKeys / 64) * kPHalfBytes;   // P: 128 rows x kPfKeys keys, bf16
   static constexpr int kKStages = 2;                         // S runs one tile ahead of the softmax
-  static constexpr int kVStages = 1;
+  static constexpr int kVStages = 2;
   static constexpr uint32_t kSCols = kPfKeys;                // one S buffer
   static constexpr uint32_t kOCol = 2 * kPfKeys;             // O accumulator starts here
   static constexpr uint32_t kTmemCols = 256;                 // two CTAs share an SM's 512 columns
-  static constexpr size_t kSmemBytes = 1024 + (size_t)kQTileBytes + (size_t)kKvTileBytes * (kKStages + kVStages) +
-                                       kPBytes + 256;
+  static constexpr size_t kSmemBytes = 1024 + (size_t)kQTileBytes + (size_t)kKvTileBytes * (kKStages + kVStages) + 256;
+  static_assert(2 * (kSmemBytes + 1024) <= 233472, "two CTAs per SM");
 };
 
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive 32-bit columns of this thread's TMEM lane from registers (here: 64 bf16 values of a row of P).
+__device__ __forceinline__ void tmem_st32u(uint32_t taddr, const uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem desc], bf16 inputs, fp32 accumulate; A is 128 rows (one per TMEM lane) of K-major
+// bf16 pairs, one pair per 32-bit column (16 K elements = 8 columns a step); issued by one thread.
+__device__ __forceinline__ void umma_bf16_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t"
+      "}\n" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
 
 // 16 consecutive fp32 columns of this thread's TMEM lane (the rescale of O works in these smaller pieces so that the
 // tile's logits can stay in registers beside it).
@@ -153,16 +178,14 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   uint8_t* q_s = smem;
   uint8_t* k_s = q_s + C::kQTileBytes;
   uint8_t* v_s = k_s + (size_t)C::kKStages * C::kKvTileBytes;
-  uint8_t* p_s = v_s + (size_t)C::kVStages * C::kKvTileBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(p_s + C::kPBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(v_s + (size_t)C::kVStages * C::kKvTileBytes);
   uint64_t* q_full = bars;             // [1]
   uint64_t* k_full = bars + 1;         // [2]
   uint64_t* k_empty = bars + 3;        // [2]
   uint64_t* v_full = bars + 5;         // [2]
   uint64_t* v_empty = bars + 7;        // [2]
   uint64_t* s_full = bars + 9;         // [2] S buffer complete (MMA -> softmax)
-  uint64_t* s_empty = bars + 11;       // [2] S buffer read (softmax -> MMA)
-  uint64_t* p_full = bars + 13;        // [1] P written, O rescaled (softmax -> MMA)
+  uint64_t* p_full = bars + 13;        // [1] P written over the tile's S buffer, O rescaled (softmax -> MMA)
   uint64_t* p_empty = bars + 14;       // [1] O += P V complete (MMA -> softmax)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 15);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
@@ -180,10 +203,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(&k_full[i], 1);
       mbar_init(&k_empty[i], 1);
       mbar_init(&s_full[i], 1);
-      mbar_init(&s_empty[i], 4);
+      mbar_init(&v_full[i], 1);
+      mbar_init(&v_empty[i], 1);
     }
-    mbar_init(v_full, 1);
-    mbar_init(v_empty, 1);
     mbar_init(p_full, 4);
     mbar_init(p_empty, 1);
     *s_abort = 0;
@@ -220,16 +242,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
     }
   } else if (warp == 6) {
-    // ------------------------------------------------------------------ producer of the V tiles (one stage)
+    // ------------------------------------------------------------------ producer of the V tiles (two stages)
     if (lane == 0) {
       bool ok = true;
       for (int j = 0; ok && j < n_kt; ++j) {
-        ok = ws_wait(v_empty, (j & 1u) ^ 1u, s_abort, p.wait_ns);
+        const uint32_t s = j & 1u;
+        ok = ws_wait(&v_empty[s], ((j >> 1) & 1u) ^ 1u, s_abort, p.wait_ns);
         if (!ok) break;
-        mbar_arrive_expect_tx(v_full, (uint32_t)C::kKvTileBytes);
+        mbar_arrive_expect_tx(&v_full[s], (uint32_t)C::kKvTileBytes);
 #pragma unroll
         for (int hf = 0; hf < C::kHalves; ++hf)
-          tma_load_3d(v_s + hf * C::kKvHalfBytes, &tmap_v, hf * 64, g, cu + j * kPfKeys, v_full);
+          tma_load_3d(v_s + (size_t)s * C::kKvTileBytes + hf * C::kKvHalfBytes, &tmap_v, hf * 64, g, cu + j * kPfKeys,
+                      &v_full[s]);
       }
     }
   } else if (warp == 5) {
@@ -237,11 +261,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     if (lane == 0) {
       bool ok = ws_wait(q_full, 0u, s_abort, p.wait_ns);
       const uint64_t q_desc = umma_desc_k128(smem_u32(q_s));
-      const uint64_t p_desc = umma_desc_k128(smem_u32(p_s));
       auto issue_qk = [&](int j) -> bool {
         const uint32_t s = j & 1u;
+        // S buffer s is free without a wait: P of tile j-2, the last thing held there, is read by that tile's
+        // O += P V, which this thread issued earlier and which therefore executes before these MMAs
         if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
-        if (!ws_wait(&s_empty[s], ((j >> 1) & 1u) ^ 1u, s_abort, p.wait_ns)) return false;
         tc_fence_after_sync();
         const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kKvTileBytes);
 #pragma unroll
@@ -261,18 +285,21 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           ok = issue_qk(j + 1);           // the next tile's logits run under this tile's softmax
           if (!ok) break;
         }
-        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(v_full, j & 1u, s_abort, p.wait_ns);
+        const uint32_t vs = j & 1u;
+        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(&v_full[vs], (j >> 1) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t v_base = smem_u32(v_s);
+        const uint32_t v_base = smem_u32(v_s) + vs * C::kKvTileBytes;
+        const uint32_t p_tmem = tmem_base + (j & 1u) * C::kSCols;      // P over the first columns of the tile's S buffer
 #pragma unroll
         for (int k = 0; k < kPfKeys / 16; ++k) {
-          // A: P[rows][keys 16k .. 16k+15], K-major; B: V[keys 16k ..][d], MN-major (16 keys = two 8-row groups)
-          const uint64_t pd = p_desc + (uint64_t)(((k / 4) * C::kPHalfBytes + (k % 4) * 32) >> 4);
+          // A: P[rows][keys 16k .. 16k+15] out of TMEM (eight columns of bf16 pairs); B: V[keys 16k ..][d], MN-major
+          // (16 keys = two 8-row groups)
           const uint64_t vd = umma_desc_mn128(v_base + k * 16 * 128, C::kKvHalfBytes);
-          umma_bf16(tmem_base + C::kOCol, pd, vd, umma_idesc_b_mn(kPfRows, D), (j > 0 || k > 0) ? 1u : 0u);
+          umma_bf16_a_tmem(tmem_base + C::kOCol, p_tmem + (uint32_t)(k * 8), vd, umma_idesc_b_mn(kPfRows, D),
+                           (j > 0 || k > 0) ? 1u : 0u);
         }
-        umma_commit(v_empty);
+        umma_commit(&v_empty[vs]);
         umma_commit(p_empty);
       }
     }
@@ -322,12 +349,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         m_ref = mx;
         l *= alpha;
       }
-      // ---- the previous tile's O += P V must be complete before P is overwritten or O rescaled
-      if (j > 0) {
+      // ---- O is rescaled only once the previous tile's O += P V is complete; a warp none of whose rows grew does
+      //      not wait for it (P of this tile goes to this tile's own S buffer)
+      if (j > 0 && __any_sync(0xffffffffu, grow)) {
         ok = __all_sync(0xffffffffu, ws_wait(p_empty, (j - 1) & 1u, s_abort, p.wait_ns));
         if (!ok) break;
         tc_fence_after_sync();
-        if (__any_sync(0xffffffffu, grow)) {
+        {
 #pragma unroll
           for (int cc = 0; cc < D; cc += 16) {
             float o[16];
@@ -340,11 +368,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           tmem_wait_st();
         }
       }
-      // ---- P = exp2(s*c - ref) as bf16 into shared memory, row sum in fp32
+      // ---- P = exp2(s*c - ref) as bf16 pairs over the first 32 columns of the tile's S buffer (the logits are in
+      //      registers by now), row sum in fp32
       float sm[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t packed[32];
 #pragma unroll
       for (int cc = 0; cc < kPfKeys; cc += 32) {
-        uint32_t packed[16];
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
           const float e0 = fast_exp2(fmaf(v[cc >> 5][i], p.scale_log2, -m_ref));
@@ -355,28 +384,18 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           sm[1] += e1;
           sm[2] += e2;
           sm[3] += e3;
-          packed[i >> 1] = pack_bf16(e0, e1);
-          packed[(i >> 1) + 1] = pack_bf16(e2, e3);
-        }
-        // 32 keys = four 16-byte pieces of the row's 128-byte line in half cc/64; piece index XOR (row & 7)
-        uint8_t* line = p_s + (cc >> 6) * C::kPHalfBytes + r * 128;
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int piece = ((cc & 63) >> 3) + q;
-          *reinterpret_cast<uint4*>(line + ((piece ^ (r & 7)) << 4)) =
-              make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+          packed[(cc + i) >> 1] = pack_bf16(e0, e1);
+          packed[((cc + i) >> 1) + 1] = pack_bf16(e2, e3);
         }
       }
+      tmem_st32u(s_addr, packed);
       const float sum = (sm[0] + sm[1]) + (sm[2] + sm[3]);
       l += sum;
-      // the S buffer has been read for the last time; P and O are ready for the MMA
+      // P and O are ready for the MMA
+      tmem_wait_st();
       tc_fence_before_sync();
-      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&s_empty[s]);
-        mbar_arrive(p_full);
-      }
+      if (lane == 0) mbar_arrive(p_full);
     }
     // ---- epilogue: O / l -> bf16, lse
     if (ok) ok = __all_sync(0xffffffffu, ws_wait(p_empty, (n_kt - 1) & 1u, s_abort, p.wait_ns));
