@@ -185,9 +185,11 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   uint64_t* v_full = bars + 5;         // [2]
   uint64_t* v_empty = bars + 7;        // [2]
   uint64_t* s_full = bars + 9;         // [2] S buffer complete (MMA -> softmax)
-  uint64_t* p_full = bars + 13;        // [1] P written over the tile's S buffer, O rescaled (softmax -> MMA)
-  uint64_t* p_empty = bars + 14;       // [1] O += P V complete (MMA -> softmax)
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 15);
+  // [2] P written over the tile's S buffer, O rescaled (softmax -> MMA), one barrier per S buffer: a softmax warp that
+  // does not have to rescale O may be a tile ahead of the others, and its arrival for tile j+1 must not count for tile j
+  uint64_t* p_full = bars + 13;
+  uint64_t* p_empty = bars + 15;       // [1] O += P V complete (MMA -> softmax)
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 16);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -206,7 +208,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(&v_full[i], 1);
       mbar_init(&v_empty[i], 1);
     }
-    mbar_init(p_full, 4);
+    mbar_init(&p_full[0], 4);
+    mbar_init(&p_full[1], 4);
     mbar_init(p_empty, 1);
     *s_abort = 0;
     fence_mbar_init();
@@ -286,7 +289,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           if (!ok) break;
         }
         const uint32_t vs = j & 1u;
-        ok = ws_wait(p_full, j & 1u, s_abort, p.wait_ns) && ws_wait(&v_full[vs], (j >> 1) & 1u, s_abort, p.wait_ns);
+        ok = ws_wait(&p_full[j & 1u], (j >> 1) & 1u, s_abort, p.wait_ns) &&
+             ws_wait(&v_full[vs], (j >> 1) & 1u, s_abort, p.wait_ns);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t v_base = smem_u32(v_s) + vs * C::kKvTileBytes;
@@ -395,7 +399,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       tmem_wait_st();
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
+      if (lane == 0) mbar_arrive(&p_full[s]);
     }
     // ---- epilogue: O / l -> bf16, lse
     if (ok) ok = __all_sync(0xffffffffu, ws_wait(p_empty, (n_kt - 1) & 1u, s_abort, p.wait_ns));

@@ -128,3 +128,27 @@ def test_score_lse_rejections():
     with pytest.raises(xkv.XkvError) as e:
         xkv.prefill_attn(sess2.dims, None, k.to(DEV), v.to(DEV), sess2.cu, 400, 400, out, None, ws)
     assert e.value.status == xkv.ERR_INVALID_ARG
+
+
+def test_prefill_attention_is_repeatable():
+    """The same call, many times: outputs and normalisers must be bit-identical every time (a hand-over between the
+    kernel's roles that depended on timing would show as a difference sooner or later)."""
+    require_lib()
+    lengths, Hq, Hkv, d, W = [3000, 1700, 900], 8, 2, 128, 32
+    q, k, v, _ = _prompt(123, lengths, Hq, Hkv, d, W)
+    T = sum(lengths)
+    sess = XkvSession(1, Hq, Hkv, d, W, 5, lengths, device=DEV)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    ws = torch.zeros(xkv.workspace_bytes(xkv.OP_PREFILL_ATTN, sess.dims), dtype=torch.uint8, device=DEV)
+    first = None
+    for rep in range(12):
+        out = torch.full((T, Hq, d), float("nan"), dtype=torch.bfloat16, device=DEV)
+        lse = torch.full((Hq, T), float("nan"), dtype=torch.float32, device=DEV)
+        xkv.prefill_attn(sess.dims, qd, kd, vd, sess.cu, T, max(lengths), out, lse, ws)
+        torch.cuda.synchronize()
+        assert xkv.read_device_status(ws) == xkv.OK
+        if first is None:
+            first = (out.clone(), lse.clone())
+        else:
+            assert torch.equal(out.view(torch.int16), first[0].view(torch.int16)), rep
+            assert torch.equal(lse.view(torch.int32), first[1].view(torch.int32)), rep
