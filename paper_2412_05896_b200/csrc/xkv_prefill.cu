@@ -188,8 +188,12 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   // [2] P written over the tile's S buffer, O rescaled (softmax -> MMA), one barrier per S buffer: a softmax warp that
   // does not have to rescale O may be a tile ahead of the others, and its arrival for tile j+1 must not count for tile j
   uint64_t* p_full = bars + 13;
-  uint64_t* p_empty = bars + 15;       // [1] O += P V complete (MMA -> softmax)
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 16);
+  // [2] O += P V of a tile complete (MMA -> softmax, and MMA -> its own next use of the S buffer), one barrier per S
+  // buffer as well: softmax warps wait here only when they rescale O and at the very end, so between two waits of a
+  // warp several products may complete, and with one barrier for all tiles the parity of "tile j-1 done" would also
+  // match "tile j-3 done"
+  uint64_t* p_empty = bars + 15;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 17);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -210,7 +214,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     mbar_init(&p_full[0], 4);
     mbar_init(&p_full[1], 4);
-    mbar_init(p_empty, 1);
+    mbar_init(&p_empty[0], 1);
+    mbar_init(&p_empty[1], 1);
     *s_abort = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_q);
@@ -266,8 +271,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const uint64_t q_desc = umma_desc_k128(smem_u32(q_s));
       auto issue_qk = [&](int j) -> bool {
         const uint32_t s = j & 1u;
-        // S buffer s is free without a wait: P of tile j-2, the last thing held there, is read by that tile's
-        // O += P V, which this thread issued earlier and which therefore executes before these MMAs
+        // S buffer s still holds P of tile j-2 until that tile's O += P V has read it: these MMAs, which overwrite
+        // it, wait for that product's completion (issue order alone does not protect an A operand in tensor memory)
+        if (j >= 2 && !ws_wait(&p_empty[s], (uint32_t)((j - 2) >> 1) & 1u, s_abort, p.wait_ns)) return false;
         if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
         tc_fence_after_sync();
         const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kKvTileBytes);
@@ -304,7 +310,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                            (j > 0 || k > 0) ? 1u : 0u);
         }
         umma_commit(&v_empty[vs]);
-        umma_commit(p_empty);
+        umma_commit(&p_empty[j & 1u]);
       }
     }
   } else {
@@ -356,7 +362,8 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       // ---- O is rescaled only once the previous tile's O += P V is complete; a warp none of whose rows grew does
       //      not wait for it (P of this tile goes to this tile's own S buffer)
       if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        ok = __all_sync(0xffffffffu, ws_wait(p_empty, (j - 1) & 1u, s_abort, p.wait_ns));
+        ok = __all_sync(0xffffffffu,
+                        ws_wait(&p_empty[(j - 1) & 1u], (uint32_t)((j - 1) >> 1) & 1u, s_abort, p.wait_ns));
         if (!ok) break;
         tc_fence_after_sync();
         {
@@ -402,7 +409,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       if (lane == 0) mbar_arrive(&p_full[s]);
     }
     // ---- epilogue: O / l -> bf16, lse
-    if (ok) ok = __all_sync(0xffffffffu, ws_wait(p_empty, (n_kt - 1) & 1u, s_abort, p.wait_ns));
+    if (ok)
+      ok = __all_sync(0xffffffffu,
+                      ws_wait(&p_empty[(n_kt - 1) & 1u], (uint32_t)((n_kt - 1) >> 1) & 1u, s_abort, p.wait_ns));
     if (ok) {
       tc_fence_after_sync();
       const float inv = l > 0.f ? 1.f / l : 0.f;
