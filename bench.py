@@ -450,6 +450,7 @@ def run_workload(ctx: Ctx, name: str, steps: int, warmup: int, headline: bool) -
             "peak_source": ctx.tf_src,
             "note": "4*d*Hq*sum_b t_b(t_b+1)/2 flops; outside the timed step (the model's own attention)"}
         lse_list = [lse_all[l] for l in range(L)]
+        time.sleep(1.0)      # as below: the scoring of the timed steps did not follow a long tensor-core phase either
         reps = 6
         for _ in range(2):
             sess.score_layers(q_win, k, lse=lse_list)
@@ -481,6 +482,7 @@ def run_workload(ctx: Ctx, name: str, steps: int, warmup: int, headline: bool) -
     # The same budgets, the kept rows stored as 8-bit integers with a scale per row (Sec. II-B: quantisation is compatible
     # with eviction): the second bandwidth lever.  Outside the timed region of the headline number.
     if world == 1 and not args.no_q8:
+        time.sleep(1.0)      # the prefill leg leaves the GPU at its power cap; compare with the timed steps' launches at like clocks
         q8 = ctx.XkvSession(L, w.n_q_heads, Hkv, d, W, w.pool_kernel, lengths, pool_mode=w.pool_mode,
                             max_new_tokens=n_dec, max_budget=w.n_max or None, total_budget=N_total,
                             curve_len=w.n_max or None, device=dev, decode_chunk_rows=args.chunk_rows,

@@ -271,9 +271,9 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const uint64_t q_desc = umma_desc_k128(smem_u32(q_s));
       auto issue_qk = [&](int j) -> bool {
         const uint32_t s = j & 1u;
-        // S buffer s still holds P of tile j-2 until that tile's O += P V has read it: these MMAs, which overwrite
-        // it, wait for that product's completion (issue order alone does not protect an A operand in tensor memory)
-        if (j >= 2 && !ws_wait(&p_empty[s], (uint32_t)((j - 2) >> 1) & 1u, s_abort, p.wait_ns)) return false;
+        // S buffer s is free without a wait: P of tile j-2, the last thing held there, is read by that tile's
+        // O += P V, which this thread issued earlier; one thread's MMAs execute in the order issued (the same
+        // ordering every accumulation chain over k-steps relies on), so these MMAs overwrite it afterwards
         if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
         tc_fence_after_sync();
         const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kKvTileBytes);
