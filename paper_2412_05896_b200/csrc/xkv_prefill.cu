@@ -5,15 +5,20 @@
 //
 // One CTA per (sequence, tile of 128 query rows, query head), 224 threads, key tiles of 64; two CTAs share an SM
 // (half of its shared memory and of its tensor memory each), so that one CTA's softmax runs under the other's MMAs:
-//   warps 0-3  softmax: thread = query row = TMEM lane.  Per key tile: row maximum out of TMEM, a reference
-//              maximum that is exact on the first tile and raised lazily afterwards (only when a logit exceeds
-//              it by 2^8, which is when the O accumulator in TMEM is rescaled: load, multiply, store),
-//              P = exp2(s*c - ref) rounded to bf16 into shared memory in the K-major 128-byte-swizzled layout
-//              the MMA reads as its A operand, row sum in fp32.  At the end O / l -> bf16 rows, lse.
-//   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles (two stages), and of the V tiles
-//              (one stage), so that a K tile never queues behind the V stage of an earlier tile
+//   warps 0-3  softmax: thread = query row = TMEM lane.  Per key tile: the row's 64 logits out of TMEM into registers
+//              (once), row maximum, a reference maximum that is exact on the first tile and raised lazily
+//              afterwards (only when a logit exceeds it by 2^8, which is when the warp waits for the previous
+//              O += P V and rescales the O accumulator in TMEM: load, multiply, store), P = exp2(s*c - ref) rounded
+//              to bf16 and stored as pairs over the first 32 columns of the tile's S buffer, where the MMA reads it
+//              as its A operand; row sum in fp32.  At the end O / l -> bf16 rows, lse.
+//   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles, and of the V tiles (two stages
+//              each), so that a K tile never queues behind the V stage of an earlier tile
 //   warp 5     MMA issuer (one lane): S = Q K^T into one of two 64-column TMEM buffers, one tile ahead of the
-//              softmax; O += P V with V as an MN-major B operand straight from its [keys][d] tile
+//              softmax; O += P V with P out of tensor memory and V as an MN-major B operand straight from its
+//              [keys][d] tile
+// Hand-overs between the roles go through one mbarrier per S buffer for each of "logits ready", "P ready" and
+// "product complete": a softmax warp may be a tile ahead of the others, and a warp that did not rescale for a while
+// has not waited for any product, so a single barrier counted over all tiles could take a later phase for an earlier.
 // Every wait is bounded; an expired wait sets the status word and lets the CTA drain.
 #include <atomic>
 
