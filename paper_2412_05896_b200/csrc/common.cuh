@@ -108,6 +108,16 @@ __device__ __forceinline__ uint32_t int8x2_to_f16x2(uint32_t word) {
       : "r"(word), "n"(kSelector));
   return r;
 }
+// The same without the subtraction: the two fp16 values are 1024 + stored byte = kInt8Bias + q.  A product summed
+// over such operands carries kInt8Bias times the sum of the other operand, which the caller removes once per output
+// instead of once per element (every value involved is an integer below 2048 times an fp16: exact until the fp32 sum).
+constexpr float kInt8Bias = 1152.f;
+template <uint32_t kSelector>
+__device__ __forceinline__ uint32_t int8x2_to_biased_f16x2(uint32_t word) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, 0x64646464, %2;" : "=r"(r) : "r"(word), "n"(kSelector));
+  return r;
+}
 // The eight bf16 of a 16-byte piece as fp32.
 __device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&x)[8]) {
   x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);

@@ -582,6 +582,19 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
     for (int mt = 0; mt < D / 16; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
     float m_ref[2] = {-3.0e38f, -3.0e38f};   // finite, so that (-inf) - m_ref stays -inf
     float l_part[2] = {0.f, 0.f};
+    // Q8: the stored bytes enter the MMAs as kInt8Bias + q.  q_bias[i] = kInt8Bias x (sum over d of the query of head
+    // 2*tig + i) comes off every logit; p_sum[i] gathers the weights P as the O^T MMAs see them, and kInt8Bias x p_sum
+    // comes off every element of O^T at the end.  Both sums are formed by the tensor core itself (an A operand of
+    // ones), so they are rounded exactly like the products they correct.
+    const uint32_t ones[4] = {0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u};
+    float q_bias[2] = {0.f, 0.f}, p_sum[4] = {0.f, 0.f, 0.f, 0.f};
+    if constexpr (Q8) {
+      float qs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) mma_f16_16816(qs, ones, qb[ks][0], qb[ks][1]);
+      q_bias[0] = kInt8Bias * qs[0];
+      q_bias[1] = kInt8Bias * qs[1];
+    }
 
     // S^T of one 16-row tile: rows gid (regs 0,1) and gid + 8 (regs 2,3), heads 2*tig, 2*tig + 1
     // Q8: address this lane hands to ldmatrix for row `row` (0..15) and 16-byte piece `piece` of a raw tile (rows of D
@@ -604,8 +617,10 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
             const int ks = 2 * j + half;
-            const uint32_t af[4] = {int8x2_to_f16x2<0x5140>(r[2 * half]), int8x2_to_f16x2<0x5140>(r[2 * half + 1]),
-                                    int8x2_to_f16x2<0x5342>(r[2 * half]), int8x2_to_f16x2<0x5342>(r[2 * half + 1])};
+            const uint32_t af[4] = {int8x2_to_biased_f16x2<0x5140>(r[2 * half]),
+                                    int8x2_to_biased_f16x2<0x5140>(r[2 * half + 1]),
+                                    int8x2_to_biased_f16x2<0x5342>(r[2 * half]),
+                                    int8x2_to_biased_f16x2<0x5342>(r[2 * half + 1])};
             if (half) mma_f16_16816(a1, af, qb[ks][0], qb[ks][1]);
             else      mma_f16_16816(a0, af, qb[ks][0], qb[ks][1]);
           }
@@ -626,7 +641,10 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
         // the rows' scales: keys gid (registers 0, 1) and gid + 8 (registers 2, 3)
         const float* kscale = raw_scales(s);
         const float s0 = kscale[gid], s1 = kscale[gid + 8];
-        acc[0] *= s0; acc[1] *= s0; acc[2] *= s1; acc[3] *= s1;
+        acc[0] = (acc[0] - q_bias[0]) * s0;
+        acc[1] = (acc[1] - q_bias[1]) * s0;
+        acc[2] = (acc[2] - q_bias[0]) * s1;
+        acc[3] = (acc[3] - q_bias[1]) * s1;
       }
     };
 
@@ -748,6 +766,12 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             o[mt][2] *= al0;
             o[mt][3] *= al1;
           }
+          if constexpr (Q8) {
+            p_sum[0] *= al0;
+            p_sum[1] *= al1;
+            p_sum[2] *= al0;
+            p_sum[3] *= al1;
+          }
         }
         const float p0 = fast_exp2(sv[0] - m_ref[0]), p1 = fast_exp2(sv[1] - m_ref[1]);
         const float p2 = fast_exp2(sv[2] - m_ref[0]), p3 = fast_exp2(sv[3] - m_ref[1]);
@@ -768,11 +792,14 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
             ldmatrix_x4_trans(r, raw_piece(vt, (mat & 1) * 8 + mrow, 2 * j + (mat >> 1)));
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-              const uint32_t af[4] = {int8x2_to_f16x2<0x5240>(r[2 * half]), int8x2_to_f16x2<0x5341>(r[2 * half]),
-                                      int8x2_to_f16x2<0x5240>(r[2 * half + 1]), int8x2_to_f16x2<0x5341>(r[2 * half + 1])};
+              const uint32_t af[4] = {int8x2_to_biased_f16x2<0x5240>(r[2 * half]),
+                                      int8x2_to_biased_f16x2<0x5341>(r[2 * half]),
+                                      int8x2_to_biased_f16x2<0x5240>(r[2 * half + 1]),
+                                      int8x2_to_biased_f16x2<0x5341>(r[2 * half + 1])};
               mma_f16_16816(o[2 * j + half], af, b0, b1);
             }
           }
+          mma_f16_16816(p_sum, ones, b0, b1);
         } else {
 #pragma unroll
           for (int mt = 0; mt < D / 16; ++mt) {
@@ -787,6 +814,15 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_cons
       fill();                                   // the stage just released takes the next tile
     }
 
+    if constexpr (Q8) {               // take the bias of the stored bytes off O^T (see p_sum above)
+#pragma unroll
+      for (int mt = 0; mt < D / 16; ++mt) {
+        o[mt][0] -= kInt8Bias * p_sum[0];
+        o[mt][1] -= kInt8Bias * p_sum[1];
+        o[mt][2] -= kInt8Bias * p_sum[0];
+        o[mt][3] -= kInt8Bias * p_sum[1];
+      }
+    }
     // ---- finish the work item: denominators of the lane's two heads over all rows
 #pragma unroll
     for (int x = 4; x < 32; x <<= 1) {
