@@ -30,7 +30,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int kPfThreads = 224;
+constexpr int kPfThreads = 256;
 constexpr int kPfRows = 128;          // query rows per CTA
 constexpr int kPfKeys = 64;           // keys per tile
 constexpr float kPfLazy = 8.f;        // log2 slack before the reference maximum is raised
@@ -270,16 +270,21 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
     }
   } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ issuer of the logit MMAs
+    // Two issuing threads, one per product: a `tcgen05.mma` holds its thread until the pipe (shared with the SM's
+    // other CTA) takes it, and with one thread for both products that time, not the softmax, set the pace of a tile.
     if (lane == 0) {
       bool ok = ws_wait(q_full, 0u, s_abort, p.wait_ns);
       const uint64_t q_desc = umma_desc_k128(smem_u32(q_s));
-      auto issue_qk = [&](int j) -> bool {
+      for (int j = 0; ok && j < n_kt; ++j) {
         const uint32_t s = j & 1u;
-        // S buffer s is free without a wait: P of tile j-2, the last thing held there, is read by that tile's
-        // O += P V, which this thread issued earlier; one thread's MMAs execute in the order issued (the same
-        // ordering every accumulation chain over k-steps relies on), so these MMAs overwrite it afterwards
-        if (!ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns)) return false;
+        // S buffer s holds P of tile j-2 until that tile's O += P V, issued by the other thread, has read it
+        if (j >= 2) {
+          ok = ws_wait(&p_empty[s], (uint32_t)((j - 2) >> 1) & 1u, s_abort, p.wait_ns);
+          if (!ok) break;
+        }
+        ok = ws_wait(&k_full[s], (j >> 1) & 1u, s_abort, p.wait_ns);
+        if (!ok) break;
         tc_fence_after_sync();
         const uint64_t k_desc = umma_desc_k128(smem_u32(k_s) + s * C::kKvTileBytes);
 #pragma unroll
@@ -291,14 +296,13 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
         umma_commit(&k_empty[s]);
         umma_commit(&s_full[s]);
-        return true;
-      };
-      if (ok) ok = issue_qk(0);
+      }
+    }
+  } else if (warp == 7) {
+    // ------------------------------------------------------------------ issuer of O += P V
+    if (lane == 0) {
+      bool ok = true;
       for (int j = 0; ok && j < n_kt; ++j) {
-        if (j + 1 < n_kt) {
-          ok = issue_qk(j + 1);           // the next tile's logits run under this tile's softmax
-          if (!ok) break;
-        }
         const uint32_t vs = j & 1u;
         ok = ws_wait(&p_full[j & 1u], (j >> 1) & 1u, s_abort, p.wait_ns) &&
              ws_wait(&v_full[vs], (j >> 1) & 1u, s_abort, p.wait_ns);
@@ -318,7 +322,7 @@ prefill_attn_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         umma_commit(&p_empty[j & 1u]);
       }
     }
-  } else {
+  } else if (warp < 4) {
     // ------------------------------------------------------------------ softmax warps 0..3
     const int r = tid;                                       // query row of the tile = TMEM lane
     const uint32_t lane_base = tmem_base + ((uint32_t)(32 * warp) << 16);
