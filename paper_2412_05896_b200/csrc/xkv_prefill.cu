@@ -3,7 +3,7 @@
 // rows are what the scoring step needs of W_attn (Alg. 2 step 1): with them xkv_score_lse forms the column
 // scores in one pass over the keys.
 //
-// One CTA per (sequence, tile of 128 query rows, query head), 224 threads, key tiles of 64; two CTAs share an SM
+// One CTA per (sequence, tile of 128 query rows, query head), 256 threads, key tiles of 64; two CTAs share an SM
 // (half of its shared memory and of its tensor memory each), so that one CTA's softmax runs under the other's MMAs:
 //   warps 0-3  softmax: thread = query row = TMEM lane.  Per key tile: the row's 64 logits out of TMEM into registers
 //              (once), row maximum, a reference maximum that is exact on the first tile and raised lazily
@@ -13,8 +13,9 @@
 //              as its A operand; row sum in fp32.  At the end O / l -> bf16 rows, lse.
 //   warps 4, 6 producers (one lane each): TMA loads of the Q tile and the K tiles, and of the V tiles (two stages
 //              each), so that a K tile never queues behind the V stage of an earlier tile
-//   warp 5     MMA issuer (one lane): S = Q K^T into one of two 64-column TMEM buffers, one tile ahead of the
-//              softmax; O += P V with P out of tensor memory and V as an MN-major B operand straight from its
+//   warps 5, 7 MMA issuers (one lane each), one per product: S = Q K^T into one of two 64-column TMEM buffers, one
+//              tile ahead of the softmax (and not before the product that last read P out of that buffer is
+//              complete); O += P V with P out of tensor memory and V as an MN-major B operand straight from its
 //              [keys][d] tile
 // Hand-overs between the roles go through one mbarrier per S buffer for each of "logits ready", "P ready" and
 // "product complete": a softmax warp may be a tile ahead of the others, and a warp that did not rescale for a while
